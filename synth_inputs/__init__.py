@@ -1,0 +1,146 @@
+"""Seeded synthetic inputs for the cross-attention path (no attention arithmetic here).
+
+The tests, ``bench.py`` and the smoke check draw every tensor from the counter-based
+generator in ``gen.c`` so that the CUDA path and the CPU oracle are fed identical
+bf16 bits.  Arrays are numpy ``uint16`` (bf16 bit patterns).
+
+The five workloads mirror the long-context inference profiling set-up of the
+paper (3B-class shapes, head dimension 128, 8 KV heads, contexts from 32K to 1M
+tokens, Section 4.4 / Section 4.1); real activations would need trained weights,
+so values are N(0,1) draws.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass, field
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gen.c")
+_LIB = os.path.join(_HERE, "libsynth_gen.so")
+_lib = None
+
+# tensor ids: one stream of random numbers per tensor
+TID_K, TID_V, TID_LENS, TID_Q0 = 1, 2, 3, 16  # Q of layer l uses TID_Q0 + l
+
+
+def build(force: bool = False) -> str:
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.run(["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC,
+                        "-lm"], check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        u64 = ctypes.c_uint64
+        lib.synth_raw_bits.argtypes = [u64, u64, u64]
+        lib.synth_raw_bits.restype = u64
+        lib.synth_normal_bf16.argtypes = [u64, u64, ctypes.c_double, u64, u64, ctypes.c_void_p]
+        lib.synth_normal_bf16.restype = None
+        _lib = lib
+    return _lib
+
+
+def normal_bf16(seed: int, tensor_id: int, count: int, mult: float = 1.0, first: int = 0,
+                out: np.ndarray | None = None) -> np.ndarray:
+    """bf16 bits of ``mult * N(0,1)`` for elements [first, first+count) of a tensor."""
+    if out is None:
+        out = np.empty(count, dtype=np.uint16)
+    assert out.dtype == np.uint16 and out.size == count and out.flags.c_contiguous
+    _load().synth_normal_bf16(seed, tensor_id, float(mult), first, count,
+                              ctypes.c_void_p(out.ctypes.data))
+    return out
+
+
+def raw_bits(seed: int, tensor_id: int, counter: int) -> int:
+    return int(_load().synth_raw_bits(seed, tensor_id, counter))
+
+
+def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32)
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = u + 0x7FFF + ((u >> 16) & 1)
+    return (u >> 16).astype(np.uint16)
+
+
+@dataclass
+class Workload:
+    """One seeded problem instance: shapes, lengths and the packed-layout offsets."""
+    name: str
+    B: int
+    Hq: int
+    Hkv: int
+    d: int
+    T: int
+    layers: int
+    seed: int
+    kv_len: np.ndarray          # [B] int32, includes the T new positions
+    k_mult: float = 1.0
+    cu: np.ndarray = field(init=False)
+
+    def __post_init__(self):
+        self.kv_len = np.asarray(self.kv_len, dtype=np.int32)
+        self.cu = np.zeros(self.B + 1, dtype=np.int32)
+        np.cumsum(self.kv_len, out=self.cu[1:])
+
+    @property
+    def total_tokens(self) -> int:
+        return int(self.cu[-1])
+
+    @property
+    def kv_elems(self) -> int:
+        return self.total_tokens * self.Hkv * self.d
+
+    @property
+    def kv_bytes(self) -> int:
+        """Algorithmic bytes of one layer call: every visible K and V element once."""
+        return 2 * self.kv_elems * 2
+
+    def make_q(self, layer: int) -> np.ndarray:
+        return normal_bf16(self.seed, TID_Q0 + layer, self.B * self.Hq * self.T * self.d).reshape(
+            self.B, self.Hq, self.T, self.d)
+
+    def make_k(self) -> np.ndarray:
+        return normal_bf16(self.seed, TID_K, self.kv_elems, mult=self.k_mult)
+
+    def make_v(self) -> np.ndarray:
+        return normal_bf16(self.seed, TID_V, self.kv_elems)
+
+
+def ragged_lengths(seed: int, B: int, lo: int, span: int) -> np.ndarray:
+    """N_i = lo + (draw_i mod span): seeded, not tile-aligned."""
+    return np.array([lo + raw_bits(seed, TID_LENS, i) % span for i in range(B)], dtype=np.int32)
+
+
+def workload(name: str) -> Workload:
+    """The five benchmark configurations (plus scaled-down variants for quick tests)."""
+    if name == "tiny":          # config 1
+        return Workload(name, B=1, Hq=4, Hkv=1, d=64, T=1, layers=2, seed=0, kv_len=[512])
+    if name == "3b_32k":        # config 2: keys scaled by 0.5 before rounding
+        return Workload(name, B=1, Hq=32, Hkv=8, d=128, T=1, layers=13, seed=1, kv_len=[32768],
+                        k_mult=0.5)
+    if name == "ragged":        # config 3: N_i uniform in [4096, 131072]
+        return Workload(name, B=16, Hq=32, Hkv=8, d=128, T=1, layers=1, seed=2,
+                        kv_len=ragged_lengths(2, 16, 4096, 126977))
+    if name == "1m":            # config 4
+        return Workload(name, B=1, Hq=32, Hkv=8, d=128, T=1, layers=13, seed=3, kv_len=[1048576])
+    if name == "chunk":         # config 5: 512 new rows appended after 262,144 cached keys
+        return Workload(name, B=2, Hq=32, Hkv=8, d=128, T=512, layers=1, seed=4,
+                        kv_len=[262144 + 512] * 2)
+    if name == "ragged_small":  # same recipe as config 3, 32x shorter
+        return Workload(name, B=16, Hq=32, Hkv=8, d=128, T=1, layers=1, seed=2,
+                        kv_len=ragged_lengths(2, 16, 128, 3969))
+    if name == "chunk_small":   # same recipe as config 5, shorter cache and chunk
+        return Workload(name, B=2, Hq=32, Hkv=8, d=128, T=160, layers=1, seed=4,
+                        kv_len=[1000 + 160, 777 + 160])
+    raise KeyError(name)
