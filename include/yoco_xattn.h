@@ -1,0 +1,160 @@
+/*
+ * yoco_xattn -- cross-decoder attention over the single shared K/V cache of the
+ * decoder-decoder architecture (Section 2.2, the cross-decoder equation block:
+ * Q^l = LN(X^l) W_Q^l,  Y^l = Attention(Q^l, K^, V^) + X^l, "standard multi-head
+ * attention", causal, grouped-query).  This library computes the Attention(...)
+ * term only:  O = softmax(scale * Q K^T + causal mask) V  per sequence and head.
+ *
+ * Every cross-decoder layer calls it with its own Q and the SAME K/V pointers
+ * (the cache is written once by the self-decoder and reused by all L/2 layers).
+ *
+ * C ABI, sm_100a only.  No call allocates or frees device memory, none
+ * synchronises the host with the device unless stated, none throws.
+ *
+ * ---------------------------------------------------------------------------
+ * Layouts (all tensors contiguous, bf16 = 16-bit bfloat bit patterns)
+ *
+ *   Q, O   [B, Hq, T, d]   device.  Query head h reads KV head h / G, G = Hq / Hkv.
+ *   K, V   packed device buffers.  Sequence i starts at TOKEN offset cu_kv[i];
+ *          inside a sequence the order is head-major [Hkv, N_i, d]:
+ *            element(i, c, j, e) = cu_kv[i]*Hkv*d + c*head_stride_i + j*d + e
+ *          head_stride_i = kv_head_stride if non-zero (a cache with spare
+ *          capacity per head; must be a multiple of d), else N_i*d (tight).
+ *          With equal lengths and tight packing this is [B, Hkv, N, d].
+ *          Both buffers must start on a 16-byte boundary.
+ *   kv_len[i] = N_i  counts ALL keys of sequence i including the T positions of
+ *          the current call (the self-decoder has already appended them).
+ *   Causal rule: query row t (0-based, T rows) sees keys j <= N_i - T + t.
+ *          T = 1 sees the whole cache.  A row with no visible key yields O = 0
+ *          and LSE = -inf.
+ *   LSE    [B, Hq, T] fp32, natural logarithm of sum_j exp(scale * q.k_j); optional.
+ *
+ * Ownership: every pointer is caller-owned and must stay valid until the
+ * stream has executed the call.  `stream` is a cudaStream_t passed as void*
+ * (NULL = legacy default stream).  Work is only enqueued; calls return
+ * immediately.  The workspace may be reused by the next call on the same
+ * stream; calls on different streams need different workspaces.
+ *
+ * Errors: every function returns YOCO_OK or a negative code.  Argument and
+ * shape checks happen before anything is enqueued.  A device-side bounded wait
+ * that ran out (never expected) is recorded in a status word inside the
+ * workspace and read back by yoco_xattn_status().
+ */
+#ifndef YOCO_XATTN_H_
+#define YOCO_XATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define YOCO_OK                        0
+#define YOCO_ERR_INVALID_ARG          (-1)  /* null pointer, negative size, misaligned buffer   */
+#define YOCO_ERR_UNSUPPORTED          (-2)  /* d not in {64,128}, Hq % Hkv != 0, G*T too large  */
+#define YOCO_ERR_WORKSPACE_TOO_SMALL  (-3)
+#define YOCO_ERR_CUDA                 (-4)  /* a CUDA call failed; see yoco_xattn_last_cuda_error */
+#define YOCO_ERR_TIMEOUT              (-5)  /* a bounded device-side wait expired               */
+
+#define YOCO_MODE_DECODE 0   /* split-KV kernel, G*T <= 16 query rows per KV head        */
+#define YOCO_MODE_CHUNK  1   /* tensor-core (tcgen05) kernel, any T >= 1                 */
+
+typedef struct yoco_xattn_shape {
+    int32_t B;               /* sequences                                                 */
+    int32_t Hq;              /* query heads                                               */
+    int32_t Hkv;             /* key/value heads, divides Hq                               */
+    int32_t d;               /* head dimension: 64 or 128                                 */
+    int32_t T;               /* query rows per sequence in this call                      */
+    float   scale;           /* 0 -> 1/sqrt(d)                                            */
+    int64_t kv_head_stride;  /* elements between KV heads of one sequence; 0 -> N_i*d     */
+    int32_t max_kv_len;      /* used as every N_i when kv_len_host is NULL                */
+    int32_t reserved;        /* must be 0                                                 */
+} yoco_xattn_shape;
+
+/* One unit of work: a contiguous key range of one (sequence, KV head) stream,
+ * executed by CTA group `group`; its partial result goes to slot `slot`. */
+typedef struct yoco_xattn_segment {
+    int32_t group;      /* CTA group that streams this range                              */
+    int32_t b;          /* sequence                                                       */
+    int32_t c;          /* KV head                                                        */
+    int32_t k_begin;    /* first key (multiple of tile_n)                                 */
+    int32_t k_end;      /* one past the last key (multiple of tile_n, or N_i)             */
+    int32_t slot;       /* partial-result slot; slots of one stream are consecutive       */
+} yoco_xattn_segment;
+
+typedef struct yoco_xattn_plan_info {
+    int32_t mode;            /* YOCO_MODE_*                                               */
+    int32_t tile_n;          /* keys per shared-memory tile                               */
+    int32_t tile_m;          /* query rows per CTA tile (16 decode, 128 chunk)            */
+    int32_t m_tiles;         /* row tiles per stream = ceil(G*T / tile_m)                 */
+    int32_t num_groups;      /* CTA groups; each streams one contiguous range of the flat
+                                (stream, key tile) space                                  */
+    int32_t num_ctas;        /* grid size = num_groups * m_tiles                          */
+    int32_t num_streams;     /* B * Hkv                                                   */
+    int32_t num_segments;    /* total work segments = number of partial slots             */
+    int32_t max_splits;      /* most segments any one stream was cut into                 */
+    int32_t needs_combine;   /* 0 when every stream has exactly one segment               */
+    int64_t total_tiles;     /* sum over streams of ceil(N_i / tile_n)                    */
+    int64_t workspace_bytes; /* what decode/chunk need for this problem                   */
+} yoco_xattn_plan_info;
+
+/* Split-count / tile heuristic (host only, integers only, deterministic).
+ * The flat space of (stream, key tile) pairs, streams ordered (b, c), is cut into
+ * num_groups contiguous ranges of equal tile count (+-1); a range that crosses a
+ * stream boundary becomes several segments.  num_groups = min(total_tiles,
+ * sm_count * groups_per_sm(mode)).  sm_count > 0 must be given (pure host call).
+ * kv_len_host: [B] or NULL (every N_i = shape->max_kv_len).
+ * segments_out: optional array of `capacity` entries; at most `capacity` are written,
+ * info->num_segments tells how many exist.  */
+int32_t yoco_xattn_plan(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
+                        int32_t sm_count, int32_t mode, yoco_xattn_plan_info* info,
+                        yoco_xattn_segment* segments_out, int32_t capacity);
+
+/* Workspace bytes for decode/chunk on this problem.  sm_count = 0 queries the
+ * current CUDA device (then YOCO_ERR_CUDA is possible).  Pure host otherwise. */
+int32_t yoco_xattn_workspace_size(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
+                                  int32_t sm_count, int32_t mode, size_t* bytes);
+
+/* Split-KV decode (flash-decoding style): a few query rows per KV head (G*T <= 16;
+ * typically T = 1, the next-token call of a cross-decoder layer) against the
+ * whole cache.  Runs the split kernel, then the merge when a stream was split.
+ *   Q, K, V, O, lse (may be NULL), workspace: device.  cu_kv_host: host [B+1] token
+ *   offsets, or NULL = prefix sums of kv_len (tight packing).  kv_len_host: host [B]
+ *   or NULL.  workspace: >= yoco_xattn_workspace_size(), 256-byte aligned.        */
+int32_t yoco_xattn_decode(const yoco_xattn_shape* shape, const void* Q, const void* K,
+                          const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
+                          void* O, float* lse, void* workspace, size_t workspace_bytes,
+                          void* stream);
+
+/* Multi-token chunk / full-sequence path: T new query rows per sequence, causal
+ * inside the chunk, as a dense contraction on the tcgen05 tensor cores (S = Q K^T
+ * and O = P V with accumulators in tensor memory).  Same arguments as decode; any
+ * T >= 1.  */
+int32_t yoco_xattn_chunk(const yoco_xattn_shape* shape, const void* Q, const void* K,
+                         const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
+                         void* O, float* lse, void* workspace, size_t workspace_bytes,
+                         void* stream);
+
+/* Stand-alone log-sum-exp merge of S partial attention results per row:
+ *   lse = log sum_s exp(lse_s),   O = sum_s exp(lse_s - lse) * O_s
+ * part_o [rows, S, d] fp32 (each O_s already normalised), part_lse [rows, S] fp32
+ * natural log, -inf marks an empty piece (weight 0; all empty -> O = 0, lse = -inf).
+ * O [rows, d] bf16, lse [rows] fp32 or NULL.  All device pointers.  d % 8 == 0, d <= 256.
+ * Also the local step of key-range sharding across GPUs (exchange partials, merge). */
+int32_t yoco_xattn_combine(int64_t rows, int32_t S, int32_t d, const float* part_o,
+                           const float* part_lse, void* O, float* lse, void* stream);
+
+/* Synchronises `stream`, reads the status word that the last decode/chunk call
+ * using `workspace` left, returns it (YOCO_OK or YOCO_ERR_TIMEOUT). */
+int32_t yoco_xattn_status(const void* workspace, void* stream);
+
+const char* yoco_xattn_strerror(int32_t code);
+
+/* cudaError_t (as int) of the most recent failing CUDA call on this thread, 0 if none. */
+int32_t yoco_xattn_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* YOCO_XATTN_H_ */

@@ -1,0 +1,152 @@
+"""Thin ctypes binding of the C-ABI library (argument marshalling only).
+
+Function names mirror ``include/yoco_xattn.h``.  Tensors are torch CUDA tensors (torch is used
+for device memory and streams only); lengths and offsets are host numpy int32 arrays.  There is
+no fallback: if the CUDA library has not been built, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libyoco_xattn.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+MODE_DECODE, MODE_CHUNK = 0, 1
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32),
+                ("d", ctypes.c_int32), ("T", ctypes.c_int32), ("scale", ctypes.c_float),
+                ("kv_head_stride", ctypes.c_int64), ("max_kv_len", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+class Segment(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("group", "b", "c", "k_begin", "k_end", "slot")]
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("mode", "tile_n", "tile_m", "m_tiles", "num_groups", "num_ctas", "num_streams",
+                 "num_segments", "max_splits", "needs_combine")] + \
+               [("total_tiles", ctypes.c_int64), ("workspace_bytes", ctypes.c_int64)]
+
+
+class YocoError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().yoco_xattn_strerror(code).decode()
+        if code == ERR_CUDA:
+            msg += f" [cudaError {lib().yoco_xattn_last_cuda_error()}]"
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libyoco_xattn.so; fails loudly when it is missing (there is no CPU path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with paper_2405_05254_b200.build.build_cuda_library()")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        L.yoco_xattn_plan.argtypes = [ctypes.POINTER(Shape), vp, i32, i32, ctypes.POINTER(PlanInfo), vp, i32]
+        L.yoco_xattn_workspace_size.argtypes = [ctypes.POINTER(Shape), vp, i32, i32, ctypes.POINTER(sz)]
+        run_args = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.yoco_xattn_decode.argtypes = run_args
+        L.yoco_xattn_chunk.argtypes = run_args
+        L.yoco_xattn_combine.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
+        L.yoco_xattn_status.argtypes = [vp, vp]
+        L.yoco_xattn_strerror.argtypes = [i32]
+        L.yoco_xattn_strerror.restype = ctypes.c_char_p
+        L.yoco_xattn_last_cuda_error.argtypes = []
+        for name in ("plan", "workspace_size", "decode", "chunk", "combine", "status", "last_cuda_error"):
+            getattr(L, "yoco_xattn_" + name).restype = i32
+        _lib = L
+    return _lib
+
+
+def make_shape(B, Hq, Hkv, d, T, scale=0.0, kv_head_stride=0, max_kv_len=0) -> Shape:
+    return Shape(B, Hq, Hkv, d, T, float(scale), int(kv_head_stride), int(max_kv_len), 0)
+
+
+def _host_i32(a):
+    if a is None:
+        return None, None
+    arr = np.ascontiguousarray(a, dtype=np.int32)
+    return arr, ctypes.c_void_p(arr.ctypes.data)
+
+
+def yoco_xattn_plan(shape: Shape, kv_len, sm_count: int, mode: int):
+    """Returns (PlanInfo, list of Segment) of the split/tile heuristic; host only."""
+    keep, p_len = _host_i32(kv_len)
+    info = PlanInfo()
+    rc = lib().yoco_xattn_plan(ctypes.byref(shape), p_len, sm_count, mode, ctypes.byref(info), None, 0)
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_plan")
+    segs = (Segment * max(1, info.num_segments))()
+    rc = lib().yoco_xattn_plan(ctypes.byref(shape), p_len, sm_count, mode, ctypes.byref(info),
+                               ctypes.cast(segs, ctypes.c_void_p), info.num_segments)
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_plan")
+    return info, list(segs)[: info.num_segments]
+
+
+def yoco_xattn_workspace_size(shape: Shape, kv_len, mode: int, sm_count: int = 0) -> int:
+    keep, p_len = _host_i32(kv_len)
+    out = ctypes.c_size_t(0)
+    rc = lib().yoco_xattn_workspace_size(ctypes.byref(shape), p_len, sm_count, mode, ctypes.byref(out))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_workspace_size")
+    return int(out.value)
+
+
+def _ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _stream_ptr(stream):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _run(fn_name, shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream):
+    keep_cu, p_cu = _host_i32(cu_kv)
+    keep_len, p_len = _host_i32(kv_len)
+    fn = getattr(lib(), fn_name)
+    rc = fn(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), p_cu, p_len, _ptr(O), _ptr(lse),
+            _ptr(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, fn_name)
+
+
+def yoco_xattn_decode(shape: Shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream=None) -> None:
+    """Enqueue split-KV decode attention (G*T <= 16 rows per KV head) on the stream."""
+    _run("yoco_xattn_decode", shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream)
+
+
+def yoco_xattn_chunk(shape: Shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream=None) -> None:
+    """Enqueue the multi-token (tcgen05) attention on the stream."""
+    _run("yoco_xattn_chunk", shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream)
+
+
+def yoco_xattn_combine(part_o, part_lse, O, lse=None, stream=None) -> None:
+    """Merge partials: part_o [rows,S,d] fp32, part_lse [rows,S] fp32 -> O [rows,d] bf16."""
+    rows, S, d = part_o.shape
+    rc = lib().yoco_xattn_combine(rows, S, d, _ptr(part_o), _ptr(part_lse), _ptr(O), _ptr(lse),
+                                  _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_combine")
+
+
+def yoco_xattn_status(workspace, stream=None) -> int:
+    """Synchronise the stream and return the device status word of the last call (0 = ok)."""
+    return int(lib().yoco_xattn_status(_ptr(workspace), _stream_ptr(stream)))

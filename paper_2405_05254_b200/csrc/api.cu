@@ -1,0 +1,336 @@
+// C ABI of the library: argument checks, plan cache, tensor maps, kernel launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstring>
+#include <list>
+#include <mutex>
+
+#include "kernels.h"
+#include "plan.h"
+#include "yoco_xattn.h"
+
+namespace yoco {
+namespace {
+
+thread_local int32_t g_last_cuda_error = 0;
+
+int32_t cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int32_t)e;
+    return YOCO_ERR_CUDA;
+}
+#define YOCO_CUDA_TRY(expr)                               \
+    do {                                                  \
+        cudaError_t e__ = (expr);                         \
+        if (e__ != cudaSuccess) return cuda_fail(e__);    \
+    } while (0)
+
+// ---- per-device state ---------------------------------------------------------------------
+constexpr int kMaxDevices = 64;
+struct DeviceState {
+    bool ready = false;
+    int sm_count = 0;
+};
+std::mutex g_mutex;
+DeviceState g_dev[kMaxDevices];
+
+int32_t device_state(DeviceState** out) {
+    int dev = 0;
+    YOCO_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return YOCO_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState& st = g_dev[dev];
+    if (!st.ready) {
+        int major = 0;
+        YOCO_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        if (major != 10) return YOCO_ERR_UNSUPPORTED;   // built for sm_100a only
+        YOCO_CUDA_TRY(cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev));
+        YOCO_CUDA_TRY(decode_kernel_setup());
+        YOCO_CUDA_TRY(chunk_kernel_setup());
+        st.ready = true;
+    }
+    *out = &st;
+    return YOCO_OK;
+}
+
+// ---- plan cache ---------------------------------------------------------------------------
+struct PlanKey {
+    yoco_xattn_shape shape;
+    int32_t sm_count, mode;
+    std::vector<int32_t> lens, cu;
+    bool operator==(const PlanKey& o) const {
+        return std::memcmp(&shape, &o.shape, sizeof shape) == 0 && sm_count == o.sm_count &&
+               mode == o.mode && lens == o.lens && cu == o.cu;
+    }
+};
+struct PlanEntry {
+    PlanKey key;
+    Plan plan;
+};
+std::list<PlanEntry> g_plans;   // most recently used first
+constexpr size_t kPlanCacheEntries = 16;
+
+// Returns a copy-free pointer valid until the entry is evicted; callers hold g_mutex only
+// inside this function, so they copy what they need out of the plan before returning to the
+// user (the launch path below finishes with the plan before it can be evicted by this thread;
+// other threads may evict it, hence the shared_ptr-free design keeps a local copy).
+int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t* lens, int32_t sm_count,
+                    int32_t mode, Plan& out) {
+    PlanKey key;
+    std::memset(&key.shape, 0, sizeof key.shape);
+    key.shape = s;
+    key.sm_count = sm_count;
+    key.mode = mode;
+    if (lens) key.lens.assign(lens, lens + s.B);
+    if (cu) key.cu.assign(cu, cu + s.B + 1);
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        for (auto it = g_plans.begin(); it != g_plans.end(); ++it)
+            if (it->key == key) {
+                g_plans.splice(g_plans.begin(), g_plans, it);
+                out = g_plans.front().plan;
+                return YOCO_OK;
+            }
+    }
+    Plan plan;
+    int32_t rc = make_plan(s, cu, lens, sm_count, mode, plan);
+    if (rc != YOCO_OK) return rc;
+    out = plan;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_plans.push_front(PlanEntry{std::move(key), std::move(plan)});
+    if (g_plans.size() > kPlanCacheEntries) g_plans.pop_back();
+    return YOCO_OK;
+}
+
+// ---- tensor maps ----------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int32_t get_encoder(EncodeTiledFn* fn) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!g_encode) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        YOCO_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q));
+        if (q != cudaDriverEntryPointSuccess || !sym) return cuda_fail(cudaErrorNotSupported);
+        g_encode = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    *fn = g_encode;
+    return YOCO_OK;
+}
+
+// 2-D bf16 map over a row-major [rows, d] matrix, box {64 channels, box_rows}, 128-byte swizzle.
+int32_t make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int32_t d, int32_t box_rows) {
+    EncodeTiledFn enc;
+    int32_t rc = get_encoder(&enc);
+    if (rc != YOCO_OK) return rc;
+    cuuint64_t gdim[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)d * 2};
+    cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+    return YOCO_OK;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const void* K, const void* V,
+            const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
+            void* workspace, size_t workspace_bytes, void* stream_v) {
+    if (!shape) return YOCO_ERR_INVALID_ARG;
+    int32_t rc = validate_shape(*shape, mode);
+    if (rc != YOCO_OK) return rc;
+    if (shape->B == 0) return YOCO_OK;
+    if (!Q || !K || !V || !O || !workspace) return YOCO_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) ||
+        !aligned(workspace, 256) || (lse && !aligned(lse, 4)))
+        return YOCO_ERR_INVALID_ARG;
+
+    DeviceState* dev = nullptr;
+    if ((rc = device_state(&dev)) != YOCO_OK) return rc;
+
+    Plan plan;
+    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, mode, plan)) != YOCO_OK)
+        return rc;
+    if ((int64_t)workspace_bytes < plan.info.workspace_bytes) return YOCO_ERR_WORKSPACE_TOO_SMALL;
+
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const float scale = shape->scale != 0.f ? shape->scale : 1.f / std::sqrt((float)shape->d);
+
+    // header (status word = 0) + work tables in one copy
+    {
+        std::vector<int32_t> blob(kWorkspaceHeaderBytes / 4 + plan.table.size(), 0);
+        std::copy(plan.table.begin(), plan.table.end(), blob.begin() + kWorkspaceHeaderBytes / 4);
+        YOCO_CUDA_TRY(cudaMemcpyAsync(ws, blob.data(), blob.size() * 4, cudaMemcpyHostToDevice, stream));
+    }
+    const int32_t* table = reinterpret_cast<const int32_t*>(ws + plan.ws_table);
+    float* part_lse = reinterpret_cast<float*>(ws + plan.ws_part_lse);
+    float* part_o = reinterpret_cast<float*>(ws + plan.ws_part_o);
+    int32_t* status = reinterpret_cast<int32_t*>(ws);
+
+    if (plan.info.num_segments > 0) {
+        if (mode == YOCO_MODE_DECODE) {
+            CUtensorMap tmK, tmV;
+            if ((rc = make_map_2d(&tmK, K, plan.kv_rows_extent, shape->d, kDecodeTileN)) != YOCO_OK) return rc;
+            if ((rc = make_map_2d(&tmV, V, plan.kv_rows_extent, shape->d, kDecodeTileN)) != YOCO_OK) return rc;
+            DecodeParams p{};
+            p.Q = static_cast<const __nv_bfloat16*>(Q);
+            p.O = static_cast<__nv_bfloat16*>(O);
+            p.lse = lse;
+            p.segments = reinterpret_cast<const DevSegment*>(table + plan.off_segments);
+            p.group_begin = table + plan.off_group_begin;
+            p.part_o = part_o;
+            p.part_lse = part_lse;
+            p.status = status;
+            p.scale_log2 = scale * 1.4426950408889634f;
+            p.T = shape->T;
+            p.rows_per_stream = plan.rows_per_stream;
+            p.d = shape->d;
+            YOCO_CUDA_TRY(launch_decode(p, tmK, tmV, plan.info.num_groups, stream));
+        } else {
+            CUtensorMap tmQ, tmK, tmV;
+            const int64_t q_rows = (int64_t)shape->B * shape->Hq * shape->T;
+            if ((rc = make_map_2d(&tmQ, Q, q_rows, shape->d, kChunkTileM)) != YOCO_OK) return rc;
+            if ((rc = make_map_2d(&tmK, K, plan.kv_rows_extent, shape->d, kChunkTileN)) != YOCO_OK) return rc;
+            if ((rc = make_map_2d(&tmV, V, plan.kv_rows_extent, shape->d, kChunkTileN)) != YOCO_OK) return rc;
+            ChunkParams p{};
+            p.O = static_cast<__nv_bfloat16*>(O);
+            p.lse = lse;
+            p.segments = reinterpret_cast<const DevSegment*>(table + plan.off_segments);
+            p.group_begin = table + plan.off_group_begin;
+            p.part_o = part_o;
+            p.part_lse = part_lse;
+            p.status = status;
+            p.scale_log2 = scale * 1.4426950408889634f;
+            p.T = shape->T;
+            p.rows_per_stream = plan.rows_per_stream;
+            p.m_tiles = plan.info.m_tiles;
+            p.d = shape->d;
+            YOCO_CUDA_TRY(launch_chunk(p, tmQ, tmK, tmV, plan.info.num_groups, stream));
+        }
+    }
+    if (plan.info.needs_combine) {
+        CombineParams c{};
+        c.rows = (int64_t)shape->B * shape->Hq * shape->T;
+        c.d = shape->d;
+        c.S = 0;
+        c.Hq = shape->Hq;
+        c.Hkv = shape->Hkv;
+        c.T = shape->T;
+        c.rows_per_stream = plan.rows_per_stream;
+        c.stream_base = table + plan.off_stream_base;
+        c.stream_nseg = table + plan.off_stream_nseg;
+        c.part_o = part_o;
+        c.part_lse = part_lse;
+        c.O = static_cast<__nv_bfloat16*>(O);
+        c.lse = lse;
+        YOCO_CUDA_TRY(launch_combine(c, stream));
+    }
+    return YOCO_OK;
+}
+
+}  // namespace
+}  // namespace yoco
+
+using namespace yoco;
+
+extern "C" {
+
+int32_t yoco_xattn_plan(const yoco_xattn_shape* shape, const int32_t* kv_len_host, int32_t sm_count,
+                        int32_t mode, yoco_xattn_plan_info* info, yoco_xattn_segment* segments_out,
+                        int32_t capacity) {
+    if (!shape || !info || capacity < 0 || (capacity > 0 && !segments_out)) return YOCO_ERR_INVALID_ARG;
+    Plan plan;
+    int32_t rc = make_plan(*shape, nullptr, kv_len_host, sm_count, mode, plan);
+    if (rc != YOCO_OK) return rc;
+    *info = plan.info;
+    const int32_t n = std::min<int32_t>(capacity, (int32_t)plan.segments.size());
+    for (int32_t k = 0; k < n; ++k) segments_out[k] = plan.segments[k];
+    return YOCO_OK;
+}
+
+int32_t yoco_xattn_workspace_size(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
+                                  int32_t sm_count, int32_t mode, size_t* bytes) {
+    if (!shape || !bytes || sm_count < 0) return YOCO_ERR_INVALID_ARG;
+    if (sm_count == 0) {
+        int32_t rc = validate_shape(*shape, mode);
+        if (rc != YOCO_OK) return rc;
+        DeviceState* dev = nullptr;
+        if ((rc = device_state(&dev)) != YOCO_OK) return rc;
+        sm_count = dev->sm_count;
+    }
+    Plan plan;
+    int32_t rc = make_plan(*shape, nullptr, kv_len_host, sm_count, mode, plan);
+    if (rc != YOCO_OK) return rc;
+    *bytes = (size_t)plan.info.workspace_bytes;
+    return YOCO_OK;
+}
+
+int32_t yoco_xattn_decode(const yoco_xattn_shape* shape, const void* Q, const void* K, const void* V,
+                          const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+    return run(shape, YOCO_MODE_DECODE, Q, K, V, cu_kv_host, kv_len_host, O, lse, workspace,
+               workspace_bytes, stream);
+}
+
+int32_t yoco_xattn_chunk(const yoco_xattn_shape* shape, const void* Q, const void* K, const void* V,
+                         const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+    return run(shape, YOCO_MODE_CHUNK, Q, K, V, cu_kv_host, kv_len_host, O, lse, workspace,
+               workspace_bytes, stream);
+}
+
+int32_t yoco_xattn_combine(int64_t rows, int32_t S, int32_t d, const float* part_o,
+                           const float* part_lse, void* O, float* lse, void* stream) {
+    if (rows < 0 || S <= 0 || d <= 0) return YOCO_ERR_INVALID_ARG;
+    if (d % 8 != 0 || d > 256) return YOCO_ERR_UNSUPPORTED;
+    if (rows == 0) return YOCO_OK;
+    if (!part_o || !part_lse || !O) return YOCO_ERR_INVALID_ARG;
+    if (!aligned(part_o, 16) || !aligned(part_lse, 4) || !aligned(O, 16)) return YOCO_ERR_INVALID_ARG;
+    if (d % 4 != 0) return YOCO_ERR_UNSUPPORTED;
+    CombineParams c{};
+    c.rows = rows;
+    c.d = d;
+    c.S = S;
+    c.stream_base = nullptr;
+    c.stream_nseg = nullptr;
+    c.part_o = part_o;
+    c.part_lse = part_lse;
+    c.O = static_cast<__nv_bfloat16*>(O);
+    c.lse = lse;
+    YOCO_CUDA_TRY(launch_combine(c, reinterpret_cast<cudaStream_t>(stream)));
+    return YOCO_OK;
+}
+
+int32_t yoco_xattn_status(const void* workspace, void* stream) {
+    if (!workspace) return YOCO_ERR_INVALID_ARG;
+    int32_t word = 0;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    YOCO_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost, s));
+    YOCO_CUDA_TRY(cudaStreamSynchronize(s));
+    return word == kStatusOk ? YOCO_OK : YOCO_ERR_TIMEOUT;
+}
+
+const char* yoco_xattn_strerror(int32_t code) {
+    switch (code) {
+        case YOCO_OK: return "ok";
+        case YOCO_ERR_INVALID_ARG: return "invalid argument";
+        case YOCO_ERR_UNSUPPORTED: return "unsupported shape or device";
+        case YOCO_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case YOCO_ERR_CUDA: return "CUDA call failed (see yoco_xattn_last_cuda_error)";
+        case YOCO_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown error code";
+    }
+}
+
+int32_t yoco_xattn_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"

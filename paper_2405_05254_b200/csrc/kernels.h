@@ -1,0 +1,76 @@
+// Launch interfaces of the kernels (device code lives in the *_kernel.cu files).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <cstdint>
+
+#include "plan.h"
+
+namespace yoco {
+
+// device status word values (first int32 of the workspace)
+constexpr int32_t kStatusOk = 0;
+constexpr int32_t kStatusTimeout = 1;
+
+struct CombineParams {
+    int64_t rows;               // output rows (B*Hq*T, or the public `rows`)
+    int32_t d;
+    // public layout ([rows][S][d]) when stream_base == nullptr
+    int32_t S;
+    // internal slot-major layout
+    int32_t Hq, Hkv, T, rows_per_stream;
+    const int32_t* stream_base; // [B*Hkv] first slot of each stream
+    const int32_t* stream_nseg; // [B*Hkv] slots of each stream
+    const float* part_o;
+    const float* part_lse;      // natural log, -inf = empty
+    __nv_bfloat16* O;
+    float* lse;                 // may be null
+};
+cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream);
+
+struct DecodeParams {
+    const __nv_bfloat16* Q;     // [B*Hq*T, d]
+    __nv_bfloat16* O;           // [B*Hq*T, d]
+    float* lse;                 // [B*Hq*T] or null
+    const DevSegment* segments;
+    const int32_t* group_begin; // [num_groups + 1]
+    float* part_o;              // [num_segments][rows_per_stream][d]
+    float* part_lse;            // [num_segments][rows_per_stream]
+    int32_t* status;
+    float scale_log2;           // scale * log2(e)
+    int32_t T;
+    int32_t rows_per_stream;    // G * T (<= 16)
+    int32_t d;
+};
+// tmK / tmV: 2-D tensor maps over the [rows, d] view of K and V, box {64, kDecodeTileN},
+// 128-byte swizzle.
+cudaError_t launch_decode(const DecodeParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                          int num_groups, cudaStream_t stream);
+// one-time per-device kernel attribute set-up (dynamic shared memory opt-in)
+cudaError_t decode_kernel_setup();
+
+
+struct ChunkParams {
+    __nv_bfloat16* O;           // [B*Hq*T, d]
+    float* lse;                 // [B*Hq*T] or null
+    const DevSegment* segments;
+    const int32_t* group_begin; // [num_groups + 1]
+    float* part_o;              // [num_segments][rows_per_stream][d]
+    float* part_lse;            // [num_segments][rows_per_stream]
+    int32_t* status;
+    float scale_log2;           // scale * log2(e)
+    int32_t T;
+    int32_t rows_per_stream;    // G * T
+    int32_t m_tiles;            // ceil(rows_per_stream / 128)
+    int32_t d;
+};
+// tmQ: [B*Hq*T, d] box {64, 128}; tmK / tmV: [rows, d] box {64, kChunkTileN}; 128-byte swizzle.
+// Grid = num_groups * m_tiles CTAs, the row tile varying fastest so that the CTAs that walk the
+// same K/V range run side by side and share it through L2.
+cudaError_t launch_chunk(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                         const CUtensorMap& tmV, int num_groups, cudaStream_t stream);
+cudaError_t chunk_kernel_setup();
+
+}  // namespace yoco

@@ -1,0 +1,212 @@
+"""Parity of the split-KV decode path (through the C ABI) against the fp64 oracle."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+from helpers import GpuRunner, assert_close, assert_lse_close, errors
+
+pytestmark = pytest.mark.gpu
+
+
+def oracle_full(w, Q, K, V, **kw):
+    return oracle.xattn(Q, K, V, w.cu, w.kv_len, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T, **kw)
+
+
+def run_workload(w, layers=None, mode="decode"):
+    K, V = w.make_k(), w.make_v()
+    r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, w.T, w.kv_len, K, V)
+    out = []
+    for l in range(w.layers if layers is None else layers):
+        Q = w.make_q(l)
+        o, lse, _ = r.run(Q, mode)
+        o_ref, lse_ref = oracle_full(w, Q, K, V)
+        out.append(assert_close(o, o_ref, f"{w.name} layer {l}"))
+        assert_lse_close(lse, lse_ref, f"{w.name} layer {l}")
+    return out
+
+
+def test_tiny_config_two_layers_share_one_cache():
+    run_workload(si.workload("tiny"))
+
+
+def test_3b_class_32k_all_thirteen_layers():
+    run_workload(si.workload("3b_32k"))
+
+
+def test_ragged_small_batch():
+    run_workload(si.workload("ragged_small"))
+
+
+@pytest.mark.parametrize("N", [1, 2, 15, 16, 17, 63, 64, 65, 127, 129, 1000, 4097])
+def test_lengths_around_tile_edges(N):
+    w = si.Workload("edge", B=2, Hq=8, Hkv=2, d=128, T=1, layers=1, seed=100 + N, kv_len=[N, max(1, N // 2)])
+    run_workload(w)
+
+
+@pytest.mark.parametrize("Hq,Hkv,T,d", [(24, 8, 1, 128), (8, 8, 1, 128), (32, 8, 2, 128), (32, 8, 4, 128),
+                                        (16, 1, 1, 128), (6, 2, 5, 64), (4, 4, 16, 64), (8, 2, 3, 128)])
+def test_group_sizes_and_small_chunks(Hq, Hkv, T, d):
+    """G = 3 (the paper's 24/8 heads), MHA, and T > 1 rows that are causal among themselves."""
+    w = si.Workload("grp", B=3, Hq=Hq, Hkv=Hkv, d=d, T=T, layers=1, seed=7, kv_len=[700, 64 + T, 333])
+    run_workload(w)
+
+
+def test_more_query_rows_than_keys_and_empty_sequences():
+    w = si.Workload("short", B=4, Hq=8, Hkv=2, d=128, T=4, layers=1, seed=8, kv_len=[2, 0, 4, 1])
+    K, V = w.make_k(), w.make_v()
+    Q = w.make_q(0)
+    r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, w.T, w.kv_len, K, V)
+    o, lse, _ = r.run(Q)
+    o_ref, lse_ref = oracle_full(w, Q, K, V)
+    assert_close(o, o_ref, "short")
+    assert_lse_close(lse, lse_ref, "short")
+    assert (o[1] == 0).all() and np.isneginf(lse[1]).all()        # empty sequence
+    assert (o[0, :, :2] == 0).all()                                # rows with no visible key
+
+
+def test_peaked_scores_exercise_the_rescale_path():
+    """A few keys late in the sequence with much larger scores force the running max to move."""
+    w = si.Workload("peaked", B=1, Hq=32, Hkv=8, d=128, T=1, layers=1, seed=9, kv_len=[20000])
+    K, V = w.make_k().reshape(8, 20000, 128).copy(), w.make_v()
+    Q = w.make_q(0)
+    qf = si.bf16_bits_to_f32(Q).reshape(8, 4, 128)
+    for c in range(8):
+        for n, (pos, gain) in enumerate([(5000, 0.4), (12345, 0.8), (19990, 1.2), (19999, 1.0)]):
+            K[c, pos] = si.f32_to_bf16_bits(gain * qf[c, n % 4])
+    r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, w.T, w.kv_len, K, V)
+    o, lse, _ = r.run(Q)
+    o_ref, lse_ref = oracle_full(w, Q, K.reshape(-1), V)
+    assert_close(o, o_ref, "peaked")
+    assert_lse_close(lse, lse_ref, "peaked")
+    assert np.abs(o_ref).max() > 0.5      # the peaks really dominate some heads
+
+
+def test_one_hot_selection_is_bit_exact_at_every_split_and_tile_edge():
+    """One key leads by > 150 in the exponent, so every other weight is exactly 0 in fp32 and the
+    output must equal that key's V bit for bit, wherever the key sits: first/last key of each
+    split, of each 64-key tile, of each warp's 16-key slice and of each ragged sequence."""
+    from paper_2405_05254_b200 import binding as bd
+    B, Hq, Hkv, d = 3, 8, 2, 128
+    lens = np.array([5000, 777, 64], dtype=np.int32)
+    w = si.Workload("onehot", B=B, Hq=Hq, Hkv=Hkv, d=d, T=1, layers=1, seed=10, kv_len=lens)
+    V = w.make_v()
+    shape = bd.make_shape(B, Hq, Hkv, d, 1)
+    _, segs = bd.yoco_xattn_plan(shape, lens, 148, bd.MODE_DECODE)
+    positions = {b: set() for b in range(B)}
+    for s in segs:
+        positions[s.b] |= {s.k_begin, s.k_end - 1}
+    for b in range(B):
+        n = int(lens[b])
+        positions[b] |= {0, n - 1, 15, 16, 63, 64} & set(range(n))
+    Q = si.f32_to_bf16_bits(np.full((B, Hq, 1, d), 16.0, dtype=np.float32))
+    Vf = si.bf16_bits_to_f32(V)
+    r = None
+    rounds = max(len(p) for p in positions.values())
+    for k in range(rounds):
+        K = np.zeros(w.kv_elems, dtype=np.float32)
+        picks = []
+        for b in range(B):
+            plist = sorted(positions[b])
+            j = plist[k % len(plist)]
+            picks.append(j)
+            for c in range(Hkv):
+                base = int(w.cu[b]) * Hkv * d + (c * int(lens[b]) + j) * d
+                K[base:base + d] = 8.0
+        r = GpuRunner(B, Hq, Hkv, d, 1, lens, si.f32_to_bf16_bits(K), V)
+        o, lse, _ = r.run(Q)
+        for b in range(B):
+            for h in range(Hq):
+                c = h // (Hq // Hkv)
+                base = int(w.cu[b]) * Hkv * d + (c * int(lens[b]) + picks[b]) * d
+                np.testing.assert_array_equal(o[b, h, 0], Vf[base:base + d].astype(np.float64),
+                                              err_msg=f"b={b} h={h} key={picks[b]}")
+        assert np.allclose(lse, 16 * 8 * d / math.sqrt(d), rtol=1e-6)
+
+
+def test_cache_with_spare_capacity_per_head_and_garbage_beyond_the_length():
+    """kv_head_stride > N*d; the slack rows hold NaN bit patterns and must not leak into O."""
+    B, Hq, Hkv, d, cap = 2, 8, 2, 128, 300
+    lens = np.array([257, 100], dtype=np.int32)
+    rng = np.random.default_rng(3)
+    K = np.full((B, Hkv, cap, d), 0x7FC0, dtype=np.uint16)    # NaN everywhere
+    V = np.full((B, Hkv, cap, d), 0x7FC0, dtype=np.uint16)
+    for b in range(B):
+        n = int(lens[b])
+        K[b, :, :n] = si.f32_to_bf16_bits(rng.standard_normal((Hkv, n, d)).astype(np.float32))
+        V[b, :, :n] = si.f32_to_bf16_bits(rng.standard_normal((Hkv, n, d)).astype(np.float32))
+    Q = si.f32_to_bf16_bits(rng.standard_normal((B, Hq, 1, d)).astype(np.float32))
+    cu = np.array([0, cap, 2 * cap], dtype=np.int32)
+    r = GpuRunner(B, Hq, Hkv, d, 1, lens, K, V, cu=cu, kv_head_stride=cap * d)
+    o, lse, _ = r.run(Q)
+    o_ref, lse_ref = oracle.xattn(Q, K, V, cu, lens, B=B, Hq=Hq, Hkv=Hkv, d=d, T=1, kv_head_stride=cap * d)
+    assert_close(o, o_ref, "capacity layout")
+    assert_lse_close(lse, lse_ref, "capacity layout")
+
+
+def test_explicit_scale_and_no_lse_output():
+    w = si.Workload("scale", B=1, Hq=8, Hkv=2, d=64, T=1, layers=1, seed=11, kv_len=[900])
+    K, V, Q = w.make_k(), w.make_v(), w.make_q(0)
+    r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, w.T, w.kv_len, K, V, scale=0.31)
+    o, _, _ = r.run(Q, want_lse=False)
+    o_ref, _ = oracle_full(w, Q, K, V, scale=0.31)
+    assert_close(o, o_ref, "explicit scale")
+
+
+def test_two_runs_are_bit_identical():
+    import torch
+    w = si.workload("ragged_small")
+    K, V, Q = w.make_k(), w.make_v(), w.make_q(0)
+    r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, w.T, w.kv_len, K, V)
+    _, _, O1 = r.run(Q)
+    a = O1.clone()
+    _, _, O2 = r.run(Q)
+    assert torch.equal(a.view(torch.int16), O2.view(torch.int16))
+
+
+def test_combine_entry_point_against_the_oracle():
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    rng = np.random.default_rng(12)
+    for rows, S, d in [(37, 5, 128), (4, 1, 64), (130, 40, 128), (3, 33, 256)]:
+        po = rng.standard_normal((rows, S, d)).astype(np.float32)
+        pl = (4 * rng.standard_normal((rows, S))).astype(np.float32)
+        pl[rng.random((rows, S)) < 0.2] = -np.inf
+        pl[0, :] = -np.inf
+        O = torch.empty((rows, d), dtype=torch.bfloat16, device="cuda")
+        L = torch.empty((rows,), dtype=torch.float32, device="cuda")
+        bd.yoco_xattn_combine(torch.from_numpy(po).cuda(), torch.from_numpy(pl).cuda(), O, L)
+        torch.cuda.synchronize()
+        o_ref, l_ref = oracle.combine(po, pl)
+        from helpers import bf16_dev_to_f64
+        assert_close(bf16_dev_to_f64(O).reshape(rows, d), o_ref, f"combine {rows}x{S}x{d}")
+        assert_lse_close(L.cpu().numpy(), l_ref, "combine lse")
+
+
+def test_combine_with_one_live_piece_is_a_bit_exact_pass_through():
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    rng = np.random.default_rng(13)
+    rows, S, d = 16, 7, 128
+    po = rng.standard_normal((rows, S, d)).astype(np.float32)
+    pl = np.full((rows, S), -np.inf, dtype=np.float32)
+    live = rng.integers(0, S, size=rows)
+    pl[np.arange(rows), live] = rng.standard_normal(rows).astype(np.float32) * 10
+    O = torch.empty((rows, d), dtype=torch.bfloat16, device="cuda")
+    bd.yoco_xattn_combine(torch.from_numpy(po).cuda(), torch.from_numpy(pl).cuda(), O)
+    want = torch.from_numpy(po[np.arange(rows), live]).bfloat16()
+    assert torch.equal(O.cpu().view(torch.int16), want.view(torch.int16))
+
+
+def test_undersized_workspace_is_refused():
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    shape = bd.make_shape(1, 32, 8, 128, 1, max_kv_len=4096)
+    t = torch.zeros(4096 * 8 * 128, dtype=torch.bfloat16, device="cuda")
+    q = torch.zeros(32 * 128, dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(512, dtype=torch.uint8, device="cuda")
+    with pytest.raises(bd.YocoError) as e:
+        bd.yoco_xattn_decode(shape, q, t, t, None, [4096], q.clone(), None, ws)
+    assert e.value.code == bd.ERR_WORKSPACE_TOO_SMALL

@@ -1,0 +1,164 @@
+"""Host-side checks (no GPU): the library loads, exports the declared symbols, validates
+arguments before touching CUDA, and the split/tile planner partitions the key space exactly."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2405_05254_b200 import binding as bd
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            src = open(os.path.join(ROOT, "include", fn)).read()
+            names |= set(re.findall(r"\b(yoco_xattn_[a-z_0-9]+)\s*\(", src))
+    return sorted(names)
+
+
+def test_library_exports_every_declared_symbol():
+    L = bd.lib()
+    syms = declared_symbols()
+    assert {"yoco_xattn_decode", "yoco_xattn_chunk", "yoco_xattn_combine", "yoco_xattn_plan",
+            "yoco_xattn_workspace_size", "yoco_xattn_status", "yoco_xattn_strerror"} <= set(syms)
+    for s in syms:
+        assert hasattr(L, s), f"{s} is declared in include/ but not exported"
+
+
+def test_strerror_covers_the_codes():
+    msgs = {bd.lib().yoco_xattn_strerror(c) for c in range(-5, 1)}
+    assert len(msgs) == 6 and b"unknown error code" not in msgs
+    assert bd.lib().yoco_xattn_strerror(-99) == b"unknown error code"
+
+
+def restated_plan(B, Hkv, lens, sm_count, mode, G, T):
+    """Test-side restatement of the rule: flat (stream, tile) space cut into equal ranges."""
+    tile_n = 64 if mode == bd.MODE_DECODE else 128
+    tile_m = 16 if mode == bd.MODE_DECODE else 128
+    m_tiles = -(-G * T // tile_m)
+    nts = [-(-int(n) // tile_n) for n in lens]
+    total = Hkv * sum(nts)
+    target = sm_count * 2 if mode == bd.MODE_DECODE else max(1, sm_count // m_tiles)
+    groups = max(1, min(target, total))
+    bounds = [p * total // groups for p in range(groups + 1)]
+    segs = []
+    flat = 0
+    for b in range(B):
+        for c in range(Hkv):
+            lo, hi = flat, flat + nts[b]
+            for p in range(groups):
+                a, e = max(lo, bounds[p]), min(hi, bounds[p + 1])
+                if a < e:
+                    segs.append((p, b, c, (a - lo) * tile_n, min((e - lo) * tile_n, int(lens[b]))))
+            flat = hi
+    return groups, m_tiles, segs
+
+
+CASES = [
+    dict(B=1, Hq=4, Hkv=1, d=64, T=1, lens=[512]),
+    dict(B=1, Hq=32, Hkv=8, d=128, T=1, lens=[32768]),
+    dict(B=1, Hq=32, Hkv=8, d=128, T=1, lens=[1048576]),
+    dict(B=16, Hq=32, Hkv=8, d=128, T=1, lens=list(range(4096, 4096 + 16 * 7919, 7919))),
+    dict(B=3, Hq=24, Hkv=8, d=128, T=2, lens=[1, 0, 65]),
+    dict(B=2, Hq=32, Hkv=8, d=128, T=512, lens=[262656, 262656]),
+    dict(B=2, Hq=32, Hkv=8, d=128, T=160, lens=[1160, 937]),
+]
+
+
+@pytest.mark.parametrize("case", CASES)
+@pytest.mark.parametrize("sm_count", [148, 7])
+def test_plan_partitions_every_stream_exactly(case, sm_count):
+    G = case["Hq"] // case["Hkv"]
+    modes = [bd.MODE_CHUNK] + ([bd.MODE_DECODE] if G * case["T"] <= 16 else [])
+    for mode in modes:
+        shape = bd.make_shape(case["B"], case["Hq"], case["Hkv"], case["d"], case["T"])
+        info, segs = bd.yoco_xattn_plan(shape, case["lens"], sm_count, mode)
+        groups, m_tiles, want = restated_plan(case["B"], case["Hkv"], case["lens"], sm_count, mode, G, case["T"])
+        assert info.num_groups == groups and info.m_tiles == m_tiles
+        assert info.num_ctas == groups * m_tiles
+        got = [(s.group, s.b, s.c, s.k_begin, s.k_end) for s in segs]
+        assert got == want                                     # integer for integer
+        assert [s.slot for s in segs] == list(range(len(segs)))  # unique, consecutive slots
+        # partition: no gap, no overlap, in order
+        for b in range(case["B"]):
+            for c in range(case["Hkv"]):
+                mine = [s for s in segs if s.b == b and s.c == c]
+                pos = 0
+                for s in mine:
+                    assert s.k_begin == pos and s.k_end > s.k_begin and s.k_begin % info.tile_n == 0
+                    pos = s.k_end
+                assert pos == case["lens"][b]
+                if mine:
+                    assert [s.slot for s in mine] == list(range(mine[0].slot, mine[0].slot + len(mine)))
+        # balance: every group streams the same number of tiles (+-1)
+        tiles = {}
+        for s in segs:
+            tiles[s.group] = tiles.get(s.group, 0) + -(-(s.k_end - s.k_begin) // info.tile_n)
+        if tiles:
+            assert max(tiles.values()) - min(tiles.values()) <= 1
+        assert info.max_splits == max([0] + [sum(1 for s in segs if (s.b, s.c) == bc)
+                                             for bc in {(s.b, s.c) for s in segs}])
+        # determinism
+        info2, segs2 = bd.yoco_xattn_plan(shape, case["lens"], sm_count, mode)
+        assert bytes(info) == bytes(info2) and [bytes(s) for s in segs] == [bytes(s) for s in segs2]
+        assert bd.yoco_xattn_workspace_size(shape, case["lens"], mode, sm_count=sm_count) == info.workspace_bytes
+
+
+def test_one_million_tokens_fills_the_machine_in_one_wave():
+    shape = bd.make_shape(1, 32, 8, 128, 1)
+    info, segs = bd.yoco_xattn_plan(shape, [1048576], 148, bd.MODE_DECODE)
+    assert info.num_groups == 296 and info.total_tiles == 8 * 16384
+    assert info.needs_combine == 1 and info.num_segments <= 296 + 8
+
+
+def test_unsplit_streams_need_no_combine():
+    shape = bd.make_shape(400, 8, 8, 128, 1)
+    info, _ = bd.yoco_xattn_plan(shape, [64] * 400, 148, bd.MODE_DECODE)
+    assert info.needs_combine == 0 and info.max_splits == 1
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(d=96), bd.ERR_UNSUPPORTED),
+    (dict(Hq=30), bd.ERR_UNSUPPORTED),
+    (dict(T=5), bd.ERR_UNSUPPORTED),           # G*T = 20 rows > 16 in decode mode
+    (dict(T=0), bd.ERR_INVALID_ARG),
+    (dict(B=-1), bd.ERR_INVALID_ARG),
+    (dict(kv_head_stride=100), bd.ERR_UNSUPPORTED),
+])
+def test_bad_shapes_are_rejected_on_the_host(kw, code):
+    args = dict(B=1, Hq=32, Hkv=8, d=128, T=1)
+    args.update(kw)
+    shape = bd.make_shape(**args)
+    with pytest.raises(bd.YocoError) as e:
+        bd.yoco_xattn_plan(shape, [100], 148, bd.MODE_DECODE)
+    assert e.value.code == code
+
+
+def test_negative_length_and_short_head_stride_are_invalid():
+    shape = bd.make_shape(1, 8, 8, 128, 1)
+    with pytest.raises(bd.YocoError) as e:
+        bd.yoco_xattn_plan(shape, [-3], 148, bd.MODE_DECODE)
+    assert e.value.code == bd.ERR_INVALID_ARG
+    shape = bd.make_shape(1, 8, 8, 128, 1, kv_head_stride=128 * 10)
+    with pytest.raises(bd.YocoError) as e:
+        bd.yoco_xattn_plan(shape, [11], 148, bd.MODE_DECODE)
+    assert e.value.code == bd.ERR_INVALID_ARG
+
+
+def test_null_and_misaligned_pointers_fail_before_any_cuda_call():
+    L = bd.lib()
+    shape = bd.make_shape(1, 8, 8, 128, 1, max_kv_len=64)
+    f = L.yoco_xattn_decode
+    assert f(ctypes.byref(shape), None, None, None, None, None, None, None, None, 0, None) == bd.ERR_INVALID_ARG
+    assert f(None, None, None, None, None, None, None, None, None, 0, None) == bd.ERR_INVALID_ARG
+    p = ctypes.c_void_p
+    assert f(ctypes.byref(shape), p(4096), p(4096 + 2), p(8192), None, None, p(4096), None, p(4096), 1 << 20,
+             None) == bd.ERR_INVALID_ARG
+    assert L.yoco_xattn_combine(4, 0, 128, None, None, None, None, None) == bd.ERR_INVALID_ARG
+    assert L.yoco_xattn_combine(4, 2, 100, p(4096), p(4096), p(4096), None, None) == bd.ERR_UNSUPPORTED
+    assert L.yoco_xattn_combine(4, 2, 128, None, p(4096), p(4096), None, None) == bd.ERR_INVALID_ARG
