@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the cross-decoder attention hot path (decode over the shared K/V cache).
+
+One step = one generated token's pass through the cross-decoder's attention: L/2 = 13
+sequential layer calls (plan -> split-KV decode kernel -> LSE combine), each with its own
+Q over the SAME 1M-token K/V cache (Section 2.2; the 3B profiling set-up of Section 4.4).
+The metric is the rate at which the cache is streamed: KV GB/s = visible K+V bytes per
+layer call / time, with microseconds per token-layer next to it.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 1m]
+
+N > 1 is launched by torchrun (one rank per GPU); every rank runs an independent replica
+(its own cache, no data-path collective), times are max over ranks, value is the sum.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+
+METRIC = "cross-attn decode KV GB/s at 1M ctx (us/token-layer alongside)"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)", d
+    return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)", {}
+
+
+def ncu_traffic_per_launch(workload: str, kv_bytes: int):
+    """DRAM bytes per launch of the decode kernel from the committed ncu capture, scaled by
+    the K/V bytes of this workload (traffic grows in proportion to the keys streamed)."""
+    p = os.path.join(ROOT, "profiles", "decode_kernel_traffic.json")
+    if not os.path.exists(p):
+        return None
+    with open(p) as f:
+        d = json.load(f)
+    return float(d["dram_bytes_per_launch"]) * kv_bytes / float(d["kv_bytes_per_launch"])
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled in the background during the run."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(prefix="clocks_", suffix=".csv")
+        self.proc = None
+        self.gpu_index = gpu_index
+        try:
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={gpu_index}", f"--query-gpu=timestamp,{self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.out.close()
+        import datetime
+        rows = []
+        with open(self.path) as f:
+            for line in f:
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 10:
+                    continue
+                try:
+                    ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(parts[2]), float(parts[3]), parts[6:10]))
+                except ValueError:
+                    continue
+        os.unlink(self.path)
+        window = "timed region"
+        sel = [r for r in rows if t0 <= r[0] <= t1]
+        if len(sel) < 3:
+            sel, window = rows, "whole run (timed region shorter than 3 samples)"
+        if not sel:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({names[k] for r in sel for k in range(4) if r[3][k].lower().startswith("active")})
+        return {"sm_mhz": statistics.median(r[1] for r in sel), "sm_max_mhz": max(r[2] for r in sel),
+                "reasons": reasons, "samples": len(sel), "window": window}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ------------------------------------------------------------------------------------------
+def oracle_sample_rate(w, Q_layers, K, V, seconds_hint=None):
+    """Times the oracle, as it stands, on one KV-head group of one layer (G query heads, every
+    key of that head): returns (KV GB/s, seconds, description, threads)."""
+    import oracle
+    G = w.Hq // w.Hkv
+    rows = np.array([(b, h, t) for b in range(w.B) for h in range(G) for t in range(w.T)], dtype=np.int32)
+    t0 = time.perf_counter()
+    oracle.xattn_rows(Q_layers[0], K, V, w.cu, w.kv_len, rows, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T)
+    dt = time.perf_counter() - t0
+    sample_bytes = w.kv_bytes / w.Hkv
+    return sample_bytes / dt / 1e9, dt, (f"one layer call restricted to KV head 0 ({G} query heads x all "
+                                         f"{w.total_tokens} keys = 1/{w.Hkv} of a layer call)"), oracle.num_threads()
+
+
+def run_reference(args):
+    """The oracle timed on the host cores (the reference arm of this tier)."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    w = si.workload(args.workload)
+    K, V = w.make_k(), w.make_v()
+    Qs = [w.make_q(l) for l in range(w.layers)]
+    G = w.Hq // w.Hkv
+    rows = np.array([(b, h, t) for b in range(w.B) for h in range(G) for t in range(w.T)], dtype=np.int32)
+    kw = dict(B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T)
+    sample_bytes = w.kv_bytes / w.Hkv
+
+    def step(k):
+        oracle.xattn_rows(Qs[k % w.layers], K, V, w.cu, w.kv_len, rows, **kw)
+
+    for k in range(args.warmup):
+        step(k)
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        step(k)
+    dt = time.perf_counter() - t0
+    per_sample = dt / args.steps
+    gbs = sample_bytes / per_sample / 1e9
+    us_tl = per_sample * w.Hkv / w.B * 1e6
+    sample = (f"each step = one layer call restricted to KV head 0 ({G} query heads x all "
+              f"{w.total_tokens} keys, 1/{w.Hkv} of a layer call); ms_per_step extrapolated x{w.Hkv} x{w.layers} layers")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_sample * w.Hkv * w.layers * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "us_per_token_layer": us_tl,
+        "config": workload_config(w, 1),
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w, n_gpus):
+    return {"workload": f"{w.name}: B={w.B} Hq={w.Hq} Hkv={w.Hkv} d={w.d} T={w.T} kv_len={int(w.kv_len.max())} "
+                        f"x {w.layers} cross-decoder layers sharing one K/V cache (seed {w.seed})",
+            "kv_bytes_per_layer_call": w.kv_bytes, "layers_per_step": w.layers,
+            "l2": "inputs larger than L2 (K+V streamed per call >> 126 MB)" if w.kv_bytes > 4 * 126e6
+                  else "L2 flushed between timed calls by writing a 512 MB buffer",
+            "parallelism": f"replicas x{n_gpus} (one cache per GPU, no collective)"}
+
+
+def run_ours(args):
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+
+    rank, local_rank, world = dist_env()
+    if world != args.gpus:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("--gpus N > 1 must be launched with torchrun (one rank per GPU)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+
+    w = si.workload(args.workload)
+    w.seed = w.seed + 1000 * rank          # every replica has its own cache contents
+    Kh, Vh = w.make_k(), w.make_v()
+    K = torch.from_numpy(Kh.view(np.int16)).to(dev).view(torch.bfloat16)
+    V = torch.from_numpy(Vh.view(np.int16)).to(dev).view(torch.bfloat16)
+    Qh = [w.make_q(l) for l in range(w.layers)]
+    Qd = [torch.from_numpy(q.view(np.int16)).to(dev).view(torch.bfloat16) for q in Qh]
+    n_rows = w.B * w.Hq * w.T
+    Od = [torch.empty(n_rows * w.d, dtype=torch.bfloat16, device=dev) for _ in range(w.layers)]
+    shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(w.kv_len.max()))
+    mode = bd.MODE_DECODE
+    ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, mode), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    small = w.kv_bytes <= 4 * 126e6
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if small else None
+
+    def one_step():
+        for l in range(w.layers):
+            if flush is not None:
+                flush.fill_(l)
+            bd.yoco_xattn_decode(shape, Qd[l], K, V, w.cu, w.kv_len, Od[l], None, ws, stream)
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    assert bd.yoco_xattn_status(ws) == 0
+
+    # ---- device-resident timing: K steps, CUDA events, barrier + synchronize on both sides ----
+    records = args.steps * w.layers
+    bd.yoco_xattn_profile_enable(records)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        one_step()
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    barrier()
+    total_ms = ev0.elapsed_time(ev1)
+    kernel_ms = bd.yoco_xattn_profile_collect(records)
+    bd.yoco_xattn_profile_enable(0)
+    if flush is not None:
+        # the flush writes sit inside the event bracket; report the attention calls alone
+        total_ms = float(kernel_ms.sum()) if len(kernel_ms) else total_ms
+    assert bd.yoco_xattn_status(ws) == 0
+
+    # ---- end to end through the same entry point with HOST Q / O buffers ----
+    Qp = [torch.from_numpy(q.reshape(-1).view(np.int16)).view(torch.bfloat16).pin_memory() for q in Qh]
+    Op = [torch.empty(n_rows * w.d, dtype=torch.bfloat16).pin_memory() for _ in range(w.layers)]
+    new_kv_row = torch.from_numpy(Kh[-w.d:].view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    Qs = torch.empty(n_rows * w.d, dtype=torch.bfloat16, device=dev)
+
+    def one_step_e2e():
+        # the new token's K/V row of the last head lands in the cache, then 13 dependent layer
+        # calls: Q_l host -> device, attention, O_l device -> host (the next layer needs it)
+        K[-w.d:].copy_(new_kv_row, non_blocking=True)
+        V[-w.d:].copy_(new_kv_row, non_blocking=True)
+        for l in range(w.layers):
+            Qs.copy_(Qp[l], non_blocking=True)
+            bd.yoco_xattn_decode(shape, Qs, K, V, w.cu, w.kv_len, Od[l], None, ws, stream)
+            Op[l].copy_(Od[l], non_blocking=True)
+            stream.synchronize()
+
+    e2e_steps = max(3, min(args.steps, 50))
+    for _ in range(2):
+        one_step_e2e()
+    barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        one_step_e2e()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(times, op=torch.distributed.ReduceOp.MAX)
+    total_ms, e2e_ms = (float(x) for x in times.cpu())
+
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+
+    if rank == 0:
+        calls = args.steps * w.layers
+        bytes_all = w.kv_bytes * calls * world
+        value = bytes_all / (total_ms * 1e-3) / 1e9
+        ms_per_step = total_ms / args.steps
+        us_tl = total_ms * 1e3 / calls / w.B
+        peak, peak_src, peaks = measured_peaks()
+        k_avg_ms = float(kernel_ms.mean()) if len(kernel_ms) else float("nan")
+        achieved = w.kv_bytes / (k_avg_ms * 1e-3) / 1e9
+        traffic = ncu_traffic_per_launch(w.name, w.kv_bytes)
+        e2e_value = w.kv_bytes * e2e_steps * w.layers * world / (e2e_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "us_per_token_layer": us_tl,
+            "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
+            "config": workload_config(w, world),
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": "GB/s",
+                    "h2d_bytes_per_step": w.layers * n_rows * w.d * 2 + 2 * w.d * 2,
+                    "d2h_bytes_per_step": w.layers * n_rows * w.d * 2,
+                    "steps": e2e_steps, "us_per_token_layer": e2e_ms * 1e3 / (e2e_steps * w.layers) / w.B,
+                    "note": "Q_l and O_l live in pinned host memory and cross PCIe every layer with a "
+                            "stream sync per layer; the K/V cache is device-resident state (it is a cache)"},
+            "gpu_launches": 2 * calls,
+            "roofline": {"bound": "hbm", "kernel": "decode_kernel (split-KV)", "achieved": achieved,
+                         "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+                         "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+                         "kernel_us": k_avg_ms * 1e3, "algorithmic_bytes_per_launch": w.kv_bytes,
+                         "traffic": traffic},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            gbs, dt, sample, cores = oracle_sample_rate(w, Qh, Kh, Vh)
+            line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                                    "sample": sample, "seconds": dt,
+                                    "us_per_token_layer": dt * w.Hkv / w.B * 1e6}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="1m", choices=["1m", "3b_32k", "ragged", "tiny"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

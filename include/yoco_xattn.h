@@ -149,6 +149,14 @@ int32_t yoco_xattn_combine(int64_t rows, int32_t S, int32_t d, const float* part
  * using `workspace` left, returns it (YOCO_OK or YOCO_ERR_TIMEOUT). */
 int32_t yoco_xattn_status(const void* workspace, void* stream);
 
+/* Measurement aid (no counterpart in the paper).  After yoco_xattn_profile_enable(n), each of
+ * the next n decode/chunk calls records a CUDA event pair on its stream around the attention
+ * kernel alone (not the merge, not the table upload).  yoco_xattn_profile_collect waits for the
+ * recorded pairs, writes their durations in milliseconds (at most `capacity`), stores how many
+ * in *count and rearms the same n pairs.  enable(0) switches it off and frees the events. */
+int32_t yoco_xattn_profile_enable(int32_t max_records);
+int32_t yoco_xattn_profile_collect(float* kernel_ms, int32_t capacity, int32_t* count);
+
 const char* yoco_xattn_strerror(int32_t code);
 
 /* cudaError_t (as int) of the most recent failing CUDA call on this thread, 0 if none. */

@@ -64,10 +64,13 @@ def lib() -> ctypes.CDLL:
         L.yoco_xattn_chunk.argtypes = run_args
         L.yoco_xattn_combine.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
         L.yoco_xattn_status.argtypes = [vp, vp]
+        L.yoco_xattn_profile_enable.argtypes = [i32]
+        L.yoco_xattn_profile_collect.argtypes = [vp, i32, vp]
         L.yoco_xattn_strerror.argtypes = [i32]
         L.yoco_xattn_strerror.restype = ctypes.c_char_p
         L.yoco_xattn_last_cuda_error.argtypes = []
-        for name in ("plan", "workspace_size", "decode", "chunk", "combine", "status", "last_cuda_error"):
+        for name in ("plan", "workspace_size", "decode", "chunk", "combine", "status", "last_cuda_error",
+                     "profile_enable", "profile_collect"):
             getattr(L, "yoco_xattn_" + name).restype = i32
         _lib = L
     return _lib
@@ -150,3 +153,19 @@ def yoco_xattn_combine(part_o, part_lse, O, lse=None, stream=None) -> None:
 def yoco_xattn_status(workspace, stream=None) -> int:
     """Synchronise the stream and return the device status word of the last call (0 = ok)."""
     return int(lib().yoco_xattn_status(_ptr(workspace), _stream_ptr(stream)))
+
+
+def yoco_xattn_profile_enable(max_records: int) -> None:
+    rc = lib().yoco_xattn_profile_enable(max_records)
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_profile_enable")
+
+
+def yoco_xattn_profile_collect(capacity: int) -> np.ndarray:
+    """Durations (ms) of the attention kernel of the calls recorded since the last collect."""
+    buf = np.zeros(max(1, capacity), dtype=np.float32)
+    n = ctypes.c_int32(0)
+    rc = lib().yoco_xattn_profile_collect(ctypes.c_void_p(buf.ctypes.data), capacity, ctypes.byref(n))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_profile_collect")
+    return buf[: n.value].copy()

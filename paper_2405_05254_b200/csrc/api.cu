@@ -139,6 +139,25 @@ int32_t make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int32_t d,
     return YOCO_OK;
 }
 
+// ---- optional per-launch timing of the attention kernel -------------------------------------
+struct Profiler {
+    std::vector<cudaEvent_t> events;   // pairs: before / after the attention kernel
+    int32_t used = 0;                  // pairs recorded so far
+} g_prof;
+
+cudaEvent_t prof_event(bool after, bool* active) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const int32_t pairs = (int32_t)g_prof.events.size() / 2;
+    if (g_prof.used >= pairs) {
+        *active = false;
+        return nullptr;
+    }
+    *active = true;
+    cudaEvent_t e = g_prof.events[2 * g_prof.used + (after ? 1 : 0)];
+    if (after) ++g_prof.used;
+    return e;
+}
+
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const void* K, const void* V,
@@ -177,6 +196,9 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
     int32_t* status = reinterpret_cast<int32_t*>(ws);
 
     if (plan.info.num_segments > 0) {
+        bool prof = false;
+        cudaEvent_t ev = prof_event(false, &prof);
+        if (prof) YOCO_CUDA_TRY(cudaEventRecord(ev, stream));
         if (mode == YOCO_MODE_DECODE) {
             CUtensorMap tmK, tmV;
             if ((rc = make_map_2d(&tmK, K, plan.kv_rows_extent, shape->d, kDecodeTileN)) != YOCO_OK) return rc;
@@ -215,6 +237,10 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             p.m_tiles = plan.info.m_tiles;
             p.d = shape->d;
             YOCO_CUDA_TRY(launch_chunk(p, tmQ, tmK, tmV, plan.info.num_groups, stream));
+        }
+        if (prof) {
+            ev = prof_event(true, &prof);
+            if (prof) YOCO_CUDA_TRY(cudaEventRecord(ev, stream));
         }
     }
     if (plan.info.needs_combine) {
@@ -317,6 +343,34 @@ int32_t yoco_xattn_status(const void* workspace, void* stream) {
     YOCO_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost, s));
     YOCO_CUDA_TRY(cudaStreamSynchronize(s));
     return word == kStatusOk ? YOCO_OK : YOCO_ERR_TIMEOUT;
+}
+
+int32_t yoco_xattn_profile_enable(int32_t max_records) {
+    if (max_records < 0) return YOCO_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    for (cudaEvent_t e : g_prof.events) cudaEventDestroy(e);
+    g_prof.events.clear();
+    g_prof.used = 0;
+    for (int32_t k = 0; k < 2 * max_records; ++k) {
+        cudaEvent_t e;
+        cudaError_t err = cudaEventCreate(&e);
+        if (err != cudaSuccess) return cuda_fail(err);
+        g_prof.events.push_back(e);
+    }
+    return YOCO_OK;
+}
+
+int32_t yoco_xattn_profile_collect(float* kernel_ms, int32_t capacity, int32_t* count) {
+    if (!count || capacity < 0 || (capacity > 0 && !kernel_ms)) return YOCO_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const int32_t n = std::min(capacity, g_prof.used);
+    for (int32_t k = 0; k < n; ++k) {
+        YOCO_CUDA_TRY(cudaEventSynchronize(g_prof.events[2 * k + 1]));
+        YOCO_CUDA_TRY(cudaEventElapsedTime(&kernel_ms[k], g_prof.events[2 * k], g_prof.events[2 * k + 1]));
+    }
+    *count = n;
+    g_prof.used = 0;
+    return YOCO_OK;
 }
 
 const char* yoco_xattn_strerror(int32_t code) {

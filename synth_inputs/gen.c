@@ -9,9 +9,9 @@
  *
  *   key   = mix(mix(seed) ^ (tensor_id * odd constant))
  *   bits  = mix(key ^ mix(pair index))           pair index = e / 2
- *   u1    = (high 32 bits + 0.5) / 2^32  in (0,1),   u2 = low 32 bits / 2^32
+ *   u1    = (bits 40..63 + 0.5) / 2^24  in (0,1],   u2 = bits 8..31 / 2^24   (single precision)
  *   z0,z1 = sqrt(-2 ln u1) * (cos, sin)(2 pi u2)   (Box-Muller), element e takes z_(e & 1)
- *   value = round-to-nearest-even bf16 of (float)(mult * z)
+ *   value = round-to-nearest-even bf16 of mult * z
  *
  * mix() is the SplitMix64 finaliser (Steele, Lea, Flood 2014).
  */
@@ -52,16 +52,16 @@ void synth_normal_bf16(uint64_t seed, uint64_t tensor_id, double mult,
 {
     const uint64_t key = tensor_key(seed, tensor_id);
     const uint64_t p0 = first / 2, p1 = (first + count + 1) / 2;
-    const double two_pi = 6.283185307179586476925286766559;
+    const float two_pi = 6.2831853071795864769f;
 #pragma omp parallel for schedule(static)
     for (uint64_t p = p0; p < p1; ++p) {
         uint64_t bits = mix(key ^ mix(p));
-        double u1 = ((double)(bits >> 32) + 0.5) * (1.0 / 4294967296.0);
-        double u2 = (double)(bits & 0xFFFFFFFFull) * (1.0 / 4294967296.0);
-        double r = sqrt(-2.0 * log(u1));
-        double z0 = r * cos(two_pi * u2), z1 = r * sin(two_pi * u2);
+        float u1 = ((float)(bits >> 40) + 0.5f) * (1.0f / 16777216.0f);
+        float u2 = (float)((bits >> 8) & 0xFFFFFFull) * (1.0f / 16777216.0f);
+        float r = sqrtf(-2.0f * logf(u1)) * (float)mult;
+        float z0 = r * cosf(two_pi * u2), z1 = r * sinf(two_pi * u2);
         uint64_t e0 = 2 * p, e1 = 2 * p + 1;
-        if (e0 >= first && e0 < first + count) out[e0 - first] = f32_to_bf16_rne((float)(mult * z0));
-        if (e1 >= first && e1 < first + count) out[e1 - first] = f32_to_bf16_rne((float)(mult * z1));
+        if (e0 >= first && e0 < first + count) out[e0 - first] = f32_to_bf16_rne(z0);
+        if (e1 >= first && e1 < first + count) out[e1 - first] = f32_to_bf16_rne(z1);
     }
 }
