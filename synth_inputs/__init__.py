@@ -134,6 +134,8 @@ def workload(name: str) -> Workload:
                         kv_len=ragged_lengths(2, 16, 4096, 126977))
     if name == "1m":            # config 4
         return Workload(name, B=1, Hq=32, Hkv=8, d=128, T=1, layers=13, seed=3, kv_len=[1048576])
+    if name == "128k":          # config 4's shape at 1/8 of the length (profiler captures)
+        return Workload(name, B=1, Hq=32, Hkv=8, d=128, T=1, layers=13, seed=3, kv_len=[131072])
     if name == "chunk":         # config 5: 512 new rows appended after 262,144 cached keys
         return Workload(name, B=2, Hq=32, Hkv=8, d=128, T=512, layers=1, seed=4,
                         kv_len=[262144 + 512] * 2)
