@@ -56,6 +56,7 @@ extern "C" {
 #define YOCO_ERR_WORKSPACE_TOO_SMALL  (-3)
 #define YOCO_ERR_CUDA                 (-4)  /* a CUDA call failed; see yoco_xattn_last_cuda_error */
 #define YOCO_ERR_TIMEOUT              (-5)  /* a bounded device-side wait expired               */
+#define YOCO_ERR_STATIC_SCRATCH_EXCEEDED (-6) /* yoco_xattn_decode_static: problem too large    */
 
 #define YOCO_MODE_DECODE 0   /* split-KV kernel, G*T <= 16 query rows per KV head        */
 #define YOCO_MODE_CHUNK  1   /* tensor-core (tcgen05) kernel, any T >= 1                 */
@@ -126,6 +127,36 @@ int32_t yoco_xattn_decode(const yoco_xattn_shape* shape, const void* Q, const vo
                           const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
                           void* O, float* lse, void* workspace, size_t workspace_bytes,
                           void* stream);
+
+/* Decode without a workspace argument.  (The paper has no counterpart: this is a packaging
+ * variant of yoco_xattn_decode, same kernels, same result.)
+ *
+ * Who needs it: code that may not create device memory at the point where it calls
+ * attention -- a plugin inside a host application that owns the allocator, a real-time loop
+ * that forbids cudaMalloc after start-up, a caller whose memory pool is sized and frozen in
+ * advance.  Such callers still pass Q, K, V, O (and lse), but the split tables and the partial
+ * results go to a 4 MiB buffer that is part of this library's device image.  Every GPU that
+ * loads the library carries those 4 MiB until the process ends.
+ *
+ * Limits and rules:
+ *  - A problem whose decode workspace (yoco_xattn_workspace_size, decode mode) exceeds
+ *    yoco_xattn_static_scratch_bytes() is refused with YOCO_ERR_STATIC_SCRATCH_EXCEEDED and
+ *    nothing is enqueued.  4 MiB covers, e.g., B = 1 at 1M tokens and 16 ragged sequences.
+ *  - No cudaMalloc / cudaFree and no allocating library routine is called.
+ *  - The first call on each device looks the buffer's device address up (and sets kernel
+ *    attributes); make that first call with the device current and before any stream capture.
+ *  - All calls on a device share the one buffer, and it keeps whatever the previous call left.
+ *    The library rewrites the tables and the status word at the start of every call, and every
+ *    partial result is written before it is read, so stale contents are never used.  Two calls
+ *    that can overlap on the GPU (different streams without an ordering between them) race on
+ *    the buffer: order them, or give one of them yoco_xattn_decode with its own workspace.
+ *  - Argument and size errors are returned directly, before anything is enqueued. */
+int32_t yoco_xattn_decode_static(const yoco_xattn_shape* shape, const void* Q, const void* K,
+                                 const void* V, const int32_t* cu_kv_host,
+                                 const int32_t* kv_len_host, void* O, float* lse, void* stream);
+
+/* Size in bytes of the built-in buffer used by yoco_xattn_decode_static. */
+int32_t yoco_xattn_static_scratch_bytes(void);
 
 /* Multi-token chunk / full-sequence path: T new query rows per sequence, causal
  * inside the chunk, as a dense contraction on the tcgen05 tensor cores (S = Q K^T

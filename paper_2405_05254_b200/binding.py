@@ -15,6 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libyoco_xattn.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+ERR_STATIC_SCRATCH_EXCEEDED = -6
 MODE_DECODE, MODE_CHUNK = 0, 1
 
 
@@ -62,6 +63,8 @@ def lib() -> ctypes.CDLL:
         run_args = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.yoco_xattn_decode.argtypes = run_args
         L.yoco_xattn_chunk.argtypes = run_args
+        L.yoco_xattn_decode_static.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp]
+        L.yoco_xattn_static_scratch_bytes.argtypes = []
         L.yoco_xattn_combine.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
         L.yoco_xattn_status.argtypes = [vp, vp]
         L.yoco_xattn_profile_enable.argtypes = [i32]
@@ -70,7 +73,7 @@ def lib() -> ctypes.CDLL:
         L.yoco_xattn_strerror.restype = ctypes.c_char_p
         L.yoco_xattn_last_cuda_error.argtypes = []
         for name in ("plan", "workspace_size", "decode", "chunk", "combine", "status", "last_cuda_error",
-                     "profile_enable", "profile_collect"):
+                     "profile_enable", "profile_collect", "decode_static", "static_scratch_bytes"):
             getattr(L, "yoco_xattn_" + name).restype = i32
         _lib = L
     return _lib
@@ -169,3 +172,20 @@ def yoco_xattn_profile_collect(capacity: int) -> np.ndarray:
     if rc != OK:
         raise YocoError(rc, "yoco_xattn_profile_collect")
     return buf[: n.value].copy()
+
+
+def yoco_xattn_decode_static(shape: Shape, Q, K, V, cu_kv, kv_len, O, lse, stream=None) -> None:
+    """Decode for callers that cannot allocate: same result as yoco_xattn_decode, but the split
+    tables and partial results live in a 4 MiB buffer built into the library instead of a
+    caller-provided workspace.  Raises YocoError(ERR_STATIC_SCRATCH_EXCEEDED) when the problem
+    needs more than that.  Calls that may overlap on the GPU must not both use this entry."""
+    keep_cu, p_cu = _host_i32(cu_kv)
+    keep_len, p_len = _host_i32(kv_len)
+    rc = lib().yoco_xattn_decode_static(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), p_cu, p_len,
+                                        _ptr(O), _ptr(lse), _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_decode_static")
+
+
+def yoco_xattn_static_scratch_bytes() -> int:
+    return int(lib().yoco_xattn_static_scratch_bytes())

@@ -263,6 +263,29 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
     return YOCO_OK;
 }
 
+
+// ---- built-in scratch for callers that cannot allocate -------------------------------------
+// Lives in every GPU that loads this library until the process exits.  In host code the
+// name below is only a handle; the device address comes from cudaGetSymbolAddress.
+constexpr size_t kStaticScratchBytes = 4u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+void* g_static_scratch_addr[kMaxDevices] = {};
+
+int32_t static_scratch_address(void** out) {
+    int dev = 0;
+    YOCO_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return YOCO_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void* ptr = nullptr;
+        YOCO_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));   // address on the current device
+        if (!ptr) return cuda_fail(cudaErrorInvalidSymbol);
+        g_static_scratch_addr[dev] = ptr;
+    }
+    *out = g_static_scratch_addr[dev];
+    return YOCO_OK;
+}
+
 }  // namespace
 }  // namespace yoco
 
@@ -306,6 +329,28 @@ int32_t yoco_xattn_decode(const yoco_xattn_shape* shape, const void* Q, const vo
     return run(shape, YOCO_MODE_DECODE, Q, K, V, cu_kv_host, kv_len_host, O, lse, workspace,
                workspace_bytes, stream);
 }
+
+int32_t yoco_xattn_decode_static(const yoco_xattn_shape* shape, const void* Q, const void* K,
+                                 const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
+                                 void* O, float* lse, void* stream) {
+    if (!shape) return YOCO_ERR_INVALID_ARG;
+    int32_t rc = validate_shape(*shape, YOCO_MODE_DECODE);
+    if (rc != YOCO_OK) return rc;
+    if (shape->B == 0) return YOCO_OK;
+    // size check first, on the host: nothing is enqueued for a problem that does not fit
+    DeviceState* dev = nullptr;
+    if ((rc = device_state(&dev)) != YOCO_OK) return rc;
+    Plan plan;
+    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, YOCO_MODE_DECODE, plan)) != YOCO_OK)
+        return rc;
+    if ((size_t)plan.info.workspace_bytes > kStaticScratchBytes) return YOCO_ERR_STATIC_SCRATCH_EXCEEDED;
+    void* scratch = nullptr;
+    if ((rc = static_scratch_address(&scratch)) != YOCO_OK) return rc;
+    return run(shape, YOCO_MODE_DECODE, Q, K, V, cu_kv_host, kv_len_host, O, lse, scratch,
+               kStaticScratchBytes, stream);
+}
+
+int32_t yoco_xattn_static_scratch_bytes(void) { return (int32_t)kStaticScratchBytes; }
 
 int32_t yoco_xattn_chunk(const yoco_xattn_shape* shape, const void* Q, const void* K, const void* V,
                          const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
@@ -381,6 +426,9 @@ const char* yoco_xattn_strerror(int32_t code) {
         case YOCO_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case YOCO_ERR_CUDA: return "CUDA call failed (see yoco_xattn_last_cuda_error)";
         case YOCO_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case YOCO_ERR_STATIC_SCRATCH_EXCEEDED:
+            return "problem needs more scratch than the built-in static buffer holds; "
+                   "use yoco_xattn_decode with a caller-provided workspace";
         default: return "unknown error code";
     }
 }
