@@ -1,7 +1,477 @@
-// placeholder until the tcgen05 kernel lands
+// Multi-token chunk / full-sequence attention on the tcgen05 tensor cores.
+//
+// One CTA owns one 128-row tile of the G*T query rows of a (sequence, KV head) stream and walks
+// a contiguous range of 128-key tiles.  Roles (192 threads):
+//   warp 0      TMA producer: Q tile once per segment, K and V tiles through two-deep rings
+//   warp 1      MMA issuer: S = Q K^T (both operands K-major in shared memory) into one of two
+//               128-column TMEM buffers, then O += P V (P K-major, V MN-major) into a third
+//   warps 2..5  softmax: thread = query row; reads its S row from TMEM, keeps the running
+//               max / sum, writes P (bf16) back to shared memory in the swizzled operand layout,
+//               rescales O in TMEM only when the row max grew by more than 2^8, and normalises
+//               and stores O (or a partial + LSE) at the end of a segment
+// All shared-memory operand tiles use the 128-byte swizzle that TMA writes and the tensor-core
+// descriptors read.  Every wait is bounded and reports through the status word.
 #include "kernels.h"
+#include "ptx.cuh"
+
 namespace yoco {
-cudaError_t launch_chunk(const ChunkParams&, const CUtensorMap&, const CUtensorMap&, const CUtensorMap&,
-                         int, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t chunk_kernel_setup() { return cudaSuccess; }
+
+namespace {
+
+constexpr int BM = kChunkTileM;   // 128 query rows
+constexpr int BN = kChunkTileN;   // 128 keys
+constexpr int kThreads = 192;
+constexpr int HALF_BYTES = 128 * 128;          // 128 rows x 64 bf16: one swizzled half tile
+constexpr uint32_t TMEM_COLS = 512;
+constexpr float kRescaleThreshold = 8.f;       // in log2 units: P stays below 2^8
+
+template <int D>
+struct CCfg {
+    static constexpr int HALVES = D / 64;
+    static constexpr int TILE_BYTES = HALVES * HALF_BYTES;     // Q, K or V tile
+    static constexpr int P_BYTES = 2 * HALF_BYTES;             // 128 x 128 bf16
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = OFF_Q + TILE_BYTES;
+    static constexpr int OFF_V = OFF_K + 2 * TILE_BYTES;
+    static constexpr int OFF_P = OFF_V + 2 * TILE_BYTES;
+    static constexpr int OFF_BAR = OFF_P + 2 * P_BYTES;
+    static constexpr int NUM_BARS = 18;
+    static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16;
+};
+
+// ---- tcgen05 wrappers -----------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
+                 "r"(ncols)
+                 : "memory");
 }
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                     smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+          "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+          "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+          "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+    const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
+        "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
+        "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+           ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: f32 accumulate, bf16 x bf16, M = 128, given N and B major-ness.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(BM >> 4) << 24);
+}
+
+struct Abort {
+    volatile int* flag;
+    int32_t* status;
+};
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, const Abort& ab) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 0) {
+            if (*ab.flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                atomicExch(ab.status, kStatusTimeout);
+                *ab.flag = 1;
+                return false;
+            }
+        }
+    }
+}
+
+// All lanes of a warp wait on the same barrier; the result is made warp-uniform so that the
+// lanes never diverge around the __syncwarp / elected arrives that follow.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, const Abort& ab) {
+    const bool r = wait_or_abort(bar, parity, ab);
+    return __all_sync(0xffffffffu, r);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+             const __grid_constant__ CUtensorMap tmV, const ChunkParams p) {
+    using C = CCfg<D>;
+    constexpr int HALVES = C::HALVES;
+    constexpr int KSTEPS_QK = D / 16;
+    constexpr int KSTEPS_PV = BN / 16;
+
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR);
+    uint64_t* q_full = bars + 0;
+    uint64_t* q_empty = bars + 1;
+    uint64_t* k_full = bars + 2;    // [2]
+    uint64_t* k_empty = bars + 4;   // [2]
+    uint64_t* v_full = bars + 6;    // [2]
+    uint64_t* v_empty = bars + 8;   // [2]
+    uint64_t* s_full = bars + 10;   // [2]
+    uint64_t* s_empty = bars + 12;  // [2]
+    uint64_t* p_full = bars + 14;   // [2]
+    uint64_t* p_empty = bars + 16;  // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::NUM_BARS);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int group = blockIdx.x / p.m_tiles, m_tile = blockIdx.x - group * p.m_tiles;
+    const int seg_lo = p.group_begin[group], seg_hi = p.group_begin[group + 1];
+    const Abort ab{abort_flag, p.status};
+    const bool aligned_ok = (smem_u32(smem) & 1023u) == 0;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = aligned_ok ? 0 : 1;
+        if (!aligned_ok) atomicExch(p.status, kStatusTimeout + 1);
+        mbar_init(q_full, 1);
+        mbar_init(q_empty, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&k_full[b], 1);
+            mbar_init(&k_empty[b], 1);
+            mbar_init(&v_full[b], 1);
+            mbar_init(&v_empty[b], 1);
+            mbar_init(&s_full[b], 1);
+            mbar_init(&s_empty[b], 4);
+            mbar_init(&p_full[b], 4);
+            mbar_init(&p_empty[b], 1);
+        }
+        mbar_fence_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ======================================= TMA producer ================================
+        if (lane == 0 && aligned_ok) {
+            tma_prefetch_desc(&tmQ);
+            tma_prefetch_desc(&tmK);
+            tma_prefetch_desc(&tmV);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int si = seg_lo; si < seg_hi && ok; ++si) {
+                const DevSegment seg = p.segments[si];
+                const uint32_t sidx = si - seg_lo;
+                if (!(ok = wait_or_abort(q_empty, (sidx & 1u) ^ 1u, ab))) break;
+                mbar_expect_tx(q_full, C::TILE_BYTES);
+                for (int h = 0; h < HALVES; ++h)
+                    tma_load_2d(smem + C::OFF_Q + h * HALF_BYTES, &tmQ, h * 64, seg.q_row0 + m_tile * BM, q_full);
+                for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
+                    const uint32_t b = it & 1u, n = it >> 1;
+                    const int row = seg.kv_row0 + (k0 - seg.k_begin);
+                    if (!(ok = wait_or_abort(&k_empty[b], (n & 1u) ^ 1u, ab))) break;
+                    mbar_expect_tx(&k_full[b], C::TILE_BYTES);
+                    for (int h = 0; h < HALVES; ++h)
+                        tma_load_2d(smem + C::OFF_K + b * C::TILE_BYTES + h * HALF_BYTES, &tmK, h * 64, row, &k_full[b]);
+                    if (!(ok = wait_or_abort(&v_empty[b], (n & 1u) ^ 1u, ab))) break;
+                    mbar_expect_tx(&v_full[b], C::TILE_BYTES);
+                    for (int h = 0; h < HALVES; ++h)
+                        tma_load_2d(smem + C::OFF_V + b * C::TILE_BYTES + h * HALF_BYTES, &tmV, h * 64, row, &v_full[b]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ======================================= MMA issuer ==================================
+        if (lane == 0 && aligned_ok) {
+            constexpr uint32_t idesc_qk = make_idesc(BN, false);
+            constexpr uint32_t idesc_pv = make_idesc(D, true);
+            const uint32_t sbase = smem_u32(smem);
+            const uint64_t q_desc = make_desc(sbase + C::OFF_Q, 16, 1024);
+            const uint32_t tmem_o = tmem_base + 2 * BN;
+            uint32_t it = 0;
+            bool ok = true;
+            // PV of the previous tile is issued after QK of the current one, so that the tensor
+            // pipe has work while the softmax warps process the previous S
+            bool have_prev = false, prev_first = false;
+            uint32_t prev_it = 0;
+            auto issue_pv = [&](uint32_t i, bool first_of_segment) -> bool {
+                const uint32_t b = i & 1u, n = i >> 1;
+                if (!wait_or_abort(&p_full[b], n & 1u, ab)) return false;
+                if (!wait_or_abort(&v_full[b], n & 1u, ab)) return false;
+                tc_fence_after();
+                const uint64_t p_desc = make_desc(sbase + C::OFF_P + b * C::P_BYTES, 16, 1024);
+                const uint64_t v_desc = make_desc(sbase + C::OFF_V + b * C::TILE_BYTES, BN * 128, 1024);
+#pragma unroll
+                for (int ks = 0; ks < KSTEPS_PV; ++ks) {
+                    const uint32_t a_off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                    const uint32_t b_off = ks * 16 * 128;
+                    umma_ss(tmem_o, p_desc + (a_off >> 4), v_desc + (b_off >> 4), idesc_pv,
+                            (first_of_segment && ks == 0) ? 0u : 1u);
+                }
+                umma_commit(&p_empty[b]);
+                umma_commit(&v_empty[b]);
+                return true;
+            };
+            for (int si = seg_lo; si < seg_hi && ok; ++si) {
+                const DevSegment seg = p.segments[si];
+                const uint32_t sidx = si - seg_lo;
+                if (have_prev) {   // finish the previous segment before waiting for the new Q
+                    if (!(ok = issue_pv(prev_it, prev_first))) break;
+                    have_prev = false;
+                }
+                if (!(ok = wait_or_abort(q_full, sidx & 1u, ab))) break;
+                for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
+                    const uint32_t b = it & 1u, n = it >> 1;
+                    if (!(ok = wait_or_abort(&k_full[b], n & 1u, ab))) break;
+                    if (!(ok = wait_or_abort(&s_empty[b], (n & 1u) ^ 1u, ab))) break;
+                    tc_fence_after();
+                    const uint64_t k_desc = make_desc(sbase + C::OFF_K + b * C::TILE_BYTES, 16, 1024);
+#pragma unroll
+                    for (int ks = 0; ks < KSTEPS_QK; ++ks) {
+                        const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                        umma_ss(tmem_base + b * BN, q_desc + (off >> 4), k_desc + (off >> 4), idesc_qk, ks > 0 ? 1u : 0u);
+                    }
+                    umma_commit(&s_full[b]);
+                    umma_commit(&k_empty[b]);
+                    if (k0 + BN >= seg.k_end) umma_commit(q_empty);   // Q may be replaced
+                    if (have_prev && !(ok = issue_pv(prev_it, prev_first))) break;
+                    have_prev = true;
+                    prev_it = it;
+                    prev_first = (k0 == seg.k_begin);
+                }
+            }
+            if (ok && have_prev) issue_pv(prev_it, prev_first);
+        }
+    } else {
+        // ======================================= softmax warps ===============================
+        const int quad = warp & 3;                     // TMEM lane quadrant this warp may access
+        const int row = quad * 32 + lane;              // row inside the 128-row tile
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const uint32_t tmem_o = tmem_base + 2 * BN + lane_addr;
+        const int r_local = m_tile * BM + row;         // row inside the stream's G*T rows
+        const bool row_valid = r_local < p.rows_per_stream;
+        uint32_t it = 0;
+        bool ok = aligned_ok;
+
+        for (int si = seg_lo; si < seg_hi; ++si) {
+            const DevSegment seg = p.segments[si];
+            const int n_full = seg.n_kv - p.T + 1;     // keys visible to every row
+            const int vis = min(seg.n_kv, max(0, n_full + (r_local % p.T)));
+            float m_ref = -INFINITY, l = 0.f;
+            const uint32_t seg_first_it = it;
+
+            for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
+                if (!ok) continue;
+                const uint32_t b = it & 1u, n = it >> 1;
+                if (!(ok = warp_wait(&s_full[b], n & 1u, ab))) continue;
+                tc_fence_after();
+                float s[BN];
+#pragma unroll
+                for (int c = 0; c < BN / 32; ++c)
+                    tmem_ld32(tmem_base + b * BN + lane_addr + c * 32, *reinterpret_cast<float(*)[32]>(&s[c * 32]));
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_empty[b]);          // S buffer may be overwritten
+
+                const bool need_mask = k0 + BN > n_full;
+                float mx = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < BN; ++j) {
+                    float v = s[j] * p.scale_log2;
+                    if (need_mask) v = (k0 + j < vis) ? v : -INFINITY;
+                    s[j] = v;
+                    mx = fmaxf(mx, v);
+                }
+                // lazy rescale: the reference max moves only when the row max outgrew it by 2^8
+                float alpha = 1.f;
+                bool grow = mx > m_ref + kRescaleThreshold || (m_ref == -INFINITY && mx > -INFINITY);
+                if (grow) {
+                    alpha = exp2f(m_ref - mx);                    // 0 when m_ref = -inf
+                    m_ref = mx;
+                    l *= alpha;
+                }
+                if (__any_sync(0xffffffffu, grow) && it > seg_first_it) {
+                    // O holds the sums of the earlier tiles of this segment: wait for the last PV
+                    const uint32_t pi = it - 1;
+                    if (!(ok = warp_wait(&p_empty[pi & 1u], (pi >> 1) & 1u, ab))) continue;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        float o[32];
+                        tmem_ld32(tmem_o + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) o[j] *= alpha;
+                        tmem_st32(tmem_o + c * 32, o);
+                    }
+                    tmem_wait_st();
+                    tc_fence_before();
+                }
+                const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
+
+                // P buffer b is free once PV of tile it-2 has completed
+                if (!(ok = warp_wait(&p_empty[b], (n & 1u) ^ 1u, ab))) continue;
+                uint8_t* prow = smem + C::OFF_P + b * C::P_BYTES + row * 128;
+                float lsum = 0.f;
+#pragma unroll
+                for (int c = 0; c < BN / 8; ++c) {                 // 8 keys = one 16-byte chunk
+                    float e[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        e[j] = exp2f(s[c * 8 + j] - m_use);
+                        lsum += e[j];
+                    }
+                    uint4 pk;
+                    pk.x = pack_bf16x2(e[0], e[1]);
+                    pk.y = pack_bf16x2(e[2], e[3]);
+                    pk.z = pack_bf16x2(e[4], e[5]);
+                    pk.w = pack_bf16x2(e[6], e[7]);
+                    *reinterpret_cast<uint4*>(prow + (c >> 3) * HALF_BYTES + (((c & 7) ^ (row & 7)) << 4)) = pk;
+                }
+                l += lsum;
+
+                // keys past the end of the sequence: their V rows may hold anything; zero them so
+                // that 0 * garbage cannot make NaN
+                if (k0 + BN > seg.n_kv) {
+                    if (!(ok = warp_wait(&v_full[b], n & 1u, ab))) continue;
+                    if (k0 + row >= seg.n_kv) {
+                        uint8_t* vrow = smem + C::OFF_V + b * C::TILE_BYTES + row * 128;
+#pragma unroll
+                        for (int h = 0; h < HALVES; ++h)
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                *reinterpret_cast<uint4*>(vrow + h * HALF_BYTES + q * 16) = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+                fence_proxy_async_smem();                           // generic writes -> tensor core reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_full[b]);
+            }
+
+            // ---- end of segment: O is complete once the last PV has finished ----
+            if (ok && it > seg_first_it) {
+                const uint32_t pi = it - 1;
+                ok = warp_wait(&p_empty[pi & 1u], (pi >> 1) & 1u, ab);
+            }
+            if (ok) {
+                tc_fence_after();
+                const bool has = l > 0.f;
+                const float inv = has ? 1.f / l : 0.f;
+                const float lse = has ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                const bool final_out = seg.stream_nseg == 1;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    float o[32];
+                    tmem_ld32(tmem_o + c * 32, o);
+                    tmem_wait_ld();
+                    if (row_valid) {
+                        if (final_out) {
+                            __nv_bfloat16* dst = p.O + ((int64_t)seg.q_row0 + r_local) * D + c * 32;
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                uint4 pk;
+                                pk.x = pack_bf16x2(has ? o[q * 8 + 0] * inv : 0.f, has ? o[q * 8 + 1] * inv : 0.f);
+                                pk.y = pack_bf16x2(has ? o[q * 8 + 2] * inv : 0.f, has ? o[q * 8 + 3] * inv : 0.f);
+                                pk.z = pack_bf16x2(has ? o[q * 8 + 4] * inv : 0.f, has ? o[q * 8 + 5] * inv : 0.f);
+                                pk.w = pack_bf16x2(has ? o[q * 8 + 6] * inv : 0.f, has ? o[q * 8 + 7] * inv : 0.f);
+                                *reinterpret_cast<uint4*>(dst + q * 8) = pk;
+                            }
+                        } else {
+                            float* dst = p.part_o + ((int64_t)seg.slot * p.rows_per_stream + r_local) * D + c * 32;
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                *reinterpret_cast<float4*>(dst + q * 4) =
+                                    make_float4(has ? o[q * 4 + 0] * inv : 0.f, has ? o[q * 4 + 1] * inv : 0.f,
+                                                has ? o[q * 4 + 2] * inv : 0.f, has ? o[q * 4 + 3] * inv : 0.f);
+                        }
+                    }
+                }
+                if (row_valid) {
+                    if (final_out) {
+                        if (p.lse) p.lse[seg.q_row0 + r_local] = lse;
+                    } else {
+                        p.part_lse[(int64_t)seg.slot * p.rows_per_stream + r_local] = lse;
+                    }
+                }
+                tc_fence_before();
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+template <int D>
+cudaError_t launch_one(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                       const CUtensorMap& tmV, int num_groups, cudaStream_t stream) {
+    chunk_kernel<D><<<num_groups * p.m_tiles, kThreads, CCfg<D>::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t chunk_kernel_setup() {
+    cudaError_t e = cudaFuncSetAttribute(chunk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         CCfg<128>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(chunk_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                CCfg<64>::SMEM_BYTES);
+}
+
+cudaError_t launch_chunk(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                         const CUtensorMap& tmV, int num_groups, cudaStream_t stream) {
+    if (num_groups <= 0) return cudaSuccess;
+    return p.d == 128 ? launch_one<128>(p, tmQ, tmK, tmV, num_groups, stream)
+                      : launch_one<64>(p, tmQ, tmK, tmV, num_groups, stream);
+}
+
+}  // namespace yoco
