@@ -67,7 +67,7 @@ typedef struct yoco_xattn_shape {
     int32_t Hkv;             /* key/value heads, divides Hq                               */
     int32_t d;               /* head dimension: 64 or 128                                 */
     int32_t T;               /* query rows per sequence in this call                      */
-    float   scale;           /* 0 -> 1/sqrt(d)                                            */
+    float   scale;           /* > 0, or 0 -> 1/sqrt(d); negative values are rejected       */
     int64_t kv_head_stride;  /* elements between KV heads of one sequence; 0 -> N_i*d     */
     int32_t max_kv_len;      /* used as every N_i when kv_len_host is NULL                */
     int32_t reserved;        /* must be 0                                                 */

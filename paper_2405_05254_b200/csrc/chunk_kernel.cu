@@ -97,6 +97,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
         "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ float ex2_approx(float x) {   // 2^x, one MUFU op; 2^-inf = 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -317,20 +322,21 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&s_empty[b]);          // S buffer may be overwritten
 
-                const bool need_mask = k0 + BN > n_full;
-                float mx = -INFINITY;
+                // row max of the raw scores (scale > 0, so it commutes with max); four independent
+                // chains keep the dependent-latency off the critical path
+                if (k0 + BN > n_full) {        // tile touches the causal edge or the sequence end
 #pragma unroll
-                for (int j = 0; j < BN; ++j) {
-                    float v = s[j] * p.scale_log2;
-                    if (need_mask) v = (k0 + j < vis) ? v : -INFINITY;
-                    s[j] = v;
-                    mx = fmaxf(mx, v);
+                    for (int j = 0; j < BN; ++j) s[j] = (k0 + j < vis) ? s[j] : -INFINITY;
                 }
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int j = 0; j < BN; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], s[j]);
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
                 // lazy rescale: the reference max moves only when the row max outgrew it by 2^8
                 float alpha = 1.f;
                 bool grow = mx > m_ref + kRescaleThreshold || (m_ref == -INFINITY && mx > -INFINITY);
                 if (grow) {
-                    alpha = exp2f(m_ref - mx);                    // 0 when m_ref = -inf
+                    alpha = ex2_approx(m_ref - mx);               // 0 when m_ref = -inf
                     m_ref = mx;
                     l *= alpha;
                 }
@@ -356,14 +362,15 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 // P buffer b is free once PV of tile it-2 has completed
                 if (!(ok = warp_wait(&p_empty[b], (n & 1u) ^ 1u, ab))) continue;
                 uint8_t* prow = smem + C::OFF_P + b * C::P_BYTES + row * 128;
-                float lsum = 0.f;
+                float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+                const float neg_m = -m_use;
 #pragma unroll
                 for (int c = 0; c < BN / 8; ++c) {                 // 8 keys = one 16-byte chunk
                     float e[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
-                        e[j] = exp2f(s[c * 8 + j] - m_use);
-                        lsum += e[j];
+                        e[j] = ex2_approx(fmaf(s[c * 8 + j], p.scale_log2, neg_m));
+                        ls4[j & 3] += e[j];
                     }
                     uint4 pk;
                     pk.x = pack_bf16x2(e[0], e[1]);
@@ -372,6 +379,7 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     pk.w = pack_bf16x2(e[6], e[7]);
                     *reinterpret_cast<uint4*>(prow + (c >> 3) * HALF_BYTES + (((c & 7) ^ (row & 7)) << 4)) = pk;
                 }
+                const float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
                 l += lsum;
 
                 // keys past the end of the sequence: their V rows may hold anything; zero them so

@@ -7,7 +7,7 @@ namespace yoco {
 
 int32_t validate_shape(const yoco_xattn_shape& s, int32_t mode) {
     if (s.B < 0 || s.Hq <= 0 || s.Hkv <= 0 || s.T <= 0 || s.d <= 0 || s.max_kv_len < 0 ||
-        s.kv_head_stride < 0 || s.reserved != 0 || !(s.scale == s.scale))
+        s.kv_head_stride < 0 || s.reserved != 0 || !(s.scale >= 0.f))
         return YOCO_ERR_INVALID_ARG;
     if (mode != YOCO_MODE_DECODE && mode != YOCO_MODE_CHUNK) return YOCO_ERR_INVALID_ARG;
     if (s.d != 64 && s.d != 128) return YOCO_ERR_UNSUPPORTED;
