@@ -44,15 +44,16 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)", {}
 
 
-def ncu_traffic_per_launch(workload: str, kv_bytes: int):
-    """DRAM bytes per launch of the decode kernel from the committed ncu capture, scaled by
-    the K/V bytes of this workload (traffic grows in proportion to the keys streamed)."""
-    p = os.path.join(ROOT, "profiles", "decode_kernel_traffic.json")
-    if not os.path.exists(p):
-        return None
-    with open(p) as f:
-        d = json.load(f)
-    return float(d["dram_bytes_per_launch"]) * kv_bytes / float(d["kv_bytes_per_launch"])
+# dram__bytes_read.sum + dram__bytes_write.sum of decode_kernel<128, 8> per launch from the ncu capture
+# summarised in profiles/decode_kernel_128k_ncu_full.md (mean of two launches, 128K-token case).
+NCU_DECODE_DRAM_BYTES = 540852736
+NCU_DECODE_KV_BYTES = 536870912
+
+
+def ncu_traffic_per_launch(kv_bytes: int):
+    """Traffic of a full-size launch: every K/V byte is read exactly once, so DRAM bytes grow in
+    proportion to the keys streamed."""
+    return NCU_DECODE_DRAM_BYTES * (kv_bytes / NCU_DECODE_KV_BYTES)
 
 
 class ClockSampler:
@@ -178,6 +179,43 @@ def workload_config(w, n_gpus):
             "parallelism": f"replicas x{n_gpus} (one cache per GPU, no collective)"}
 
 
+def measure_chunk(dev, peaks, name="chunk"):
+    """The multi-token path on its own workload (512 new rows after 262,144 cached keys, B = 2):
+    achieved TFLOP/s of the tcgen05 kernel against the measured bf16 peaks."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    w = si.workload(name)
+    to_dev = lambda a: torch.from_numpy(a.reshape(-1).view(np.int16)).to(dev).view(torch.bfloat16)  # noqa: E731
+    K, V, Q = to_dev(w.make_k()), to_dev(w.make_v()), to_dev(w.make_q(0))
+    shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(w.kv_len.max()))
+    ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_CHUNK), dtype=torch.uint8, device=dev)
+    O = torch.empty(w.B * w.Hq * w.T * w.d, dtype=torch.bfloat16, device=dev)
+    for _ in range(3):
+        bd.yoco_xattn_chunk(shape, Q, K, V, w.cu, w.kv_len, O, None, ws)
+    assert bd.yoco_xattn_status(ws) == 0
+    n = 10
+    bd.yoco_xattn_profile_enable(n)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        bd.yoco_xattn_chunk(shape, Q, K, V, w.cu, w.kv_len, O, None, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    call_ms = e0.elapsed_time(e1) / n
+    k_ms = float(bd.yoco_xattn_profile_collect(n).mean())
+    bd.yoco_xattn_profile_enable(0)
+    flop = sum(w.Hq * (w.T * (int(nk) - w.T) + w.T * (w.T + 1) / 2) * 4 * w.d for nk in w.kv_len)
+    tf = flop / (k_ms * 1e-3) / 1e12
+    burst = float(peaks.get("bf16_tflops", 1590.0))
+    sustained = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    return {"workload": f"{w.name}: B={w.B} Hq={w.Hq} Hkv={w.Hkv} d={w.d} T={w.T} kv_len={int(w.kv_len[0])}",
+            "flop_causal_exact": flop, "kernel_ms": k_ms, "call_ms": call_ms, "bound": "tensor",
+            "achieved": tf, "unit": "TFLOP/s", "peak": burst, "frac": tf / burst,
+            "peak_sustained": sustained, "frac_of_sustained": tf / sustained,
+            "peak_source": "measured (MEASURED_PEAKS.json)" if peaks else "fallback",
+            "kv_bytes": w.kv_bytes}
+
+
 def run_ours(args):
     import torch
     from paper_2405_05254_b200 import binding as bd
@@ -188,6 +226,10 @@ def run_ours(args):
             raise SystemExit("--gpus N > 1 must be launched with torchrun (one rank per GPU)")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    if args.only_chunk:
+        if rank == 0:
+            print(json.dumps({"chunk": measure_chunk(dev, measured_peaks()[2], args.chunk_workload)}), flush=True)
+        return
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
@@ -293,7 +335,7 @@ def run_ours(args):
         peak, peak_src, peaks = measured_peaks()
         k_avg_ms = float(kernel_ms.mean()) if len(kernel_ms) else float("nan")
         achieved = w.kv_bytes / (k_avg_ms * 1e-3) / 1e9
-        traffic = ncu_traffic_per_launch(w.name, w.kv_bytes)
+        traffic = ncu_traffic_per_launch(w.kv_bytes)
         e2e_value = w.kv_bytes * e2e_steps * w.layers * world / (e2e_ms * 1e-3) / 1e9
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
@@ -316,6 +358,10 @@ def run_ours(args):
                          "kernel_us": k_avg_ms * 1e3, "algorithmic_bytes_per_launch": w.kv_bytes,
                          "traffic": traffic},
         }
+        if world == 1 and not args.no_chunk:
+            del K, V
+            torch.cuda.empty_cache()
+            line["chunk"] = measure_chunk(dev, peaks, args.chunk_workload)
         if world == 1 and not args.no_cpu_baseline:
             gbs, dt, sample, cores = oracle_sample_rate(w, Qh, Kh, Vh)
             line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
@@ -334,6 +380,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="1m", choices=["1m", "128k", "3b_32k", "ragged", "tiny"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-chunk", action="store_true", help="skip the extra measurement of the chunk path")
+    ap.add_argument("--only-chunk", action="store_true", help="measure the chunk path alone")
+    ap.add_argument("--chunk-workload", default="chunk", choices=["chunk", "chunk_32k"])
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

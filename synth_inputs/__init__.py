@@ -139,6 +139,9 @@ def workload(name: str) -> Workload:
     if name == "chunk":         # config 5: 512 new rows appended after 262,144 cached keys
         return Workload(name, B=2, Hq=32, Hkv=8, d=128, T=512, layers=1, seed=4,
                         kv_len=[262144 + 512] * 2)
+    if name == "chunk_32k":     # config 5 with a 32K cache (profiler captures)
+        return Workload(name, B=2, Hq=32, Hkv=8, d=128, T=512, layers=1, seed=4,
+                        kv_len=[32768 + 512] * 2)
     if name == "ragged_small":  # same recipe as config 3, 32x shorter
         return Workload(name, B=16, Hq=32, Hkv=8, d=128, T=1, layers=1, seed=2,
                         kv_len=ragged_lengths(2, 16, 128, 3969))
