@@ -109,8 +109,7 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sel), "window": window}
 
 
-def dist_env():
-    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+from paper_2405_05254_b200.ranks import dist_env, job_throughput_gbs, max_over_ranks, replica_seed  # noqa: E402
 
 
 # ------------------------------------------------------------------------------------------
@@ -241,7 +240,7 @@ def run_ours(args):
     sampler = ClockSampler(local_rank) if rank == 0 else None
 
     w = si.workload(args.workload)
-    w.seed = w.seed + 1000 * rank          # every replica has its own cache contents
+    w.seed = replica_seed(w.seed, rank)    # every replica has its own cache contents
     Kh, Vh = w.make_k(), w.make_v()
     K = torch.from_numpy(Kh.view(np.int16)).to(dev).view(torch.bfloat16)
     V = torch.from_numpy(Vh.view(np.int16)).to(dev).view(torch.bfloat16)
@@ -319,24 +318,20 @@ def run_ours(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(times, op=torch.distributed.ReduceOp.MAX)
-    total_ms, e2e_ms = (float(x) for x in times.cpu())
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dev)
 
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
 
     if rank == 0:
         calls = args.steps * w.layers
-        bytes_all = w.kv_bytes * calls * world
-        value = bytes_all / (total_ms * 1e-3) / 1e9
+        value = job_throughput_gbs(w.kv_bytes, calls, world, total_ms)
         ms_per_step = total_ms / args.steps
         us_tl = total_ms * 1e3 / calls / w.B
         peak, peak_src, peaks = measured_peaks()
         k_avg_ms = float(kernel_ms.mean()) if len(kernel_ms) else float("nan")
         achieved = w.kv_bytes / (k_avg_ms * 1e-3) / 1e9
         traffic = ncu_traffic_per_launch(w.kv_bytes)
-        e2e_value = w.kv_bytes * e2e_steps * w.layers * world / (e2e_ms * 1e-3) / 1e9
+        e2e_value = job_throughput_gbs(w.kv_bytes, e2e_steps * w.layers, world, e2e_ms)
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
