@@ -87,7 +87,8 @@ typedef struct yoco_xattn_segment {
 typedef struct yoco_xattn_plan_info {
     int32_t mode;            /* YOCO_MODE_*                                               */
     int32_t tile_n;          /* keys per shared-memory tile                               */
-    int32_t tile_m;          /* query rows per CTA tile (16 decode, 128 chunk)            */
+    int32_t tile_m;          /* query rows per CTA: 16 decode; chunk 128, or 256 (two
+                                tensor-core tiles sharing K/V) when G*T > 128             */
     int32_t m_tiles;         /* row tiles per stream = ceil(G*T / tile_m)                 */
     int32_t num_groups;      /* CTA groups; each streams one contiguous range of the flat
                                 (stream, key tile) space                                  */

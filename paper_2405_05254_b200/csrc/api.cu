@@ -48,6 +48,7 @@ int32_t device_state(DeviceState** out) {
         YOCO_CUDA_TRY(cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev));
         YOCO_CUDA_TRY(decode_kernel_setup());
         YOCO_CUDA_TRY(chunk_kernel_setup());
+        YOCO_CUDA_TRY(chunk_pair_kernel_setup());
         st.ready = true;
     }
     *out = &st;
@@ -236,7 +237,10 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             p.rows_per_stream = plan.rows_per_stream;
             p.m_tiles = plan.info.m_tiles;
             p.d = shape->d;
-            YOCO_CUDA_TRY(launch_chunk(p, tmQ, tmK, tmV, plan.info.num_groups, stream));
+            if (plan.info.tile_m == kChunkPairTileM)
+                YOCO_CUDA_TRY(launch_chunk_pair(p, tmQ, tmK, tmV, plan.info.num_groups, stream));
+            else
+                YOCO_CUDA_TRY(launch_chunk(p, tmQ, tmK, tmV, plan.info.num_groups, stream));
         }
         if (prof) {
             ev = prof_event(true, &prof);

@@ -1,0 +1,461 @@
+// Multi-token chunk / full-sequence attention on the tcgen05 tensor cores, two row tiles per CTA.
+//
+// One CTA owns 256 of the G*T query rows of a (sequence, KV head) stream, as two 128-row tiles
+// that share every K/V tile brought into shared memory, and walks a contiguous range of 128-key
+// tiles.  Three warpgroups (384 threads):
+//   warpgroup 0   warp 0 = TMA producer (both Q tiles once per segment; K through a three-deep and
+//                 V through a two-deep ring), warps 1 and 2 = MMA issuers of row tiles 0 and 1
+//                 (the per-instruction issue cost is what limits one issuer), warp 3 idle; gives
+//                 most of its registers away
+//   warpgroup 1   softmax of row tile 0 (thread = query row)
+//   warpgroup 2   softmax of row tile 1
+// Every 128-key tile is processed as two 64-key half steps.  Tensor memory (512 columns):
+//   S_0^0 S_0^1 | S_1^0 S_1^1 | O_0 | O_1      (64 fp32 columns per S buffer, 128 per O)
+// S_r^h receives the scores of row tile r against half h of the key tile, so the scores of the
+// next half step are already being computed while a warpgroup works on the current one: the
+// softmax never waits for the tensor pipe and the tensor pipe never waits for one particular
+// softmax.  A softmax thread reads its S row, keeps the running max / sum, and writes P (bf16,
+// two per 32-bit column) over the first 32 columns of the same S buffer; O_r += P_r V then takes
+// P straight from tensor memory as the A operand, so P never touches shared memory.
+// O in tensor memory is rescaled only when a row max outgrew the reference by more than 2^8.
+// Every wait is bounded and reports through the status word.
+#include "kernels.h"
+#include "ptx.cuh"
+#include "tcgen05.cuh"
+
+namespace yoco {
+
+namespace {
+
+constexpr int BM = 128;                        // rows of one tensor-core tile
+constexpr int BN = kChunkTileN;                // 128 keys per shared-memory tile
+constexpr int BH = BN / 2;                     // keys per half step
+constexpr int kThreads = 384;
+constexpr int HALF_BYTES = 128 * 128;          // 128 rows x 64 bf16: one swizzled half tile
+constexpr uint32_t TMEM_COLS = 512;
+constexpr float kRescaleThreshold = 8.f;       // in log2 units: P stays below 2^8
+// Register split after launch.  The CTA starts with 168 registers per thread (what 384 threads
+// allow); warpgroup 0 gives back down to kRegsOther and the softmax warpgroups grow to
+// kRegsSoftmax.  The total must fit in what the CTA was launched with, or the request to grow
+// would never be granted.
+constexpr int kRegsLaunch = 168, kRegsSoftmax = 224, kRegsOther = 56;
+static_assert(128 * kRegsOther + 256 * kRegsSoftmax <= kRegsLaunch * kThreads, "register pool of the CTA");
+
+template <int D>
+struct PCfg {
+    static constexpr int HALVES = D / 64;
+    static constexpr int TILE_BYTES = HALVES * HALF_BYTES;     // one Q, K or V tile
+    static constexpr int K_STAGES = 3, V_STAGES = 2;
+    static constexpr int OFF_Q = 0;                            // two tiles
+    static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
+    static constexpr int OFF_V = OFF_K + K_STAGES * TILE_BYTES;
+    static constexpr int OFF_BAR = OFF_V + V_STAGES * TILE_BYTES;
+    static constexpr int NUM_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 10;
+    static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16;
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
+};
+
+// position in the CTA's flat sequence of (segment, key tile) pairs
+struct TileCursor {
+    int si, k0, k_begin, k_end, h;
+    uint32_t it;      // key tile number since the start of the CTA (selects ring stages and phases)
+    bool valid;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                  const __grid_constant__ CUtensorMap tmV, const ChunkParams p) {
+    using C = PCfg<D>;
+    constexpr int HALVES = C::HALVES;
+    constexpr int KS = C::K_STAGES, VS = C::V_STAGES;
+    constexpr int KSTEPS_QK = D / 16;
+    constexpr int KSTEPS_PV = BH / 16;
+
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR);
+    uint64_t* q_full = bars + 0;
+    uint64_t* q_empty = bars + 1;
+    uint64_t* k_full = bars + 2;             // [KS]
+    uint64_t* k_empty = k_full + KS;         // [KS]
+    uint64_t* v_full = k_empty + KS;         // [VS]
+    uint64_t* v_empty = v_full + VS;         // [VS]
+    uint64_t* s_full = v_empty + VS;         // [2][2]  S_r^h holds the scores of the current half step
+    uint64_t* p_full = s_full + 4;           // [2][2]  P_r^h has been written over S_r^h
+    uint64_t* pv_done = p_full + 4;          // [2]     O_r includes the current half step
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::NUM_BARS);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int group = blockIdx.x / p.m_tiles, m_tile = blockIdx.x - group * p.m_tiles;
+    const int seg_lo = p.group_begin[group], seg_hi = p.group_begin[group + 1];
+    const Abort ab{abort_flag, p.status};
+    const bool aligned_ok = (smem_u32(smem) & 1023u) == 0;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = aligned_ok ? 0 : 1;
+        if (!aligned_ok) atomicExch(p.status, kStatusTimeout + 1);
+        mbar_init(q_full, 1);
+        mbar_init(q_empty, 2);
+        for (int b = 0; b < KS; ++b) {
+            mbar_init(&k_full[b], 1);
+            mbar_init(&k_empty[b], 2);            // released by both issuers
+        }
+        for (int b = 0; b < VS; ++b) {
+            mbar_init(&v_full[b], 1);
+            mbar_init(&v_empty[b], 2);
+        }
+        for (int r = 0; r < 2; ++r) {
+            for (int h = 0; h < 2; ++h) {
+                mbar_init(&s_full[r * 2 + h], 1);
+                mbar_init(&p_full[r * 2 + h], 4);
+            }
+            mbar_init(&pv_done[r], 1);
+        }
+        mbar_fence_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < 4) {
+        setmaxnreg_dec<kRegsOther>();
+        if (warp == 0 && lane == 0 && aligned_ok) {
+            // =================================== TMA producer ================================
+            tma_prefetch_desc(&tmQ);
+            tma_prefetch_desc(&tmK);
+            tma_prefetch_desc(&tmV);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int si = seg_lo; si < seg_hi && ok; ++si) {
+                const DevSegment seg = p.segments[si];
+                const uint32_t sidx = si - seg_lo;
+                if (!(ok = wait_or_abort(q_empty, (sidx & 1u) ^ 1u, ab))) break;
+                mbar_expect_tx(q_full, 2 * C::TILE_BYTES);
+                for (int r = 0; r < 2; ++r)
+                    for (int h = 0; h < HALVES; ++h)
+                        tma_load_2d(smem + C::OFF_Q + r * C::TILE_BYTES + h * HALF_BYTES, &tmQ, h * 64,
+                                    seg.q_row0 + (m_tile * 2 + r) * BM, q_full);
+                for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
+                    const int row = seg.kv_row0 + (k0 - seg.k_begin);
+                    const uint32_t kb = it % KS, kn = it / KS;
+                    if (!(ok = wait_or_abort(&k_empty[kb], (kn & 1u) ^ 1u, ab))) break;
+                    mbar_expect_tx(&k_full[kb], C::TILE_BYTES);
+                    for (int h = 0; h < HALVES; ++h)
+                        tma_load_2d(smem + C::OFF_K + kb * C::TILE_BYTES + h * HALF_BYTES, &tmK, h * 64, row,
+                                    &k_full[kb]);
+                    const uint32_t vb = it % VS, vn = it / VS;
+                    if (!(ok = wait_or_abort(&v_empty[vb], (vn & 1u) ^ 1u, ab))) break;
+                    mbar_expect_tx(&v_full[vb], C::TILE_BYTES);
+                    for (int h = 0; h < HALVES; ++h)
+                        tma_load_2d(smem + C::OFF_V + vb * C::TILE_BYTES + h * HALF_BYTES, &tmV, h * 64, row,
+                                    &v_full[vb]);
+                }
+            }
+        } else if ((warp == 1 || warp == 2) && aligned_ok) {
+            // =================================== MMA issuer ==================================
+            // One issuer warp per row tile.  The whole warp walks the schedule (so that addresses
+            // and descriptors stay warp-uniform); one elected lane issues the tensor-core
+            // instructions.  The products of one row tile are issued by one thread and therefore
+            // execute in order; the two row tiles touch disjoint tensor memory.
+            const int r = warp - 1;
+            constexpr uint32_t idesc_qk = make_idesc(BH, false);
+            constexpr uint32_t idesc_pv = make_idesc(D, true);
+            const uint32_t sbase = smem_u32(smem);
+            // a cursor walks the CTA's flat sequence of half steps: (segment, key tile, half)
+            auto cur_load = [&](TileCursor& c) {
+                c.valid = c.si < seg_hi;
+                c.h = 0;
+                if (c.valid) {
+                    c.k_begin = c.k0 = p.segments[c.si].k_begin;
+                    c.k_end = p.segments[c.si].k_end;
+                }
+            };
+            auto cur_next = [&](TileCursor& c) {
+                if (c.h == 0) {
+                    c.h = 1;
+                    return;
+                }
+                c.h = 0;
+                ++c.it;
+                c.k0 += BN;
+                if (c.k0 >= c.k_end) {
+                    ++c.si;
+                    cur_load(c);
+                }
+            };
+            // S_r^h = Q_r K_h^T for the half step under cursor c
+            auto issue_qk = [&](const TileCursor& c) -> bool {
+                const uint32_t kb = c.it % KS, kn = c.it / KS;
+                if (c.h == 0) {
+                    if (c.k0 == c.k_begin && !warp_wait(q_full, (uint32_t)(c.si - seg_lo) & 1u, ab))
+                        return false;
+                    if (!warp_wait(&k_full[kb], kn & 1u, ab)) return false;
+                    tc_fence_after();
+                }
+                const uint64_t q_desc = make_desc(sbase + C::OFF_Q + r * C::TILE_BYTES, 16, 1024);
+                const uint64_t k_desc = make_desc(sbase + C::OFF_K + kb * C::TILE_BYTES + c.h * BH * 128, 16, 1024);
+                const uint32_t d_tmem = tmem_base + r * BN + c.h * BH;
+                if (elect_one()) {
+#pragma unroll
+                    for (int ks = 0; ks < KSTEPS_QK; ++ks) {
+                        const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                        umma_ss(d_tmem, q_desc + (off >> 4), k_desc + (off >> 4), idesc_qk, ks > 0 ? 1u : 0u);
+                    }
+                    umma_commit(&s_full[r * 2 + c.h]);
+                    if (c.h == 1) {
+                        umma_commit(&k_empty[kb]);
+                        if (c.k0 + BN >= c.k_end) umma_commit(q_empty);   // both Q tiles may be replaced
+                    }
+                }
+                __syncwarp();
+                return true;
+            };
+            // O_r += P_r^h V_h for the half step under cursor c
+            auto issue_pv = [&](const TileCursor& c) -> bool {
+                const uint32_t vb = c.it % VS, vn = c.it / VS;
+                if (!warp_wait(&p_full[r * 2 + c.h], c.it & 1u, ab)) return false;
+                if (c.h == 0 && !warp_wait(&v_full[vb], vn & 1u, ab)) return false;
+                tc_fence_after();
+                const uint64_t v_desc = make_desc(sbase + C::OFF_V + vb * C::TILE_BYTES + c.h * BH * 128, BN * 128, 1024);
+                const bool first = c.k0 == c.k_begin && c.h == 0;
+                const uint32_t a_tmem = tmem_base + r * BN + c.h * BH;
+                if (elect_one()) {
+#pragma unroll
+                    for (int ks = 0; ks < KSTEPS_PV; ++ks)
+                        umma_ts(tmem_base + 2 * BN + r * BN, a_tmem + ks * 8,
+                                v_desc + ((uint32_t)(ks * 16 * 128) >> 4), idesc_pv, (first && ks == 0) ? 0u : 1u);
+                    umma_commit(&pv_done[r]);
+                    if (c.h == 1) umma_commit(&v_empty[vb]);
+                }
+                __syncwarp();
+                return true;
+            };
+
+            TileCursor cq, cp;
+            cq.si = cp.si = seg_lo;
+            cq.it = cp.it = 0;
+            cur_load(cq);
+            cur_load(cp);
+            bool ok = true, pv_active = false;   // the first pass only issues the first half step's QK
+            while (ok && (cq.valid || pv_active)) {
+                // scores of the next half step first, so that the tensor pipe has work while the
+                // softmax warpgroups finish the current one
+                if (cq.valid) {
+                    ok = issue_qk(cq);
+                    cur_next(cq);
+                }
+                if (ok && pv_active) {
+                    ok = issue_pv(cp);
+                    cur_next(cp);
+                }
+                pv_active = cp.valid;
+            }
+        }
+    } else {
+        // ======================================= softmax warpgroups ==========================
+        setmaxnreg_inc<kRegsSoftmax>();
+        const int r = (warp >> 2) - 1;                 // row tile of this warpgroup
+        const int quad = warp & 3;                     // TMEM lane quadrant this warp may access
+        const int row = quad * 32 + lane;              // row inside the 128-row tile
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const uint32_t tmem_s = tmem_base + r * BN + lane_addr;
+        const uint32_t tmem_o = tmem_base + 2 * BN + r * BN + lane_addr;
+        const int r_local = (m_tile * 2 + r) * BM + row;   // row inside the stream's G*T rows
+        const bool row_valid = r_local < p.rows_per_stream;
+        uint32_t it = 0;
+        bool ok = aligned_ok;
+
+        for (int si = seg_lo; si < seg_hi; ++si) {
+            const DevSegment seg = p.segments[si];
+            const int n_full = seg.n_kv - p.T + 1;     // keys visible to every row
+            const int vis = min(seg.n_kv, max(0, n_full + (r_local % p.T)));
+            float m_ref = -INFINITY, l = 0.f;
+            const uint32_t seg_first_it = it, seg_first_u = 2 * it;
+
+            for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (!ok) continue;
+                    const uint32_t u = 2 * it + h;             // half step number
+                    const int kh = k0 + h * BH;                // first key of the half step
+                    if (!(ok = warp_wait(&s_full[r * 2 + h], it & 1u, ab))) continue;
+                    tc_fence_after();
+                    float s[BH];
+#pragma unroll
+                    for (int c = 0; c < BH / 32; ++c)
+                        tmem_ld32(tmem_s + h * BH + c * 32, *reinterpret_cast<float(*)[32]>(&s[c * 32]));
+                    tmem_wait_ld();
+
+                    if (kh + BH > n_full) {    // touches the causal edge or the sequence end
+#pragma unroll
+                        for (int j = 0; j < BH; ++j) s[j] = (kh + j < vis) ? s[j] : -INFINITY;
+                    }
+                    // row max of the raw scores (scale > 0, so it commutes with max)
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int j = 0; j < BH; j += 2) mx4[(j >> 1) & 3] = fmax3(mx4[(j >> 1) & 3], s[j], s[j + 1]);
+                    const float mx = fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * p.scale_log2;
+                    // lazy rescale: the reference max moves only when the row max outgrew it by 2^8
+                    float alpha = 1.f;
+                    const bool grow = mx > m_ref + kRescaleThreshold || (m_ref == -INFINITY && mx > -INFINITY);
+                    if (grow) {
+                        alpha = ex2_approx(m_ref - mx);               // 0 when m_ref = -inf
+                        m_ref = mx;
+                        l *= alpha;
+                    }
+                    if (__any_sync(0xffffffffu, grow) && u > seg_first_u) {
+                        // O_r holds the sums of the earlier half steps of this segment: wait for
+                        // the product of the previous one (the scores just read were issued after
+                        // the product two half steps back, so the barrier is at most one phase behind)
+                        if (!(ok = warp_wait(&pv_done[r], (u - 1) & 1u, ab))) continue;
+                        tc_fence_after();
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            float o[32];
+                            tmem_ld32(tmem_o + c * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) o[j] *= alpha;
+                            tmem_st32(tmem_o + c * 32, o);
+                        }
+                    }
+                    const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
+
+                    float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int c = 0; c < BH / 32; ++c) {                // 32 keys -> 16 packed columns
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float e0 = ex2_approx(fmaf(s[c * 32 + 2 * j], p.scale_log2, neg_m));
+                            const float e1 = ex2_approx(fmaf(s[c * 32 + 2 * j + 1], p.scale_log2, neg_m));
+                            ls4[j & 3] += e0 + e1;
+                            pk[j] = pack_bf16x2(e0, e1);
+                        }
+                        tmem_st16(tmem_s + h * BH + c * 16, pk);
+                    }
+                    l += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+                    tmem_wait_st();
+                    tc_fence_before();
+
+                    // keys past the end of the sequence: their V rows may hold anything; zero them
+                    // so that 0 * garbage cannot make NaN.  Both warpgroups write the same zeros in
+                    // the first half step, each before it releases its own first product on this tile.
+                    if (h == 0 && k0 + BN > seg.n_kv) {
+                        const uint32_t vb = it % VS, vn = it / VS;
+                        if (!(ok = warp_wait(&v_full[vb], vn & 1u, ab))) continue;
+                        if (k0 + row >= seg.n_kv) {
+                            uint8_t* vrow = smem + C::OFF_V + vb * C::TILE_BYTES + row * 128;
+#pragma unroll
+                            for (int hh = 0; hh < HALVES; ++hh)
+#pragma unroll
+                                for (int q = 0; q < 8; ++q)
+                                    *reinterpret_cast<uint4*>(vrow + hh * HALF_BYTES + q * 16) =
+                                        make_uint4(0u, 0u, 0u, 0u);
+                        }
+                        fence_proxy_async_smem();                   // generic writes -> tensor core reads
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&p_full[r * 2 + h]);
+                }
+            }
+
+            // ---- end of segment: O_r is complete once the last PV has finished ----
+            // (a parity wait is only meaningful for the phase in progress or the one before it.
+            // Having read the scores of the last half step, this warp knows that every product
+            // up to two half steps back has completed, so it steps through the last two phases.)
+            if (ok && it > seg_first_it)
+                ok = warp_wait(&pv_done[r], 0u, ab) && warp_wait(&pv_done[r], 1u, ab);
+            if (ok) {
+                tc_fence_after();
+                const bool has = l > 0.f;
+                const float inv = has ? 1.f / l : 0.f;
+                const float lse = has ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                const bool final_out = seg.stream_nseg == 1;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    float o[32];
+                    tmem_ld32(tmem_o + c * 32, o);
+                    tmem_wait_ld();
+                    if (row_valid) {
+                        if (final_out) {
+                            __nv_bfloat16* dst = p.O + ((int64_t)seg.q_row0 + r_local) * D + c * 32;
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                uint4 pk;
+                                pk.x = pack_bf16x2(has ? o[q * 8 + 0] * inv : 0.f, has ? o[q * 8 + 1] * inv : 0.f);
+                                pk.y = pack_bf16x2(has ? o[q * 8 + 2] * inv : 0.f, has ? o[q * 8 + 3] * inv : 0.f);
+                                pk.z = pack_bf16x2(has ? o[q * 8 + 4] * inv : 0.f, has ? o[q * 8 + 5] * inv : 0.f);
+                                pk.w = pack_bf16x2(has ? o[q * 8 + 6] * inv : 0.f, has ? o[q * 8 + 7] * inv : 0.f);
+                                *reinterpret_cast<uint4*>(dst + q * 8) = pk;
+                            }
+                        } else {
+                            float* dst = p.part_o + ((int64_t)seg.slot * p.rows_per_stream + r_local) * D + c * 32;
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                *reinterpret_cast<float4*>(dst + q * 4) =
+                                    make_float4(has ? o[q * 4 + 0] * inv : 0.f, has ? o[q * 4 + 1] * inv : 0.f,
+                                                has ? o[q * 4 + 2] * inv : 0.f, has ? o[q * 4 + 3] * inv : 0.f);
+                        }
+                    }
+                }
+                if (row_valid) {
+                    if (final_out) {
+                        if (p.lse) p.lse[seg.q_row0 + r_local] = lse;
+                    } else {
+                        p.part_lse[(int64_t)seg.slot * p.rows_per_stream + r_local] = lse;
+                    }
+                }
+                tc_fence_before();
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+template <int D>
+cudaError_t launch_one(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                       const CUtensorMap& tmV, int num_groups, cudaStream_t stream) {
+    chunk_pair_kernel<D><<<num_groups * p.m_tiles, kThreads, PCfg<D>::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, p);
+    return cudaGetLastError();
+}
+
+
+template <int D>
+cudaError_t setup_one() {
+    cudaError_t e = cudaFuncSetAttribute(chunk_pair_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         PCfg<D>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    // the register split inside the kernel assumes the launch allocation it was written for
+    cudaFuncAttributes attr;
+    if ((e = cudaFuncGetAttributes(&attr, chunk_pair_kernel<D>)) != cudaSuccess) return e;
+    return attr.numRegs >= kRegsLaunch ? cudaSuccess : cudaErrorLaunchOutOfResources;
+}
+
+}  // namespace
+
+cudaError_t chunk_pair_kernel_setup() {
+    cudaError_t e = setup_one<128>();
+    return e != cudaSuccess ? e : setup_one<64>();
+}
+
+cudaError_t launch_chunk_pair(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                              const CUtensorMap& tmV, int num_groups, cudaStream_t stream) {
+    if (num_groups <= 0) return cudaSuccess;
+    return p.d == 128 ? launch_one<128>(p, tmQ, tmK, tmV, num_groups, stream)
+                      : launch_one<64>(p, tmQ, tmK, tmV, num_groups, stream);
+}
+
+}  // namespace yoco

@@ -72,5 +72,10 @@ struct ChunkParams {
 cudaError_t launch_chunk(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                          const CUtensorMap& tmV, int num_groups, cudaStream_t stream);
 cudaError_t chunk_kernel_setup();
+// Same interface for streams with more than 128 rows: one CTA owns two 128-row tiles (m_tiles =
+// ceil(rows_per_stream / 256)), tmQ box is still {64, 128}.
+cudaError_t launch_chunk_pair(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                              const CUtensorMap& tmV, int num_groups, cudaStream_t stream);
+cudaError_t chunk_pair_kernel_setup();
 
 }  // namespace yoco

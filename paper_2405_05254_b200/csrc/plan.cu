@@ -28,7 +28,8 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     const int G = s.Hq / s.Hkv;
     const int rows_per_stream = G * s.T;
     const int tile_n = mode == YOCO_MODE_DECODE ? kDecodeTileN : kChunkTileN;
-    const int tile_m = mode == YOCO_MODE_DECODE ? kDecodeTileM : kChunkTileM;
+    const int tile_m = mode == YOCO_MODE_DECODE ? kDecodeTileM
+                       : rows_per_stream > kChunkTileM ? kChunkPairTileM : kChunkTileM;
     const int m_tiles = (rows_per_stream + tile_m - 1) / tile_m;
     const int num_streams = s.B * s.Hkv;
 

@@ -19,6 +19,8 @@ constexpr int kDecodeTileM = 16;      // query rows of one mma.sync tile
 constexpr int kDecodeGroupsPerSm = 2; // resident decode CTAs per SM
 constexpr int kChunkTileN = 128;      // keys per tcgen05 tile
 constexpr int kChunkTileM = 128;      // query rows per tcgen05 tile
+constexpr int kChunkPairTileM = 256;  // rows per CTA when a stream has more than 128 rows: two tiles
+                                      // that share every K/V tile in shared memory
 constexpr int kWorkspaceHeaderBytes = 256;
 
 // One work segment as the kernels read it (8 x int32 = 32 bytes).

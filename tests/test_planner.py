@@ -39,7 +39,7 @@ def test_strerror_covers_the_codes():
 def restated_plan(B, Hkv, lens, sm_count, mode, G, T):
     """Test-side restatement of the rule: flat (stream, tile) space cut into equal ranges."""
     tile_n = 64 if mode == bd.MODE_DECODE else 128
-    tile_m = 16 if mode == bd.MODE_DECODE else 128
+    tile_m = 16 if mode == bd.MODE_DECODE else (256 if G * T > 128 else 128)
     m_tiles = -(-G * T // tile_m)
     nts = [-(-int(n) // tile_n) for n in lens]
     total = Hkv * sum(nts)
