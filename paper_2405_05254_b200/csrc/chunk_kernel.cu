@@ -3,7 +3,7 @@
 // One CTA owns one 128-row tile of the G*T query rows of a (sequence, KV head) stream and walks
 // a contiguous range of 128-key tiles.  Roles (192 threads):
 //   warp 0      TMA producer: Q tile once per segment, K and V tiles through two-deep rings
-//   warp 1      MMA issuer: S = Q K^T (both operands K-major in shared memory) into one of two
+//   warp 1      MMA issuer (one elected lane): S = Q K^T (both operands K-major in shared memory) into one of two
 //               128-column TMEM buffers, then O += P V (P K-major, V MN-major) into a third
 //   warps 2..5  softmax: thread = query row; reads its S row from TMEM, keeps the running
 //               max / sum, writes P (bf16) back to shared memory in the swizzled operand layout,
@@ -127,7 +127,9 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         }
     } else if (warp == 1) {
         // ======================================= MMA issuer ==================================
-        if (lane == 0 && aligned_ok) {
+        // The whole warp walks the schedule, so that addresses and descriptors stay warp-uniform;
+        // one elected lane issues the tensor-core instructions.
+        if (aligned_ok) {
             constexpr uint32_t idesc_qk = make_idesc(BN, false);
             constexpr uint32_t idesc_pv = make_idesc(D, true);
             const uint32_t sbase = smem_u32(smem);
@@ -141,20 +143,23 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             uint32_t prev_it = 0;
             auto issue_pv = [&](uint32_t i, bool first_of_segment) -> bool {
                 const uint32_t b = i & 1u, n = i >> 1;
-                if (!wait_or_abort(&p_full[b], n & 1u, ab)) return false;
-                if (!wait_or_abort(&v_full[b], n & 1u, ab)) return false;
+                if (!warp_wait(&p_full[b], n & 1u, ab)) return false;
+                if (!warp_wait(&v_full[b], n & 1u, ab)) return false;
                 tc_fence_after();
                 const uint64_t p_desc = make_desc(sbase + C::OFF_P + b * C::P_BYTES, 16, 1024);
                 const uint64_t v_desc = make_desc(sbase + C::OFF_V + b * C::TILE_BYTES, BN * 128, 1024);
+                if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < KSTEPS_PV; ++ks) {
-                    const uint32_t a_off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-                    const uint32_t b_off = ks * 16 * 128;
-                    umma_ss(tmem_o, p_desc + (a_off >> 4), v_desc + (b_off >> 4), idesc_pv,
-                            (first_of_segment && ks == 0) ? 0u : 1u);
+                    for (int ks = 0; ks < KSTEPS_PV; ++ks) {
+                        const uint32_t a_off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                        const uint32_t b_off = ks * 16 * 128;
+                        umma_ss(tmem_o, p_desc + (a_off >> 4), v_desc + (b_off >> 4), idesc_pv,
+                                (first_of_segment && ks == 0) ? 0u : 1u);
+                    }
+                    umma_commit(&p_empty[b]);
+                    umma_commit(&v_empty[b]);
                 }
-                umma_commit(&p_empty[b]);
-                umma_commit(&v_empty[b]);
+                __syncwarp();
                 return true;
             };
             for (int si = seg_lo; si < seg_hi && ok; ++si) {
@@ -164,21 +169,25 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     if (!(ok = issue_pv(prev_it, prev_first))) break;
                     have_prev = false;
                 }
-                if (!(ok = wait_or_abort(q_full, sidx & 1u, ab))) break;
+                if (!(ok = warp_wait(q_full, sidx & 1u, ab))) break;
                 for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
                     const uint32_t b = it & 1u, n = it >> 1;
-                    if (!(ok = wait_or_abort(&k_full[b], n & 1u, ab))) break;
-                    if (!(ok = wait_or_abort(&s_empty[b], (n & 1u) ^ 1u, ab))) break;
+                    if (!(ok = warp_wait(&k_full[b], n & 1u, ab))) break;
+                    if (!(ok = warp_wait(&s_empty[b], (n & 1u) ^ 1u, ab))) break;
                     tc_fence_after();
                     const uint64_t k_desc = make_desc(sbase + C::OFF_K + b * C::TILE_BYTES, 16, 1024);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < KSTEPS_QK; ++ks) {
-                        const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-                        umma_ss(tmem_base + b * BN, q_desc + (off >> 4), k_desc + (off >> 4), idesc_qk, ks > 0 ? 1u : 0u);
+                        for (int ks = 0; ks < KSTEPS_QK; ++ks) {
+                            const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                            umma_ss(tmem_base + b * BN, q_desc + (off >> 4), k_desc + (off >> 4), idesc_qk,
+                                    ks > 0 ? 1u : 0u);
+                        }
+                        umma_commit(&s_full[b]);
+                        umma_commit(&k_empty[b]);
+                        if (k0 + BN >= seg.k_end) umma_commit(q_empty);   // Q may be replaced
                     }
-                    umma_commit(&s_full[b]);
-                    umma_commit(&k_empty[b]);
-                    if (k0 + BN >= seg.k_end) umma_commit(q_empty);   // Q may be replaced
+                    __syncwarp();
                     if (have_prev && !(ok = issue_pv(prev_it, prev_first))) break;
                     have_prev = true;
                     prev_it = it;

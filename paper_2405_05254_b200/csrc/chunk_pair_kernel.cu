@@ -4,9 +4,8 @@
 // that share every K/V tile brought into shared memory, and walks a contiguous range of 128-key
 // tiles.  Three warpgroups (384 threads):
 //   warpgroup 0   warp 0 = TMA producer (both Q tiles once per segment; K through a three-deep and
-//                 V through a two-deep ring), warps 1 and 2 = MMA issuers of row tiles 0 and 1
-//                 (the per-instruction issue cost is what limits one issuer), warp 3 idle; gives
-//                 most of its registers away
+//                 V through a two-deep ring), warps 1 and 2 = issuers of the score products of row
+//                 tiles 0 and 1, warp 3 = issuer of the PV products; gives most of its registers away
 //   warpgroup 1   softmax of row tile 0 (thread = query row)
 //   warpgroup 2   softmax of row tile 1
 // Every 128-key tile is processed as two 64-key half steps.  Tensor memory (512 columns):
@@ -50,15 +49,24 @@ struct PCfg {
     static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
     static constexpr int OFF_V = OFF_K + K_STAGES * TILE_BYTES;
     static constexpr int OFF_BAR = OFF_V + V_STAGES * TILE_BYTES;
-    static constexpr int NUM_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 10;
+    static constexpr int NUM_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 12;
     static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16;
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
 };
 
+// Which of the 16 score pairs of a 32-key chunk take the polynomial exponential: spread evenly so
+// that the two instruction streams interleave.
+constexpr int kPolyPairs = 4;
+__host__ __device__ constexpr bool poly_pair(int j) {
+    return ((j + 1) * kPolyPairs) / 16 != (j * kPolyPairs) / 16;
+}
+
 // position in the CTA's flat sequence of (segment, key tile) pairs
 struct TileCursor {
-    int si, k0, k_begin, k_end, h;
-    uint32_t it;      // key tile number since the start of the CTA (selects ring stages and phases)
+    int si, k0, k_end, h;
+    uint32_t tp;                 // parity of the key tile number since the start of the CTA
+    uint32_t kb, kph, vb, vph;   // ring stage and phase parity of the K and V tiles
+    bool first_tile;             // first key tile of its segment
     bool valid;
 };
 
@@ -82,7 +90,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     uint64_t* v_empty = v_full + VS;         // [VS]
     uint64_t* s_full = v_empty + VS;         // [2][2]  S_r^h holds the scores of the current half step
     uint64_t* p_full = s_full + 4;           // [2][2]  P_r^h has been written over S_r^h
-    uint64_t* pv_done = p_full + 4;          // [2]     O_r includes the current half step
+    uint64_t* pv_done = p_full + 4;          // [2][2]  O_r includes the current half step; P_r^h is dead
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -103,14 +111,14 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         for (int b = 0; b < VS; ++b) {
             mbar_init(&v_full[b], 1);
-            mbar_init(&v_empty[b], 2);
+            mbar_init(&v_empty[b], 1);
         }
         for (int r = 0; r < 2; ++r) {
             for (int h = 0; h < 2; ++h) {
                 mbar_init(&s_full[r * 2 + h], 1);
                 mbar_init(&p_full[r * 2 + h], 4);
+                mbar_init(&pv_done[r * 2 + h], 1);
             }
-            mbar_init(&pv_done[r], 1);
         }
         mbar_fence_init();
     }
@@ -157,104 +165,117 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                                     &v_full[vb]);
                 }
             }
-        } else if ((warp == 1 || warp == 2) && aligned_ok) {
-            // =================================== MMA issuer ==================================
-            // One issuer warp per row tile.  The whole warp walks the schedule (so that addresses
-            // and descriptors stay warp-uniform); one elected lane issues the tensor-core
-            // instructions.  The products of one row tile are issued by one thread and therefore
-            // execute in order; the two row tiles touch disjoint tensor memory.
-            const int r = warp - 1;
+        } else if (warp >= 1 && aligned_ok) {
+            // =================================== MMA issuers =================================
+            // Issuing a tensor-core instruction costs a single warp tens of cycles (a chain of
+            // dependent scalar instructions), about as long as the instruction runs, so the work is
+            // spread over three warps: warps 1 and 2 issue S_r = Q_r K^T for row tiles 0 and 1,
+            // warp 3 issues O_r += P_r V for both.  Each whole warp walks the schedule (addresses
+            // and descriptors stay warp-uniform) and one elected lane issues.  Instructions of
+            // different threads are ordered only through the barriers: a score product waits for
+            // the product that last read its buffer (pv_done), a PV product for its P (p_full).
             constexpr uint32_t idesc_qk = make_idesc(BH, false);
             constexpr uint32_t idesc_pv = make_idesc(D, true);
             const uint32_t sbase = smem_u32(smem);
-            // a cursor walks the CTA's flat sequence of half steps: (segment, key tile, half)
-            auto cur_load = [&](TileCursor& c) {
+            TileCursor c;
+            c.si = seg_lo;
+            c.h = 0;
+            c.tp = 0;
+            c.kb = c.kph = c.vb = c.vph = 0;
+            c.first_tile = false;
+            auto cur_load = [&]() {
                 c.valid = c.si < seg_hi;
-                c.h = 0;
                 if (c.valid) {
-                    c.k_begin = c.k0 = p.segments[c.si].k_begin;
+                    c.k0 = p.segments[c.si].k_begin;
                     c.k_end = p.segments[c.si].k_end;
+                    c.first_tile = true;
                 }
             };
-            auto cur_next = [&](TileCursor& c) {
+            auto cur_next = [&]() {      // one half step forward
                 if (c.h == 0) {
                     c.h = 1;
                     return;
                 }
                 c.h = 0;
-                ++c.it;
+                c.tp ^= 1u;
+                if (++c.kb == KS) {
+                    c.kb = 0;
+                    c.kph ^= 1u;
+                }
+                if (++c.vb == VS) {
+                    c.vb = 0;
+                    c.vph ^= 1u;
+                }
+                c.first_tile = false;
                 c.k0 += BN;
                 if (c.k0 >= c.k_end) {
                     ++c.si;
-                    cur_load(c);
+                    cur_load();
                 }
             };
-            // S_r^h = Q_r K_h^T for the half step under cursor c
-            auto issue_qk = [&](const TileCursor& c) -> bool {
-                const uint32_t kb = c.it % KS, kn = c.it / KS;
-                if (c.h == 0) {
-                    if (c.k0 == c.k_begin && !warp_wait(q_full, (uint32_t)(c.si - seg_lo) & 1u, ab))
-                        return false;
-                    if (!warp_wait(&k_full[kb], kn & 1u, ab)) return false;
-                    tc_fence_after();
-                }
-                const uint64_t q_desc = make_desc(sbase + C::OFF_Q + r * C::TILE_BYTES, 16, 1024);
-                const uint64_t k_desc = make_desc(sbase + C::OFF_K + kb * C::TILE_BYTES + c.h * BH * 128, 16, 1024);
-                const uint32_t d_tmem = tmem_base + r * BN + c.h * BH;
-                if (elect_one()) {
-#pragma unroll
-                    for (int ks = 0; ks < KSTEPS_QK; ++ks) {
-                        const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-                        umma_ss(d_tmem, q_desc + (off >> 4), k_desc + (off >> 4), idesc_qk, ks > 0 ? 1u : 0u);
-                    }
-                    umma_commit(&s_full[r * 2 + c.h]);
-                    if (c.h == 1) {
-                        umma_commit(&k_empty[kb]);
-                        if (c.k0 + BN >= c.k_end) umma_commit(q_empty);   // both Q tiles may be replaced
-                    }
-                }
-                __syncwarp();
-                return true;
-            };
-            // O_r += P_r^h V_h for the half step under cursor c
-            auto issue_pv = [&](const TileCursor& c) -> bool {
-                const uint32_t vb = c.it % VS, vn = c.it / VS;
-                if (!warp_wait(&p_full[r * 2 + c.h], c.it & 1u, ab)) return false;
-                if (c.h == 0 && !warp_wait(&v_full[vb], vn & 1u, ab)) return false;
-                tc_fence_after();
-                const uint64_t v_desc = make_desc(sbase + C::OFF_V + vb * C::TILE_BYTES + c.h * BH * 128, BN * 128, 1024);
-                const bool first = c.k0 == c.k_begin && c.h == 0;
-                const uint32_t a_tmem = tmem_base + r * BN + c.h * BH;
-                if (elect_one()) {
-#pragma unroll
-                    for (int ks = 0; ks < KSTEPS_PV; ++ks)
-                        umma_ts(tmem_base + 2 * BN + r * BN, a_tmem + ks * 8,
-                                v_desc + ((uint32_t)(ks * 16 * 128) >> 4), idesc_pv, (first && ks == 0) ? 0u : 1u);
-                    umma_commit(&pv_done[r]);
-                    if (c.h == 1) umma_commit(&v_empty[vb]);
-                }
-                __syncwarp();
-                return true;
-            };
+            cur_load();
+            bool ok = true;
+            uint32_t tiles_seen = 0;     // key tiles finished by this warp (phase 0 has no predecessor)
 
-            TileCursor cq, cp;
-            cq.si = cp.si = seg_lo;
-            cq.it = cp.it = 0;
-            cur_load(cq);
-            cur_load(cp);
-            bool ok = true, pv_active = false;   // the first pass only issues the first half step's QK
-            while (ok && (cq.valid || pv_active)) {
-                // scores of the next half step first, so that the tensor pipe has work while the
-                // softmax warpgroups finish the current one
-                if (cq.valid) {
-                    ok = issue_qk(cq);
-                    cur_next(cq);
+            if (warp < 3) {
+                const int r = warp - 1;
+                const uint32_t q_lo = desc_lo(sbase + C::OFF_Q + r * C::TILE_BYTES, 16);
+                uint32_t seg_par = 0;
+                while (ok && c.valid) {
+                    if (c.h == 0) {
+                        if (c.first_tile) {
+                            ok = warp_wait(q_full, seg_par, ab);
+                            seg_par ^= 1u;
+                        }
+                        ok = ok && warp_wait(&k_full[c.kb], c.kph, ab);
+                    }
+                    // the buffer S_r^h still holds the P of the previous key tile until its product ran
+                    if (ok && tiles_seen > 0) ok = warp_wait(&pv_done[r * 2 + c.h], c.tp ^ 1u, ab);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t k_lo = desc_lo(sbase + C::OFF_K + c.kb * C::TILE_BYTES + c.h * BH * 128, 16);
+                    const uint32_t d_tmem = tmem_base + r * BN + c.h * BH;
+                    if (elect_one()) {
+#pragma unroll
+                        for (int ks = 0; ks < KSTEPS_QK; ++ks) {
+                            const uint32_t off = ((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4;
+                            umma_ss(d_tmem, desc_from_lo(q_lo + off, 1024), desc_from_lo(k_lo + off, 1024), idesc_qk,
+                                    ks > 0 ? 1u : 0u);
+                        }
+                        umma_commit(&s_full[r * 2 + c.h]);
+                        if (c.h == 1) {
+                            umma_commit(&k_empty[c.kb]);
+                            if (c.k0 + BN >= c.k_end) umma_commit(q_empty);   // both Q tiles may be replaced
+                        }
+                    }
+                    __syncwarp();
+                    if (c.h == 1) ++tiles_seen;
+                    cur_next();
                 }
-                if (ok && pv_active) {
-                    ok = issue_pv(cp);
-                    cur_next(cp);
+            } else {
+                while (ok && c.valid) {
+                    if (c.h == 0) ok = warp_wait(&v_full[c.vb], c.vph, ab);
+                    const uint32_t v_lo = desc_lo(sbase + C::OFF_V + c.vb * C::TILE_BYTES + c.h * BH * 128, BN * 128);
+                    const uint32_t first = (c.first_tile && c.h == 0) ? 0u : 1u;
+#pragma unroll
+                    for (int r = 0; r < 2; ++r) {
+                        ok = ok && warp_wait(&p_full[r * 2 + c.h], c.tp, ab);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t a_tmem = tmem_base + r * BN + c.h * BH;
+                        if (elect_one()) {
+#pragma unroll
+                            for (int ks = 0; ks < KSTEPS_PV; ++ks)
+                                umma_ts(tmem_base + 2 * BN + r * BN, a_tmem + ks * 8,
+                                        desc_from_lo(v_lo + ((uint32_t)(ks * 16 * 128) >> 4), 1024), idesc_pv,
+                                        ks == 0 ? first : 1u);
+                            umma_commit(&pv_done[r * 2 + c.h]);
+                            if (r == 1 && c.h == 1) umma_commit(&v_empty[c.vb]);
+                        }
+                        __syncwarp();
+                    }
+                    cur_next();
                 }
-                pv_active = cp.valid;
             }
         }
     } else {
@@ -311,9 +332,9 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     }
                     if (__any_sync(0xffffffffu, grow) && u > seg_first_u) {
                         // O_r holds the sums of the earlier half steps of this segment: wait for
-                        // the product of the previous one (the scores just read were issued after
-                        // the product two half steps back, so the barrier is at most one phase behind)
-                        if (!(ok = warp_wait(&pv_done[r], (u - 1) & 1u, ab))) continue;
+                        // the product of the previous one (the other buffer; it belongs to this key
+                        // tile when h = 1, to the previous one when h = 0)
+                        if (!(ok = warp_wait(&pv_done[r * 2 + (h ^ 1)], (it ^ (h ^ 1)) & 1u, ab))) continue;
                         tc_fence_after();
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c) {
@@ -327,20 +348,54 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     }
                     const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
 
-                    float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+                    // P = 2^(s * scale - m_ref), two elements per instruction where the hardware
+                    // allows.  On tiles without masked keys, kPolyPairs of every 16 pairs take their
+                    // exponential on the FMA pipe so that the special-function unit (16 results per
+                    // clock per SM) is not the only limit.
+                    const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negm2 = f2_pack(neg_m, neg_m);
+                    uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};            // packed partial row sums
+                    const bool unmasked = kh + BH <= n_full;
 #pragma unroll
                     for (int c = 0; c < BH / 32; ++c) {                // 32 keys -> 16 packed columns
                         uint32_t pk[16];
+                        if (unmasked) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float e0 = ex2_approx(fmaf(s[c * 32 + 2 * j], p.scale_log2, neg_m));
-                            const float e1 = ex2_approx(fmaf(s[c * 32 + 2 * j + 1], p.scale_log2, neg_m));
-                            ls4[j & 3] += e0 + e1;
-                            pk[j] = pack_bf16x2(e0, e1);
+                            for (int j = 0; j < 16; ++j) {
+                                const uint64_t x2 = f2_fma(f2_pack(s[c * 32 + 2 * j], s[c * 32 + 2 * j + 1]), scale2, negm2);
+                                uint64_t e2;
+                                if (poly_pair(j)) {
+                                    e2 = f2_exp2_poly(x2);
+                                } else {
+                                    float x0, x1;
+                                    f2_unpack(x2, x0, x1);
+                                    e2 = f2_pack(ex2_approx(x0), ex2_approx(x1));
+                                }
+                                ls2[j & 3] = f2_add(ls2[j & 3], e2);
+                                float e0, e1;
+                                f2_unpack(e2, e0, e1);
+                                pk[j] = pack_bf16x2(e0, e1);
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const uint64_t x2 = f2_fma(f2_pack(s[c * 32 + 2 * j], s[c * 32 + 2 * j + 1]), scale2, negm2);
+                                float x0, x1;
+                                f2_unpack(x2, x0, x1);
+                                const uint64_t e2 = f2_pack(ex2_approx(x0), ex2_approx(x1));
+                                ls2[j & 3] = f2_add(ls2[j & 3], e2);
+                                float e0, e1;
+                                f2_unpack(e2, e0, e1);
+                                pk[j] = pack_bf16x2(e0, e1);
+                            }
                         }
                         tmem_st16(tmem_s + h * BH + c * 16, pk);
                     }
-                    l += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+                    {
+                        float a0, a1, b0, b1;
+                        f2_unpack(f2_add(ls2[0], ls2[1]), a0, a1);
+                        f2_unpack(f2_add(ls2[2], ls2[3]), b0, b1);
+                        l += (a0 + a1) + (b0 + b1);
+                    }
                     tmem_wait_st();
                     tc_fence_before();
 
@@ -367,11 +422,8 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             }
 
             // ---- end of segment: O_r is complete once the last PV has finished ----
-            // (a parity wait is only meaningful for the phase in progress or the one before it.
-            // Having read the scores of the last half step, this warp knows that every product
-            // up to two half steps back has completed, so it steps through the last two phases.)
-            if (ok && it > seg_first_it)
-                ok = warp_wait(&pv_done[r], 0u, ab) && warp_wait(&pv_done[r], 1u, ab);
+            // (the products of one row tile complete in order, so the last one covers all)
+            if (ok && it > seg_first_it) ok = warp_wait(&pv_done[r * 2 + 1], (it - 1) & 1u, ab);
             if (ok) {
                 tc_fence_after();
                 const bool has = l > 0.f;

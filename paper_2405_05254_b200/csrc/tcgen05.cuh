@@ -104,6 +104,50 @@ template <int N>
 __device__ __forceinline__ void setmaxnreg_dec() {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
+// ---- packed fp32 pairs (two lanes of one 64-bit register; one instruction does both) ---------
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// 2^x for a pair on the FMA pipe instead of the special-function unit: x = n + f with n the nearest
+// integer (magic-number rounding) and f in [-0.5, 0.5]; 2^f by a cubic fitted to 7.5e-5 relative
+// error (far below the bf16 rounding that follows); n is added to the exponent field.  x is
+// clamped to >= -125 so that the exponent stays in range: anything below comes out as ~2^-125,
+// which vanishes against a row sum >= 2^-8 (callers must not use this on masked scores, which
+// have to come out as exactly 0).
+__device__ __forceinline__ uint64_t f2_exp2_poly(uint64_t x2) {
+    float x0, x1;
+    f2_unpack(x2, x0, x1);
+    x2 = f2_pack(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+    const uint64_t magic = f2_pack(12582912.f, 12582912.f), neg_magic = f2_pack(-12582912.f, -12582912.f);
+    const uint64_t t2 = f2_add(x2, magic);                         // low mantissa bits = round(x)
+    const uint64_t n2 = f2_add(t2, neg_magic);                     // round(x) as a float
+    const uint64_t f2 = f2_fma(n2, f2_pack(-1.f, -1.f), x2);       // x - round(x)
+    uint64_t p2 = f2_fma(f2, f2_pack(0.0551716648042202f, 0.0551716648042202f),
+                         f2_pack(0.2426111400127411f, 0.2426111400127411f));
+    p2 = f2_fma(p2, f2, f2_pack(0.6932609677314758f, 0.6932609677314758f));
+    p2 = f2_fma(p2, f2, f2_pack(0.9999280571937561f, 0.9999280571937561f));
+    float p0, p1, t0, t1;
+    f2_unpack(p2, p0, p1);
+    f2_unpack(t2, t0, t1);
+    const float e0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
+    const float e1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
+    return f2_pack(e0, e1);
+}
 __device__ __forceinline__ float fmax3(float a, float b, float c) {   // one three-input max
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -121,6 +165,16 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
            ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// The same descriptor split in two: only the low word (address and leading-dimension offset)
+// changes from one instruction to the next, and stepping through a tile never carries out of the
+// 14-bit address field, so the issuer adds to a 32-bit value and pairs it with a constant.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+__device__ __forceinline__ uint64_t desc_from_lo(uint32_t lo, uint32_t sbo_bytes) {
+    const uint32_t hi = (sbo_bytes >> 4) | (1u << 14) | (2u << 29);
+    return ((uint64_t)hi << 32) | lo;
 }
 // Instruction descriptor: f32 accumulate, bf16 x bf16, M = 128, given N and B major-ness.
 __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major) {
