@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstring>
 #include <list>
+#include <memory>
 #include <mutex>
 
 #include "kernels.h"
@@ -65,19 +66,25 @@ struct PlanKey {
                mode == o.mode && lens == o.lens && cu == o.cu;
     }
 };
+// A cached plan with the launch-ready forms of its tables.
+struct ReadyPlan {
+    Plan plan;
+    std::vector<int32_t> blob;           // workspace image: zeroed header + tables (upload path)
+    bool fits_inline = false;            // tables small enough to travel as kernel parameters
+    DecodeInlineTables decode_tab;
+    CombineInlineTables combine_tab;
+};
 struct PlanEntry {
     PlanKey key;
-    Plan plan;
+    std::shared_ptr<const ReadyPlan> ready;
 };
 std::list<PlanEntry> g_plans;   // most recently used first
 constexpr size_t kPlanCacheEntries = 16;
 
-// Returns a copy-free pointer valid until the entry is evicted; callers hold g_mutex only
-// inside this function, so they copy what they need out of the plan before returning to the
-// user (the launch path below finishes with the plan before it can be evicted by this thread;
-// other threads may evict it, hence the shared_ptr-free design keeps a local copy).
+// Looks the plan up (most recently used first) or makes it.  The shared pointer keeps the entry
+// alive for the caller even if another thread evicts it from the cache meanwhile.
 int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t* lens, int32_t sm_count,
-                    int32_t mode, Plan& out) {
+                    int32_t mode, std::shared_ptr<const ReadyPlan>& out) {
     PlanKey key;
     std::memset(&key.shape, 0, sizeof key.shape);
     key.shape = s;
@@ -90,16 +97,33 @@ int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t*
         for (auto it = g_plans.begin(); it != g_plans.end(); ++it)
             if (it->key == key) {
                 g_plans.splice(g_plans.begin(), g_plans, it);
-                out = g_plans.front().plan;
+                out = g_plans.front().ready;
                 return YOCO_OK;
             }
     }
-    Plan plan;
-    int32_t rc = make_plan(s, cu, lens, sm_count, mode, plan);
+    auto ready = std::make_shared<ReadyPlan>();
+    int32_t rc = make_plan(s, cu, lens, sm_count, mode, ready->plan);
     if (rc != YOCO_OK) return rc;
-    out = plan;
+    const Plan& plan = ready->plan;
+    ready->blob.assign(kWorkspaceHeaderBytes / 4 + plan.table.size(), 0);
+    std::copy(plan.table.begin(), plan.table.end(), ready->blob.begin() + kWorkspaceHeaderBytes / 4);
+    ready->fits_inline = mode == YOCO_MODE_DECODE && plan.info.num_segments <= kInlineSegments &&
+                         plan.info.num_groups <= kInlineGroups && plan.info.num_streams <= kInlineStreams;
+    if (ready->fits_inline) {
+        std::memset(&ready->decode_tab, 0, sizeof ready->decode_tab);
+        std::memset(&ready->combine_tab, 0, sizeof ready->combine_tab);
+        std::memcpy(ready->decode_tab.seg, plan.table.data() + plan.off_segments,
+                    (size_t)plan.info.num_segments * sizeof(DevSegment));
+        std::memcpy(ready->decode_tab.group_begin, plan.table.data() + plan.off_group_begin,
+                    (size_t)(plan.info.num_groups + 1) * 4);
+        std::memcpy(ready->combine_tab.stream_base, plan.table.data() + plan.off_stream_base,
+                    (size_t)plan.info.num_streams * 4);
+        std::memcpy(ready->combine_tab.stream_nseg, plan.table.data() + plan.off_stream_nseg,
+                    (size_t)plan.info.num_streams * 4);
+    }
+    out = ready;
     std::lock_guard<std::mutex> lock(g_mutex);
-    g_plans.push_front(PlanEntry{std::move(key), std::move(plan)});
+    g_plans.push_front(PlanEntry{std::move(key), std::move(ready)});
     if (g_plans.size() > kPlanCacheEntries) g_plans.pop_back();
     return YOCO_OK;
 }
@@ -176,20 +200,25 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
     DeviceState* dev = nullptr;
     if ((rc = device_state(&dev)) != YOCO_OK) return rc;
 
-    Plan plan;
-    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, mode, plan)) != YOCO_OK)
+    std::shared_ptr<const ReadyPlan> ready;
+    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, mode, ready)) != YOCO_OK)
         return rc;
+    const Plan& plan = ready->plan;
     if ((int64_t)workspace_bytes < plan.info.workspace_bytes) return YOCO_ERR_WORKSPACE_TOO_SMALL;
 
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     const float scale = shape->scale != 0.f ? shape->scale : 1.f / std::sqrt((float)shape->d);
 
-    // header (status word = 0) + work tables in one copy
-    {
-        std::vector<int32_t> blob(kWorkspaceHeaderBytes / 4 + plan.table.size(), 0);
-        std::copy(plan.table.begin(), plan.table.end(), blob.begin() + kWorkspaceHeaderBytes / 4);
-        YOCO_CUDA_TRY(cudaMemcpyAsync(ws, blob.data(), blob.size() * 4, cudaMemcpyHostToDevice, stream));
+    const bool inline_tables = ready->fits_inline;
+    if (inline_tables) {
+        // the tables travel as kernel parameters: only the status word has to be cleared
+        YOCO_CUDA_TRY(cudaMemsetAsync(ws, 0, kWorkspaceHeaderBytes, stream));
+    } else {
+        // header (status word = 0) + work tables in one copy.  The source is pageable memory,
+        // which the runtime stages before the call returns, so the cache entry may go away.
+        YOCO_CUDA_TRY(cudaMemcpyAsync(ws, ready->blob.data(), ready->blob.size() * 4, cudaMemcpyHostToDevice,
+                                      stream));
     }
     const int32_t* table = reinterpret_cast<const int32_t*>(ws + plan.ws_table);
     float* part_lse = reinterpret_cast<float*>(ws + plan.ws_part_lse);
@@ -217,7 +246,8 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             p.T = shape->T;
             p.rows_per_stream = plan.rows_per_stream;
             p.d = shape->d;
-            YOCO_CUDA_TRY(launch_decode(p, tmK, tmV, plan.info.num_groups, stream));
+            YOCO_CUDA_TRY(launch_decode(p, tmK, tmV, plan.info.num_groups, stream,
+                                        inline_tables ? &ready->decode_tab : nullptr));
         } else {
             CUtensorMap tmQ, tmK, tmV;
             const int64_t q_rows = (int64_t)shape->B * shape->Hq * shape->T;
@@ -256,13 +286,17 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
         c.Hkv = shape->Hkv;
         c.T = shape->T;
         c.rows_per_stream = plan.rows_per_stream;
+        c.max_pieces = plan.info.max_splits;
         c.stream_base = table + plan.off_stream_base;
         c.stream_nseg = table + plan.off_stream_nseg;
         c.part_o = part_o;
         c.part_lse = part_lse;
         c.O = static_cast<__nv_bfloat16*>(O);
         c.lse = lse;
-        YOCO_CUDA_TRY(launch_combine(c, stream));
+        // directly behind the attention kernel (no event in between): its launch may overlap
+        // that kernel's tail
+        const bool chained = plan.info.num_segments > 0 && g_prof.events.empty();
+        YOCO_CUDA_TRY(launch_combine(c, stream, inline_tables ? &ready->combine_tab : nullptr, chained));
     }
     return YOCO_OK;
 }
@@ -344,10 +378,10 @@ int32_t yoco_xattn_decode_static(const yoco_xattn_shape* shape, const void* Q, c
     // size check first, on the host: nothing is enqueued for a problem that does not fit
     DeviceState* dev = nullptr;
     if ((rc = device_state(&dev)) != YOCO_OK) return rc;
-    Plan plan;
-    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, YOCO_MODE_DECODE, plan)) != YOCO_OK)
+    std::shared_ptr<const ReadyPlan> ready;
+    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, YOCO_MODE_DECODE, ready)) != YOCO_OK)
         return rc;
-    if ((size_t)plan.info.workspace_bytes > kStaticScratchBytes) return YOCO_ERR_STATIC_SCRATCH_EXCEEDED;
+    if ((size_t)ready->plan.info.workspace_bytes > kStaticScratchBytes) return YOCO_ERR_STATIC_SCRATCH_EXCEEDED;
     void* scratch = nullptr;
     if ((rc = static_scratch_address(&scratch)) != YOCO_OK) return rc;
     return run(shape, YOCO_MODE_DECODE, Q, K, V, cu_kv_host, kv_len_host, O, lse, scratch,
@@ -375,6 +409,7 @@ int32_t yoco_xattn_combine(int64_t rows, int32_t S, int32_t d, const float* part
     c.rows = rows;
     c.d = d;
     c.S = S;
+    c.max_pieces = S;
     c.stream_base = nullptr;
     c.stream_nseg = nullptr;
     c.part_o = part_o;

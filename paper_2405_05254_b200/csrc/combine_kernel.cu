@@ -2,7 +2,10 @@
 //
 //   lse = log sum_s exp(lse_s),   O = sum_s exp(lse_s - lse) * O_s
 //
-// One warp per output row; lanes cover the head dimension with 128-bit loads.
+// Lanes cover the head dimension with 128-bit loads.  With few pieces per row one warp merges a
+// row; with many (a long sequence cut into dozens of splits) the four warps of a CTA share the
+// pieces of one row, and the loop carries no load-to-branch dependence, so that several pieces are
+// in flight at once: the merge is a chain of dependent memory latencies otherwise.
 #include "kernels.h"
 
 namespace yoco {
@@ -11,11 +14,15 @@ namespace {
 
 constexpr int kCombineWarps = 4;
 
-// VEC = floats per lane (d = 32 * VEC for the packed widths, else generic loop)
-__global__ void __launch_bounds__(kCombineWarps * 32)
-combine_kernel(CombineParams p) {
+template <int WPR>   // warps per output row: 1 or kCombineWarps
+__device__ __forceinline__ void combine_body(const CombineParams& p) {
+    // When launched behind the attention kernel with programmatic stream serialisation, this
+    // grid may start before that kernel has finished: wait for it (and for its writes) here.
+    // Without that launch attribute the instruction returns at once.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * kCombineWarps + warp;
+    const int64_t row = WPR == 1 ? (int64_t)blockIdx.x * kCombineWarps + warp : (int64_t)blockIdx.x;
+    const int sub = WPR == 1 ? 0 : warp;
     if (row >= p.rows) return;
 
     // where this row's partials live
@@ -51,46 +58,107 @@ combine_kernel(CombineParams p) {
     for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
 
     __nv_bfloat16* out = p.O + row * p.d;
-    if (m == -INFINITY) {   // no piece carries weight (also nseg == 0)
-        for (int e = lane; e < p.d; e += 32) out[e] = __float2bfloat16(0.f);
-        if (p.lse && lane == 0) p.lse[row] = -INFINITY;
+    if (m == -INFINITY) {   // no piece carries weight (also nseg == 0); the same for every warp of the row
+        if (sub == 0) {
+            for (int e = lane; e < p.d; e += 32) out[e] = __float2bfloat16(0.f);
+            if (p.lse && lane == 0) p.lse[row] = -INFINITY;
+        }
         return;
     }
     float denom = 0.f;
     for (int s = lane; s < nseg; s += 32) {
         const float l = p.part_lse[lse_base + s * lse_stride];
-        if (l != -INFINITY) denom += __expf(l - m);
+        denom += l == -INFINITY ? 0.f : __expf(l - m);
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, o);
     const float inv = 1.f / denom;
 
-    // each lane owns 4 consecutive channels per 128-channel block
-    for (int e0 = lane * 4; e0 < p.d; e0 += 128) {
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = 0; s < nseg; ++s) {
-            const float l = p.part_lse[lse_base + s * lse_stride];
-            if (l == -INFINITY) continue;
-            const float w = __expf(l - m) * inv;
-            const float4 v = *reinterpret_cast<const float4*>(p.part_o + o_base + s * o_stride + e0);
-            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+    // each lane owns 4 consecutive channels of each 128-channel block (d <= 256: two blocks)
+    float4 acc[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+    const int e0 = lane * 4;
+#pragma unroll 4
+    for (int s = sub; s < nseg; s += WPR) {
+        const float l = p.part_lse[lse_base + s * lse_stride];
+        const float w = l == -INFINITY ? 0.f : __expf(l - m) * inv;
+        const float* src = p.part_o + o_base + s * o_stride;
+#pragma unroll
+        for (int blk = 0; blk < 2; ++blk) {
+            if (e0 + blk * 128 < p.d) {
+                const float4 v = *reinterpret_cast<const float4*>(src + e0 + blk * 128);
+                // an empty piece may hold anything: select, never multiply by zero
+                acc[blk].x += w != 0.f ? w * v.x : 0.f;
+                acc[blk].y += w != 0.f ? w * v.y : 0.f;
+                acc[blk].z += w != 0.f ? w * v.z : 0.f;
+                acc[blk].w += w != 0.f ? w * v.w : 0.f;
+            }
         }
-        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
-        uint2 pk;
-        pk.x = *reinterpret_cast<uint32_t*>(&lo);
-        pk.y = *reinterpret_cast<uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(out + e0) = pk;
+    }
+    if (WPR > 1) {
+        __shared__ float4 red[kCombineWarps][2][32];
+        red[warp][0][lane] = acc[0];
+        red[warp][1][lane] = acc[1];
+        __syncthreads();
+        if (warp != 0) return;
+#pragma unroll
+        for (int blk = 0; blk < 2; ++blk) {
+            float4 t = red[0][blk][lane];
+#pragma unroll
+            for (int w2 = 1; w2 < kCombineWarps; ++w2) {
+                const float4 u = red[w2][blk][lane];
+                t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+            }
+            acc[blk] = t;
+        }
+    }
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) {
+        if (e0 + blk * 128 < p.d) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(acc[blk].x, acc[blk].y), hi = __floats2bfloat162_rn(acc[blk].z, acc[blk].w);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&lo);
+            pk.y = *reinterpret_cast<uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(out + e0 + blk * 128) = pk;
+        }
     }
     if (p.lse && lane == 0) p.lse[row] = m + __logf(denom);
 }
 
+template <int WPR>
+__global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const CombineParams p) { combine_body<WPR>(p); }
+
+// stream tables as kernel parameters
+template <int WPR>
+__global__ void __launch_bounds__(kCombineWarps * 32)
+combine_kernel_inline(const CombineParams p0, const __grid_constant__ CombineInlineTables tab) {
+    CombineParams p = p0;
+    p.stream_base = tab.stream_base;
+    p.stream_nseg = tab.stream_nseg;
+    combine_body<WPR>(p);
+}
+
 }  // namespace
 
-cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream) {
+cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream, const CombineInlineTables* inline_tab,
+                           bool after_attention) {
     if (p.rows == 0) return cudaSuccess;
-    const int64_t blocks = (p.rows + kCombineWarps - 1) / kCombineWarps;
-    combine_kernel<<<(unsigned)blocks, kCombineWarps * 32, 0, stream>>>(p);
-    return cudaGetLastError();
+    const bool wide = p.max_pieces > kCombineWarps;      // many pieces per row: one CTA per row
+    const int64_t blocks = wide ? p.rows : (p.rows + kCombineWarps - 1) / kCombineWarps;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(kCombineWarps * 32);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_attention ? 1 : 0;
+    if (inline_tab)
+        return wide ? cudaLaunchKernelEx(&cfg, combine_kernel_inline<kCombineWarps>, p, *inline_tab)
+                    : cudaLaunchKernelEx(&cfg, combine_kernel_inline<1>, p, *inline_tab);
+    return wide ? cudaLaunchKernelEx(&cfg, combine_kernel<kCombineWarps>, p)
+                : cudaLaunchKernelEx(&cfg, combine_kernel<1>, p);
 }
 
 }  // namespace yoco

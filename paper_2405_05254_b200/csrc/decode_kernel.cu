@@ -42,9 +42,8 @@ __device__ __forceinline__ uint32_t ld_global_u32(const __nv_bfloat16* p) {
 }
 
 template <int D, int ROWS>
-__global__ void __launch_bounds__(kThreads, 2)
-decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-              const DecodeParams p) {
+__device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtensorMap& tmV,
+                                            const DecodeParams& p) {
     using C = Cfg<D, ROWS>;
     constexpr int STAGES = C::STAGES;
     constexpr int KSTEPS = D / 16;
@@ -60,6 +59,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int seg_lo = p.group_begin[blockIdx.x], seg_hi = p.group_begin[blockIdx.x + 1];
+    // lets a merge kernel queued behind this one be launched early; it still waits for this
+    // grid to finish before it reads anything
+    asm volatile("griddepcontrol.launch_dependents;");
 
     if ((smem_u32(smem) & 1023u) != 0) {   // the swizzle arithmetic below needs 1 KB alignment
         if (threadIdx.x == 0) atomicExch(p.status, kStatusTimeout + 1);
@@ -316,17 +318,42 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
 }
 
+// work tables in global memory (the workspace)
+template <int D, int ROWS>
+__global__ void __launch_bounds__(kThreads, 2)
+decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+              const DecodeParams p) {
+    decode_body<D, ROWS>(tmK, tmV, p);
+}
+
+// work tables as kernel parameters
+template <int D, int ROWS>
+__global__ void __launch_bounds__(kThreads, 2)
+decode_kernel_inline(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                     const DecodeParams p0, const __grid_constant__ DecodeInlineTables tab) {
+    DecodeParams p = p0;
+    p.segments = tab.seg;
+    p.group_begin = tab.group_begin;
+    decode_body<D, ROWS>(tmK, tmV, p);
+}
+
 template <int D, int ROWS>
 cudaError_t launch_one(const DecodeParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                       int num_groups, cudaStream_t stream) {
+                       int num_groups, cudaStream_t stream, const DecodeInlineTables* inline_tab) {
     using C = Cfg<D, ROWS>;
-    decode_kernel<D, ROWS><<<num_groups, kThreads, C::SMEM_BYTES, stream>>>(tmK, tmV, p);
+    if (inline_tab)
+        decode_kernel_inline<D, ROWS><<<num_groups, kThreads, C::SMEM_BYTES, stream>>>(tmK, tmV, p, *inline_tab);
+    else
+        decode_kernel<D, ROWS><<<num_groups, kThreads, C::SMEM_BYTES, stream>>>(tmK, tmV, p);
     return cudaGetLastError();
 }
 
 template <int D, int ROWS>
 cudaError_t setup_one() {
-    return cudaFuncSetAttribute(decode_kernel<D, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<D, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         Cfg<D, ROWS>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(decode_kernel_inline<D, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 Cfg<D, ROWS>::SMEM_BYTES);
 }
 
@@ -341,14 +368,14 @@ cudaError_t decode_kernel_setup() {
 }
 
 cudaError_t launch_decode(const DecodeParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                          int num_groups, cudaStream_t stream) {
+                          int num_groups, cudaStream_t stream, const DecodeInlineTables* tab) {
     if (num_groups <= 0) return cudaSuccess;
     const bool wide = p.rows_per_stream > 8;
     if (p.d == 128)
-        return wide ? launch_one<128, 16>(p, tmK, tmV, num_groups, stream)
-                    : launch_one<128, 8>(p, tmK, tmV, num_groups, stream);
-    return wide ? launch_one<64, 16>(p, tmK, tmV, num_groups, stream)
-                : launch_one<64, 8>(p, tmK, tmV, num_groups, stream);
+        return wide ? launch_one<128, 16>(p, tmK, tmV, num_groups, stream, tab)
+                    : launch_one<128, 8>(p, tmK, tmV, num_groups, stream, tab);
+    return wide ? launch_one<64, 16>(p, tmK, tmV, num_groups, stream, tab)
+                : launch_one<64, 8>(p, tmK, tmV, num_groups, stream, tab);
 }
 
 }  // namespace yoco

@@ -14,6 +14,20 @@ namespace yoco {
 constexpr int32_t kStatusOk = 0;
 constexpr int32_t kStatusTimeout = 1;
 
+// Work tables small enough to travel as kernel parameters (the decode call then needs no
+// host-to-device copy): every benchmark shape fits; larger problems read them from the workspace.
+constexpr int kInlineSegments = 448;
+constexpr int kInlineGroups = 303;
+constexpr int kInlineStreams = 256;
+struct DecodeInlineTables {
+    DevSegment seg[kInlineSegments];
+    int32_t group_begin[kInlineGroups + 1];
+};
+struct CombineInlineTables {
+    int32_t stream_base[kInlineStreams];
+    int32_t stream_nseg[kInlineStreams];
+};
+
 struct CombineParams {
     int64_t rows;               // output rows (B*Hq*T, or the public `rows`)
     int32_t d;
@@ -21,6 +35,7 @@ struct CombineParams {
     int32_t S;
     // internal slot-major layout
     int32_t Hq, Hkv, T, rows_per_stream;
+    int32_t max_pieces;         // most pieces any row has (S, or the plan's max_splits): picks the launch shape
     const int32_t* stream_base; // [B*Hkv] first slot of each stream
     const int32_t* stream_nseg; // [B*Hkv] slots of each stream
     const float* part_o;
@@ -28,7 +43,12 @@ struct CombineParams {
     __nv_bfloat16* O;
     float* lse;                 // may be null
 };
-cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream);
+// inline_tab (host, may be null): stream tables passed as kernel parameters instead of
+// p.stream_base / p.stream_nseg.  after_attention: launched right behind the attention kernel of
+// the same call; the launch is then allowed to overlap that kernel's tail (the merge itself still
+// waits for it).
+cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream,
+                           const CombineInlineTables* inline_tab = nullptr, bool after_attention = false);
 
 struct DecodeParams {
     const __nv_bfloat16* Q;     // [B*Hq*T, d]
@@ -46,8 +66,10 @@ struct DecodeParams {
 };
 // tmK / tmV: 2-D tensor maps over the [rows, d] view of K and V, box {64, kDecodeTileN},
 // 128-byte swizzle.
+// inline_tab (host, may be null): segments and group offsets passed as kernel parameters instead
+// of p.segments / p.group_begin.
 cudaError_t launch_decode(const DecodeParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                          int num_groups, cudaStream_t stream);
+                          int num_groups, cudaStream_t stream, const DecodeInlineTables* inline_tab = nullptr);
 // one-time per-device kernel attribute set-up (dynamic shared memory opt-in)
 cudaError_t decode_kernel_setup();
 
