@@ -37,7 +37,7 @@ def _load():
         build()
         lib = ctypes.CDLL(_LIB)
         i32, i64, f64, ptr = ctypes.c_int32, ctypes.c_int64, ctypes.c_double, ctypes.c_void_p
-        common = [i32, i32, i32, i32, i32, f64, ptr, ptr, ptr, ptr, ptr, i64]
+        common = [i32, i32, i32, i32, i32, f64, ptr, ptr, ptr, ptr, ptr, i64, i32]
         lib.oracle_xattn.argtypes = common + [ptr, ptr]
         lib.oracle_xattn_rows.argtypes = common + [i64, ptr, ptr, ptr, ptr, ptr]
         lib.oracle_xattn_split_merge.argtypes = common + [i32, ptr, ptr, ptr]
@@ -80,20 +80,22 @@ def _check_extent(K, V, cu, kv_len, Hkv, d, kv_head_stride):
         raise ValueError("K/V buffers are smaller than the layout requires")
 
 
-def xattn(Q, K, V, cu, kv_len, *, B, Hq, Hkv, d, T, scale=0.0, kv_head_stride=0):
-    """Definition of the cross-attention; returns (O [B,Hq,T,d], LSE [B,Hq,T]) in fp64."""
+def xattn(Q, K, V, cu, kv_len, *, B, Hq, Hkv, d, T, scale=0.0, kv_head_stride=0, window=0):
+    """Definition of the cross-attention; returns (O [B,Hq,T,d], LSE [B,Hq,T]) in fp64.
+    ``window`` = C > 0 keeps, for the row at position i, only the keys i - C < j <= i (the
+    sliding-window mask of Section 3.2); 0 = plain causal."""
     Q, K, V, cu, kv_len = _prep(Q, K, V, cu, kv_len, B, Hq, T, d)
     _check_extent(K, V, cu, kv_len, Hkv, d, kv_head_stride)
     O = np.empty((B, Hq, T, d), dtype=np.float64)
     LSE = np.empty((B, Hq, T), dtype=np.float64)
     rc = _load().oracle_xattn(B, Hq, Hkv, d, T, float(scale), _p(Q), _p(K), _p(V), _p(cu),
-                              _p(kv_len), int(kv_head_stride), _p(O), _p(LSE))
+                              _p(kv_len), int(kv_head_stride), int(window), _p(O), _p(LSE))
     if rc:
         raise ValueError(f"oracle_xattn failed ({rc})")
     return O, LSE
 
 
-def xattn_rows(Q, K, V, cu, kv_len, rows, *, B, Hq, Hkv, d, T, scale=0.0, kv_head_stride=0):
+def xattn_rows(Q, K, V, cu, kv_len, rows, *, B, Hq, Hkv, d, T, scale=0.0, kv_head_stride=0, window=0):
     """Same definition for selected rows; ``rows`` is an (n, 3) array of (b, h, t)."""
     Q, K, V, cu, kv_len = _prep(Q, K, V, cu, kv_len, B, Hq, T, d)
     _check_extent(K, V, cu, kv_len, Hkv, d, kv_head_stride)
@@ -105,14 +107,14 @@ def xattn_rows(Q, K, V, cu, kv_len, rows, *, B, Hq, Hkv, d, T, scale=0.0, kv_hea
     O = np.empty((n, d), dtype=np.float64)
     LSE = np.empty((n,), dtype=np.float64)
     rc = _load().oracle_xattn_rows(B, Hq, Hkv, d, T, float(scale), _p(Q), _p(K), _p(V), _p(cu),
-                                   _p(kv_len), int(kv_head_stride), n, _p(rb), _p(rh), _p(rt),
+                                   _p(kv_len), int(kv_head_stride), int(window), n, _p(rb), _p(rh), _p(rt),
                                    _p(O), _p(LSE))
     if rc:
         raise ValueError(f"oracle_xattn_rows failed ({rc})")
     return O, LSE
 
 
-def xattn_split_merge(Q, K, V, cu, kv_len, cuts, *, B, Hq, Hkv, d, T, scale=0.0, kv_head_stride=0):
+def xattn_split_merge(Q, K, V, cu, kv_len, cuts, *, B, Hq, Hkv, d, T, scale=0.0, kv_head_stride=0, window=0):
     """The attention evaluated piecewise between the key positions ``cuts`` and merged by LSE."""
     Q, K, V, cu, kv_len = _prep(Q, K, V, cu, kv_len, B, Hq, T, d)
     _check_extent(K, V, cu, kv_len, Hkv, d, kv_head_stride)
@@ -120,7 +122,7 @@ def xattn_split_merge(Q, K, V, cu, kv_len, cuts, *, B, Hq, Hkv, d, T, scale=0.0,
     O = np.empty((B, Hq, T, d), dtype=np.float64)
     LSE = np.empty((B, Hq, T), dtype=np.float64)
     rc = _load().oracle_xattn_split_merge(B, Hq, Hkv, d, T, float(scale), _p(Q), _p(K), _p(V),
-                                          _p(cu), _p(kv_len), int(kv_head_stride),
+                                          _p(cu), _p(kv_len), int(kv_head_stride), int(window),
                                           int(cuts.size), _p(cuts), _p(O), _p(LSE))
     if rc:
         raise ValueError(f"oracle_xattn_split_merge failed ({rc})")

@@ -24,6 +24,11 @@
  *
  * Two passes over the keys (max, then sums); no tiling, no online rescaling.
  *
+ * Optional sliding window (Section 3.2, the window causal mask B_ij = 0 iff
+ * i - C < j <= i, -inf otherwise): with window C > 0 the row at absolute position
+ * i = N_i - T + t sees only the keys j with i - C < j <= i, i.e. the C most recent
+ * ones, itself included.  C = 0 means no window (plain causal).
+ *
  * Layout (the same bits the GPU reads): Q is [B, Hq, T, d] bf16.  K and V are
  * packed buffers of bf16; sequence i starts at token offset cu[i]; inside a
  * sequence the order is [Hkv, N_i, d] (head-major), the distance between heads
@@ -69,6 +74,7 @@ typedef struct {
     const int32_t *cu;
     const int32_t *kv_len;
     int64_t kv_head_stride;
+    int32_t window;
 } problem_t;
 
 static int64_t kv_base(const problem_t *p, int i, int c)
@@ -83,6 +89,16 @@ static int64_t visible_keys(const problem_t *p, int i, int t)
     if (n < 0) n = 0;
     if (n > p->kv_len[i]) n = p->kv_len[i];
     return n;
+}
+
+/* First key of the row's window: the mask keeps i - C < j, so the lowest kept j is
+ * i - C + 1 (never below 0); without a window every key from 0 on is kept. */
+static int64_t first_visible(const problem_t *p, int i, int t)
+{
+    if (p->window <= 0) return 0;
+    int64_t pos = (int64_t)p->kv_len[i] - p->T + t;   /* absolute position of the query row */
+    int64_t lo = pos - p->window + 1;
+    return lo < 0 ? 0 : lo;
 }
 
 /* Attention of one query row over keys [j0, j1) of its KV head (already
@@ -139,11 +155,11 @@ static int check_shape(int B, int Hq, int Hkv, int d, int T)
 /* Full output: O [B, Hq, T, d] and LSE [B, Hq, T], both fp64. */
 int oracle_xattn(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t T, double scale,
                  const uint16_t *Q, const uint16_t *K, const uint16_t *V,
-                 const int32_t *cu, const int32_t *kv_len, int64_t kv_head_stride,
+                 const int32_t *cu, const int32_t *kv_len, int64_t kv_head_stride, int32_t window,
                  double *O, double *LSE)
 {
-    if (check_shape(B, Hq, Hkv, d, T)) return -1;
-    problem_t p = {B, Hq, Hkv, d, T, resolve_scale(scale, d), Q, K, V, cu, kv_len, kv_head_stride};
+    if (check_shape(B, Hq, Hkv, d, T) || window < 0) return -1;
+    problem_t p = {B, Hq, Hkv, d, T, resolve_scale(scale, d), Q, K, V, cu, kv_len, kv_head_stride, window};
     int64_t max_len = 1;
     for (int i = 0; i < B; ++i)
         if (kv_len[i] > max_len) max_len = kv_len[i];
@@ -161,7 +177,7 @@ int oracle_xattn(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t T, doubl
                 if (!scores) continue;
                 for (int t = 0; t < T; ++t) {
                     int64_t row = ((int64_t)i * Hq + h) * T + t;
-                    row_over_range(&p, i, h, t, 0, visible_keys(&p, i, t), scores,
+                    row_over_range(&p, i, h, t, first_visible(&p, i, t), visible_keys(&p, i, t), scores,
                                    O + row * d, LSE + row);
                 }
             }
@@ -173,12 +189,12 @@ int oracle_xattn(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t T, doubl
 /* Selected rows only: row r is (rows_b[r], rows_h[r], rows_t[r]); O [n_rows, d], LSE [n_rows]. */
 int oracle_xattn_rows(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t T, double scale,
                       const uint16_t *Q, const uint16_t *K, const uint16_t *V,
-                      const int32_t *cu, const int32_t *kv_len, int64_t kv_head_stride,
+                      const int32_t *cu, const int32_t *kv_len, int64_t kv_head_stride, int32_t window,
                       int64_t n_rows, const int32_t *rows_b, const int32_t *rows_h,
                       const int32_t *rows_t, double *O, double *LSE)
 {
-    if (check_shape(B, Hq, Hkv, d, T)) return -1;
-    problem_t p = {B, Hq, Hkv, d, T, resolve_scale(scale, d), Q, K, V, cu, kv_len, kv_head_stride};
+    if (check_shape(B, Hq, Hkv, d, T) || window < 0) return -1;
+    problem_t p = {B, Hq, Hkv, d, T, resolve_scale(scale, d), Q, K, V, cu, kv_len, kv_head_stride, window};
     for (int64_t r = 0; r < n_rows; ++r)
         if (rows_b[r] < 0 || rows_b[r] >= B || rows_h[r] < 0 || rows_h[r] >= Hq ||
             rows_t[r] < 0 || rows_t[r] >= T)
@@ -198,7 +214,7 @@ int oracle_xattn_rows(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t T, 
         for (int64_t r = 0; r < n_rows; ++r) {
             if (!scores) continue;
             int i = rows_b[r], t = rows_t[r];
-            row_over_range(&p, i, rows_h[r], t, 0, visible_keys(&p, i, t), scores,
+            row_over_range(&p, i, rows_h[r], t, first_visible(&p, i, t), visible_keys(&p, i, t), scores,
                            O + r * d, LSE + r);
         }
         free(scores);
@@ -238,13 +254,13 @@ static void merge_pieces(int S, int d, const double *po, const double *plse,
  * pieces are merged by log-sum-exp.  Used to check "split + merge = unsplit". */
 int oracle_xattn_split_merge(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t T, double scale,
                              const uint16_t *Q, const uint16_t *K, const uint16_t *V,
-                             const int32_t *cu, const int32_t *kv_len, int64_t kv_head_stride,
+                             const int32_t *cu, const int32_t *kv_len, int64_t kv_head_stride, int32_t window,
                              int32_t n_cuts, const int64_t *cuts, double *O, double *LSE)
 {
-    if (check_shape(B, Hq, Hkv, d, T) || n_cuts < 0) return -1;
+    if (check_shape(B, Hq, Hkv, d, T) || n_cuts < 0 || window < 0) return -1;
     for (int k = 1; k < n_cuts; ++k)
         if (cuts[k] < cuts[k - 1]) return -1;
-    problem_t p = {B, Hq, Hkv, d, T, resolve_scale(scale, d), Q, K, V, cu, kv_len, kv_head_stride};
+    problem_t p = {B, Hq, Hkv, d, T, resolve_scale(scale, d), Q, K, V, cu, kv_len, kv_head_stride, window};
     int64_t max_len = 1;
     for (int i = 0; i < B; ++i)
         if (kv_len[i] > max_len) max_len = kv_len[i];
@@ -259,11 +275,11 @@ int oracle_xattn_split_merge(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int3
     for (int i = 0; i < B; ++i)
         for (int h = 0; h < Hq; ++h)
             for (int t = 0; t < T; ++t) {
-                int64_t n_vis = visible_keys(&p, i, t);
+                int64_t n_vis = visible_keys(&p, i, t), n_lo = first_visible(&p, i, t);
                 for (int s = 0; s < S; ++s) {
                     int64_t j0 = s == 0 ? 0 : cuts[s - 1];
                     int64_t j1 = s == n_cuts ? n_vis : cuts[s];
-                    if (j0 < 0) j0 = 0;
+                    if (j0 < n_lo) j0 = n_lo;
                     if (j1 > n_vis) j1 = n_vis;
                     if (j0 > n_vis) j0 = n_vis;
                     row_over_range(&p, i, h, t, j0, j1, scores, po + (int64_t)s * d, plse + s);
