@@ -24,8 +24,10 @@
  *          Both buffers must start on a 16-byte boundary.
  *   kv_len[i] = N_i  counts ALL keys of sequence i including the T positions of
  *          the current call (the self-decoder has already appended them).
- *   Causal rule: query row t (0-based, T rows) sees keys j <= N_i - T + t.
- *          T = 1 sees the whole cache.  A row with no visible key yields O = 0
+ *   Causal rule: query row t (0-based, T rows) sits at position i = N_i - T + t and sees keys
+ *          j <= i.  T = 1 sees the whole cache.  With shape.window = C > 0 it sees only
+ *          i - C < j <= i (the sliding-window mask of Section 3.2, B_ij = 0 iff i - C < j <= i);
+ *          keys that no row of the call can see are neither read nor planned.  A row with no visible key yields O = 0
  *          and LSE = -inf.
  *   LSE    [B, Hq, T] fp32, natural logarithm of sum_j exp(scale * q.k_j); optional.
  *
@@ -70,7 +72,8 @@ typedef struct yoco_xattn_shape {
     float   scale;           /* > 0, or 0 -> 1/sqrt(d); negative values are rejected       */
     int64_t kv_head_stride;  /* elements between KV heads of one sequence; 0 -> N_i*d     */
     int32_t max_kv_len;      /* used as every N_i when kv_len_host is NULL                */
-    int32_t reserved;        /* must be 0                                                 */
+    int32_t window;          /* sliding window C (Section 3.2: row i sees i - C < j <= i);
+                                0 = none (plain causal); negative values are rejected     */
 } yoco_xattn_shape;
 
 /* One unit of work: a contiguous key range of one (sequence, KV head) stream,

@@ -23,7 +23,7 @@ class Shape(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32),
                 ("d", ctypes.c_int32), ("T", ctypes.c_int32), ("scale", ctypes.c_float),
                 ("kv_head_stride", ctypes.c_int64), ("max_kv_len", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("window", ctypes.c_int32)]
 
 
 class Segment(ctypes.Structure):
@@ -79,8 +79,9 @@ def lib() -> ctypes.CDLL:
     return _lib
 
 
-def make_shape(B, Hq, Hkv, d, T, scale=0.0, kv_head_stride=0, max_kv_len=0) -> Shape:
-    return Shape(B, Hq, Hkv, d, T, float(scale), int(kv_head_stride), int(max_kv_len), 0)
+def make_shape(B, Hq, Hkv, d, T, scale=0.0, kv_head_stride=0, max_kv_len=0, window=0) -> Shape:
+    """``window`` = C > 0 selects the sliding-window mask (row i sees i - C < j <= i); 0 = none."""
+    return Shape(B, Hq, Hkv, d, T, float(scale), int(kv_head_stride), int(max_kv_len), int(window))
 
 
 def _host_i32(a):

@@ -211,6 +211,9 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             const DevSegment seg = p.segments[si];
             const int n_full = seg.n_kv - p.T + 1;     // keys visible to every row
             const int vis = min(seg.n_kv, max(0, n_full + (r_local % p.T)));
+            // sliding window: the row at position i keeps i - C < j; lo_max is the highest such bound
+            const int lo = p.window > 0 ? max(0, n_full + (r_local % p.T) - p.window) : 0;
+            const int lo_max = p.window > 0 ? seg.n_kv - p.window : 0;
             float m_ref = -INFINITY, l = 0.f;
             const uint32_t seg_first_it = it;
 
@@ -230,9 +233,9 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
                 // row max of the raw scores (scale > 0, so it commutes with max); four independent
                 // chains keep the dependent-latency off the critical path
-                if (k0 + BN > n_full) {        // tile touches the causal edge or the sequence end
+                if (k0 + BN > n_full || k0 < lo_max) {   // causal edge, sequence end or window start
 #pragma unroll
-                    for (int j = 0; j < BN; ++j) s[j] = (k0 + j < vis) ? s[j] : -INFINITY;
+                    for (int j = 0; j < BN; ++j) s[j] = (k0 + j < vis && k0 + j >= lo) ? s[j] : -INFINITY;
                 }
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll

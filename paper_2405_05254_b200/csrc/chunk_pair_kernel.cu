@@ -296,6 +296,9 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const DevSegment seg = p.segments[si];
             const int n_full = seg.n_kv - p.T + 1;     // keys visible to every row
             const int vis = min(seg.n_kv, max(0, n_full + (r_local % p.T)));
+            // sliding window: the row at position i keeps i - C < j; lo_max is the highest such bound
+            const int lo = p.window > 0 ? max(0, n_full + (r_local % p.T) - p.window) : 0;
+            const int lo_max = p.window > 0 ? seg.n_kv - p.window : 0;
             float m_ref = -INFINITY, l = 0.f;
             const uint32_t seg_first_it = it, seg_first_u = 2 * it;
 
@@ -313,9 +316,10 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         tmem_ld32(tmem_s + h * BH + c * 32, *reinterpret_cast<float(*)[32]>(&s[c * 32]));
                     tmem_wait_ld();
 
-                    if (kh + BH > n_full) {    // touches the causal edge or the sequence end
+                    const bool unmasked = kh + BH <= n_full && kh >= lo_max;
+                    if (!unmasked) {           // causal edge, sequence end or window start
 #pragma unroll
-                        for (int j = 0; j < BH; ++j) s[j] = (kh + j < vis) ? s[j] : -INFINITY;
+                        for (int j = 0; j < BH; ++j) s[j] = (kh + j < vis && kh + j >= lo) ? s[j] : -INFINITY;
                     }
                     // row max of the raw scores (scale > 0, so it commutes with max)
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -354,7 +358,6 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     // clock per SM) is not the only limit.
                     const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negm2 = f2_pack(neg_m, neg_m);
                     uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};            // packed partial row sums
-                    const bool unmasked = kh + BH <= n_full;
 #pragma unroll
                     for (int c = 0; c < BH / 32; ++c) {                // 32 keys -> 16 packed columns
                         uint32_t pk[16];

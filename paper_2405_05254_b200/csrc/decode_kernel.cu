@@ -173,7 +173,15 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
                     }
                 }
                 // ---- scale, mask, online softmax ----
-                const bool need_mask = kw + 16 > n_full;
+                // sliding window: the row at position i = n_kv - T + t keeps i - C < j, i.e.
+                // j >= i - C + 1 = n_full + t - C; the highest such bound of any row is n_kv - C
+                const bool need_mask = kw + 16 > n_full || (p.window > 0 && kw < seg.n_kv - p.window);
+                // window start of the two rows this lane holds (no window: below every key)
+                int lo0 = -1, lo1 = -1;
+                if (need_mask && p.window > 0) {
+                    lo0 = n_full + (g % p.T) - p.window;
+                    lo1 = n_full + ((g + 8) % p.T) - p.window;
+                }
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
@@ -181,7 +189,7 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
                         float v = s[nt][e] * p.scale_log2;
                         if (need_mask) {
                             const int j = kw + nt * 8 + tq * 2 + (e & 1);
-                            v = j < ((e & 2) ? vis1 : vis0) ? v : -INFINITY;
+                            v = (j < ((e & 2) ? vis1 : vis0) && j >= ((e & 2) ? lo1 : lo0)) ? v : -INFINITY;
                         }
                         s[nt][e] = v;
                     }

@@ -63,6 +63,7 @@ struct DecodeParams {
     int32_t T;
     int32_t rows_per_stream;    // G * T (<= 16)
     int32_t d;
+    int32_t window;             // sliding window C, 0 = none
 };
 // tmK / tmV: 2-D tensor maps over the [rows, d] view of K and V, box {64, kDecodeTileN},
 // 128-byte swizzle.
@@ -87,6 +88,7 @@ struct ChunkParams {
     int32_t rows_per_stream;    // G * T
     int32_t m_tiles;            // ceil(rows_per_stream / 128)
     int32_t d;
+    int32_t window;             // sliding window C, 0 = none
 };
 // tmQ: [B*Hq*T, d] box {64, 128}; tmK / tmV: [rows, d] box {64, kChunkTileN}; 128-byte swizzle.
 // Grid = num_groups * m_tiles CTAs, the row tile varying fastest so that the CTAs that walk the

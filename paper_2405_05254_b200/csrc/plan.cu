@@ -7,7 +7,7 @@ namespace yoco {
 
 int32_t validate_shape(const yoco_xattn_shape& s, int32_t mode) {
     if (s.B < 0 || s.Hq <= 0 || s.Hkv <= 0 || s.T <= 0 || s.d <= 0 || s.max_kv_len < 0 ||
-        s.kv_head_stride < 0 || s.reserved != 0 || !(s.scale >= 0.f))
+        s.kv_head_stride < 0 || s.window < 0 || !(s.scale >= 0.f))
         return YOCO_ERR_INVALID_ARG;
     if (mode != YOCO_MODE_DECODE && mode != YOCO_MODE_CHUNK) return YOCO_ERR_INVALID_ARG;
     if (s.d != 64 && s.d != 128) return YOCO_ERR_UNSUPPORTED;
@@ -52,8 +52,17 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     }
     if (extent >= (1ll << 31)) return YOCO_ERR_UNSUPPORTED;
 
+    // With a sliding window the lowest key any row of the call sees is that of row 0:
+    // (N - T) - C + 1.  Whole tiles below it are left out of the plan.
+    std::vector<int64_t> tile_lo(s.B, 0);
     int64_t total_tiles = 0;
-    for (int i = 0; i < s.B; ++i) total_tiles += (int64_t)s.Hkv * ((len[i] + tile_n - 1) / tile_n);
+    for (int i = 0; i < s.B; ++i) {
+        if (s.window > 0) {
+            const int64_t lo = (int64_t)len[i] - s.T - s.window + 1;
+            tile_lo[i] = std::min<int64_t>(std::max<int64_t>(lo, 0) / tile_n, (len[i] + tile_n - 1) / tile_n);
+        }
+        total_tiles += (int64_t)s.Hkv * ((len[i] + tile_n - 1) / tile_n - tile_lo[i]);
+    }
 
     // number of CTA groups
     int64_t target;
@@ -80,10 +89,11 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
         for (int c = 0; c < s.Hkv; ++c) {
             const int stream = b * s.Hkv + c;
             stream_base[stream] = (int32_t)dev.size();
-            int64_t t = 0;  // tile inside the stream
+            const int64_t t0 = tile_lo[b];
+            int64_t t = t0;  // tile inside the stream
             while (t < nt) {
-                while (group_lo(g + 1) <= flat + t) ++g;     // group owning flat tile flat+t
-                const int64_t t_end = std::min<int64_t>(nt, group_lo(g + 1) - flat);
+                while (group_lo(g + 1) <= flat + (t - t0)) ++g;     // group owning this flat tile
+                const int64_t t_end = std::min<int64_t>(nt, group_lo(g + 1) - flat + t0);
                 DevSegment d{};
                 d.k_begin = (int32_t)(t * tile_n);
                 d.k_end = (int32_t)std::min<int64_t>(t_end * tile_n, len[b]);
@@ -98,7 +108,7 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
                 ++stream_nseg[stream];
                 t = t_end;
             }
-            flat += nt;
+            flat += nt - t0;
         }
     }
     int32_t max_splits = 0, needs_combine = 0;

@@ -47,7 +47,7 @@ def assert_lse_close(got, ref, what=""):
 class GpuRunner:
     """Holds device copies of K/V and runs decode / chunk calls through the binding."""
 
-    def __init__(self, B, Hq, Hkv, d, T, kv_len, K_bits, V_bits, cu=None, kv_head_stride=0, scale=0.0):
+    def __init__(self, B, Hq, Hkv, d, T, kv_len, K_bits, V_bits, cu=None, kv_head_stride=0, scale=0.0, window=0):
         import torch
         from paper_2405_05254_b200 import binding
         self.torch, self.bd = torch, binding
@@ -55,7 +55,7 @@ class GpuRunner:
         self.kv_len = np.asarray(kv_len, dtype=np.int32)
         self.cu = None if cu is None else np.asarray(cu, dtype=np.int32)
         self.shape = binding.make_shape(B, Hq, Hkv, d, T, scale=scale, kv_head_stride=kv_head_stride,
-                                        max_kv_len=int(self.kv_len.max()) if B else 0)
+                                        max_kv_len=int(self.kv_len.max()) if B else 0, window=window)
         self.K = to_dev_bf16(K_bits.reshape(-1))
         self.V = to_dev_bf16(V_bits.reshape(-1))
 

@@ -162,3 +162,46 @@ def test_null_and_misaligned_pointers_fail_before_any_cuda_call():
     assert L.yoco_xattn_combine(4, 0, 128, None, None, None, None, None) == bd.ERR_INVALID_ARG
     assert L.yoco_xattn_combine(4, 2, 100, p(4096), p(4096), p(4096), None, None) == bd.ERR_UNSUPPORTED
     assert L.yoco_xattn_combine(4, 2, 128, None, p(4096), p(4096), None, None) == bd.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("case", [
+    dict(B=1, Hq=32, Hkv=8, d=128, T=1, lens=[32768], C=1024),
+    dict(B=3, Hq=8, Hkv=2, d=128, T=1, lens=[100, 5000, 63], C=130),
+    dict(B=2, Hq=8, Hkv=2, d=128, T=40, lens=[4000, 41], C=300),
+    dict(B=1, Hq=8, Hkv=2, d=128, T=4, lens=[1000], C=1),
+    dict(B=1, Hq=8, Hkv=2, d=128, T=1, lens=[1000], C=5000),
+])
+def test_sliding_window_plan_skips_only_tiles_no_row_can_see(case):
+    """With a window C the lowest key any row sees is that of row 0, (N - T) - C + 1; the plan
+    starts at the tile that holds it and still partitions the rest exactly."""
+    G, T, C = case["Hq"] // case["Hkv"], case["T"], case["C"]
+    modes = [bd.MODE_CHUNK] + ([bd.MODE_DECODE] if G * T <= 16 else [])
+    for mode in modes:
+        shape = bd.make_shape(case["B"], case["Hq"], case["Hkv"], case["d"], T, window=C)
+        info, segs = bd.yoco_xattn_plan(shape, case["lens"], 148, mode)
+        want_total = 0
+        for b, n in enumerate(case["lens"]):
+            first_key = max(0, (n - T) - C + 1)
+            start = min(first_key // info.tile_n, -(-n // info.tile_n)) * info.tile_n
+            want_total += case["Hkv"] * (-(-n // info.tile_n) - start // info.tile_n)
+            for c in range(case["Hkv"]):
+                mine = [s for s in segs if s.b == b and s.c == c]
+                pos = start
+                for s in mine:
+                    assert s.k_begin == pos and s.k_end > s.k_begin
+                    pos = s.k_end
+                assert pos == (n if mine else start) and (mine or start >= n or n == 0)
+                assert start <= first_key < start + info.tile_n or n - T - C + 1 <= 0
+        assert info.total_tiles == want_total
+        tiles = {}
+        for s in segs:
+            tiles[s.group] = tiles.get(s.group, 0) + -(-(s.k_end - s.k_begin) // info.tile_n)
+        if tiles:
+            assert max(tiles.values()) - min(tiles.values()) <= 1
+
+
+def test_negative_window_is_rejected():
+    shape = bd.make_shape(1, 8, 8, 128, 1, window=-1)
+    with pytest.raises(bd.YocoError) as e:
+        bd.yoco_xattn_plan(shape, [100], 148, bd.MODE_DECODE)
+    assert e.value.code == bd.ERR_INVALID_ARG
