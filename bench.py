@@ -215,6 +215,42 @@ def measure_chunk(dev, peaks, name="chunk"):
             "kv_bytes": w.kv_bytes}
 
 
+def measure_window(dev, peak_gbs, name="swa"):
+    """Batched decode under the sliding-window mask: 128 sequences, window 1,024.  Only the keys
+    inside a window are planned and read, so the algorithmic bytes are those of the windows."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    w = si.workload(name)
+    to_dev = lambda a: torch.from_numpy(a.reshape(-1).view(np.int16)).to(dev).view(torch.bfloat16)  # noqa: E731
+    K, V, Q = to_dev(w.make_k()), to_dev(w.make_v()), to_dev(w.make_q(0))
+    shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(w.kv_len.max()), window=w.window)
+    ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_DECODE), dtype=torch.uint8, device=dev)
+    O = torch.empty(w.B * w.Hq * w.T * w.d, dtype=torch.bfloat16, device=dev)
+    for _ in range(3):
+        bd.yoco_xattn_decode(shape, Q, K, V, w.cu, w.kv_len, O, None, ws)
+    assert bd.yoco_xattn_status(ws) == 0
+    n = 20
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        bd.yoco_xattn_decode(shape, Q, K, V, w.cu, w.kv_len, O, None, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    call_us = e0.elapsed_time(e1) * 1e3 / n
+    bd.yoco_xattn_profile_enable(n)
+    for _ in range(n):
+        bd.yoco_xattn_decode(shape, Q, K, V, w.cu, w.kv_len, O, None, ws)
+    k_us = float(bd.yoco_xattn_profile_collect(n).mean()) * 1e3
+    bd.yoco_xattn_profile_enable(0)
+    window_bytes = int(sum(min(int(nk), w.window) for nk in w.kv_len)) * 2 * w.Hkv * w.d * 2
+    achieved = window_bytes / (k_us * 1e-6) / 1e9
+    return {"workload": f"{w.name}: B={w.B} Hq={w.Hq} Hkv={w.Hkv} d={w.d} T=1 kv_len in [2048,4096] window={w.window}",
+            "algorithmic_bytes_per_launch": window_bytes, "kernel_us": k_us, "call_us": call_us,
+            "us_per_token_layer": call_us / w.B, "bound": "hbm", "achieved": achieved, "unit": "GB/s",
+            "peak": peak_gbs, "frac": achieved / peak_gbs,
+            "l2": "the windows of one call total more than L2 (K+V of the windows > 126 MB)"}
+
+
 def run_ours(args):
     import torch
     from paper_2405_05254_b200 import binding as bd
@@ -367,6 +403,8 @@ def run_ours(args):
             del K, V
             torch.cuda.empty_cache()
             line["chunk"] = measure_chunk(dev, peaks, args.chunk_workload)
+        if world == 1 and not args.no_window:
+            line["sliding_window"] = measure_window(dev, peak)
         if world == 1 and not args.no_cpu_baseline:
             gbs, dt, sample, cores = oracle_sample_rate(w, Qh, Kh, Vh)
             line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
@@ -386,6 +424,7 @@ def main():
     ap.add_argument("--workload", default="1m", choices=["1m", "128k", "3b_32k", "ragged", "tiny"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-chunk", action="store_true", help="skip the extra measurement of the chunk path")
+    ap.add_argument("--no-window", action="store_true", help="skip the sliding-window decode measurement")
     ap.add_argument("--only-chunk", action="store_true", help="measure the chunk path alone")
     ap.add_argument("--chunk-workload", default="chunk", choices=["chunk", "chunk_32k"])
     args = ap.parse_args()

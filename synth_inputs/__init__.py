@@ -86,6 +86,7 @@ class Workload:
     seed: int
     kv_len: np.ndarray          # [B] int32, includes the T new positions
     k_mult: float = 1.0
+    window: int = 0             # sliding window C (0 = plain causal)
     cu: np.ndarray = field(init=False)
 
     def __post_init__(self):
@@ -142,6 +143,9 @@ def workload(name: str) -> Workload:
     if name == "chunk_32k":     # config 5 with a 32K cache (profiler captures)
         return Workload(name, B=2, Hq=32, Hkv=8, d=128, T=512, layers=1, seed=4,
                         kv_len=[32768 + 512] * 2)
+    if name == "swa":           # batched decode under the paper's window of 1,024 (Section 4.1)
+        return Workload(name, B=128, Hq=32, Hkv=8, d=128, T=1, layers=1, seed=6,
+                        kv_len=ragged_lengths(6, 128, 2048, 2049), window=1024)
     if name == "ragged_small":  # same recipe as config 3, 32x shorter
         return Workload(name, B=16, Hq=32, Hkv=8, d=128, T=1, layers=1, seed=2,
                         kv_len=ragged_lengths(2, 16, 128, 3969))
