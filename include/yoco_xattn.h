@@ -180,6 +180,28 @@ int32_t yoco_xattn_chunk(const yoco_xattn_shape* shape, const void* Q, const voi
 int32_t yoco_xattn_combine(int64_t rows, int32_t S, int32_t d, const float* part_o,
                            const float* part_lse, void* O, float* lse, void* stream);
 
+/* The same merge for pieces laid out piece-major: part_o [S, rows, d], part_lse [S, rows] -- what
+ * an all-gather over S ranks leaves when every rank contributes its [rows, d] partial result and
+ * its [rows] log-sum-exp.  Otherwise as yoco_xattn_combine. */
+int32_t yoco_xattn_combine_gathered(int64_t rows, int32_t S, int32_t d, const float* part_o,
+                                    const float* part_lse, void* O, float* lse, void* stream);
+
+/* Decode over ONE SHARD of the keys, for key-range sharding of a long cache across GPUs (the
+ * K^, V^ of Section 2.2 split along the sequence, as sequence-parallel prefill leaves them).
+ * K, V, cu_kv_host, kv_len_host describe the keys this GPU holds (an ordinary packed cache,
+ * kv_len[i] may be 0); the result is the attention over those keys only:
+ *   part_o   [B*Hq, d] fp32, normalised over the shard's keys (0 where the shard is empty)
+ *   part_lse [B*Hq]    fp32, natural-log sum of exp(score) over the shard's keys (-inf if empty)
+ * Exchanging (part_o, part_lse) between the shards and merging them with
+ * yoco_xattn_combine_gathered gives exactly softmax(QK^T)V over the whole cache (the log-sum-exp
+ * merge is algebraically exact).  Requires T = 1 and no window: with one query row per head every
+ * key of a shard is visible whichever shard holds the row's own position.  Workspace as for
+ * yoco_xattn_decode.  All pointers device unless marked host. */
+int32_t yoco_xattn_decode_partial(const yoco_xattn_shape* shape, const void* Q, const void* K,
+                                  const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
+                                  float* part_o, float* part_lse, void* workspace,
+                                  size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, reads the status word that the last decode/chunk call
  * using `workspace` left, returns it (YOCO_OK or YOCO_ERR_TIMEOUT). */
 int32_t yoco_xattn_status(const void* workspace, void* stream);

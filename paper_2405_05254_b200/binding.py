@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.yoco_xattn_decode_static.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp]
         L.yoco_xattn_static_scratch_bytes.argtypes = []
         L.yoco_xattn_combine.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
+        L.yoco_xattn_combine_gathered.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
+        L.yoco_xattn_decode_partial.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.yoco_xattn_status.argtypes = [vp, vp]
         L.yoco_xattn_profile_enable.argtypes = [i32]
         L.yoco_xattn_profile_collect.argtypes = [vp, i32, vp]
@@ -73,7 +75,8 @@ def lib() -> ctypes.CDLL:
         L.yoco_xattn_strerror.restype = ctypes.c_char_p
         L.yoco_xattn_last_cuda_error.argtypes = []
         for name in ("plan", "workspace_size", "decode", "chunk", "combine", "status", "last_cuda_error",
-                     "profile_enable", "profile_collect", "decode_static", "static_scratch_bytes"):
+                     "profile_enable", "profile_collect", "decode_static", "static_scratch_bytes",
+                     "combine_gathered", "decode_partial"):
             getattr(L, "yoco_xattn_" + name).restype = i32
         _lib = L
     return _lib
@@ -152,6 +155,27 @@ def yoco_xattn_combine(part_o, part_lse, O, lse=None, stream=None) -> None:
                                   _stream_ptr(stream))
     if rc != OK:
         raise YocoError(rc, "yoco_xattn_combine")
+
+
+def yoco_xattn_combine_gathered(part_o, part_lse, O, lse=None, stream=None) -> None:
+    """Merge piece-major partials: part_o [S,rows,d] fp32, part_lse [S,rows] fp32 -> O [rows,d] bf16."""
+    S, rows, d = part_o.shape
+    rc = lib().yoco_xattn_combine_gathered(rows, S, d, _ptr(part_o), _ptr(part_lse), _ptr(O), _ptr(lse),
+                                           _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_combine_gathered")
+
+
+def yoco_xattn_decode_partial(shape: Shape, Q, K, V, cu_kv, kv_len, part_o, part_lse, workspace,
+                              stream=None) -> None:
+    """Decode over the key shard this GPU holds: fp32 partial rows + their log-sum-exp (T = 1)."""
+    keep_cu, p_cu = _host_i32(cu_kv)
+    keep_len, p_len = _host_i32(kv_len)
+    rc = lib().yoco_xattn_decode_partial(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), p_cu, p_len,
+                                         _ptr(part_o), _ptr(part_lse), _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_decode_partial")
 
 
 def yoco_xattn_status(workspace, stream=None) -> int:

@@ -187,12 +187,14 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 
 int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const void* K, const void* V,
             const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
-            void* workspace, size_t workspace_bytes, void* stream_v) {
+            void* workspace, size_t workspace_bytes, void* stream_v, float* part_out = nullptr) {
+    // part_out != null: the result is a partial one (fp32 rows + their LSE in `lse`, no bf16 O)
     if (!shape) return YOCO_ERR_INVALID_ARG;
     int32_t rc = validate_shape(*shape, mode);
     if (rc != YOCO_OK) return rc;
     if (shape->B == 0) return YOCO_OK;
-    if (!Q || !K || !V || !O || !workspace) return YOCO_ERR_INVALID_ARG;
+    if (!Q || !K || !V || !(O || part_out) || !workspace) return YOCO_ERR_INVALID_ARG;
+    if (part_out && (!lse || !aligned(part_out, 16))) return YOCO_ERR_INVALID_ARG;
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) ||
         !aligned(workspace, 256) || (lse && !aligned(lse, 4)))
         return YOCO_ERR_INVALID_ARG;
@@ -247,6 +249,7 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             p.rows_per_stream = plan.rows_per_stream;
             p.d = shape->d;
             p.window = shape->window;
+            p.force_partial = part_out ? 1 : 0;
             YOCO_CUDA_TRY(launch_decode(p, tmK, tmV, plan.info.num_groups, stream,
                                         inline_tables ? &ready->decode_tab : nullptr));
         } else {
@@ -279,7 +282,7 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             if (prof) YOCO_CUDA_TRY(cudaEventRecord(ev, stream));
         }
     }
-    if (plan.info.needs_combine) {
+    if (plan.info.needs_combine || part_out) {
         CombineParams c{};
         c.rows = (int64_t)shape->B * shape->Hq * shape->T;
         c.d = shape->d;
@@ -293,8 +296,10 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
         c.stream_nseg = table + plan.off_stream_nseg;
         c.part_o = part_o;
         c.part_lse = part_lse;
-        c.O = static_cast<__nv_bfloat16*>(O);
+        c.O = part_out ? nullptr : static_cast<__nv_bfloat16*>(O);
         c.lse = lse;
+        c.O_f32 = part_out;
+        c.merge_unsplit = part_out ? 1 : 0;
         // directly behind the attention kernel (no event in between): its launch may overlap
         // that kernel's tail
         const bool chained = plan.info.num_segments > 0 && g_prof.events.empty();
@@ -399,14 +404,14 @@ int32_t yoco_xattn_chunk(const yoco_xattn_shape* shape, const void* Q, const voi
                workspace_bytes, stream);
 }
 
-int32_t yoco_xattn_combine(int64_t rows, int32_t S, int32_t d, const float* part_o,
-                           const float* part_lse, void* O, float* lse, void* stream) {
+namespace {
+int32_t combine_public(int64_t rows, int32_t S, int32_t d, const float* part_o, const float* part_lse, void* O,
+                       float* lse, void* stream, int32_t piece_major) {
     if (rows < 0 || S <= 0 || d <= 0) return YOCO_ERR_INVALID_ARG;
     if (d % 8 != 0 || d > 256) return YOCO_ERR_UNSUPPORTED;
     if (rows == 0) return YOCO_OK;
     if (!part_o || !part_lse || !O) return YOCO_ERR_INVALID_ARG;
     if (!aligned(part_o, 16) || !aligned(part_lse, 4) || !aligned(O, 16)) return YOCO_ERR_INVALID_ARG;
-    if (d % 4 != 0) return YOCO_ERR_UNSUPPORTED;
     CombineParams c{};
     c.rows = rows;
     c.d = d;
@@ -418,8 +423,31 @@ int32_t yoco_xattn_combine(int64_t rows, int32_t S, int32_t d, const float* part
     c.part_lse = part_lse;
     c.O = static_cast<__nv_bfloat16*>(O);
     c.lse = lse;
+    c.piece_major = piece_major;
     YOCO_CUDA_TRY(launch_combine(c, reinterpret_cast<cudaStream_t>(stream)));
     return YOCO_OK;
+}
+}  // namespace
+
+int32_t yoco_xattn_combine(int64_t rows, int32_t S, int32_t d, const float* part_o,
+                           const float* part_lse, void* O, float* lse, void* stream) {
+    return combine_public(rows, S, d, part_o, part_lse, O, lse, stream, 0);
+}
+
+int32_t yoco_xattn_combine_gathered(int64_t rows, int32_t S, int32_t d, const float* part_o,
+                                    const float* part_lse, void* O, float* lse, void* stream) {
+    return combine_public(rows, S, d, part_o, part_lse, O, lse, stream, 1);
+}
+
+int32_t yoco_xattn_decode_partial(const yoco_xattn_shape* shape, const void* Q, const void* K, const void* V,
+                                  const int32_t* cu_kv_host, const int32_t* kv_len_host, float* part_o,
+                                  float* part_lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!shape || !part_o || !part_lse) return YOCO_ERR_INVALID_ARG;
+    // one query row per head: then every key of a shard is visible whatever follows it on other
+    // shards, and a shard is an ordinary (shorter) cache; a window would need global positions
+    if (shape->T != 1 || shape->window != 0) return YOCO_ERR_UNSUPPORTED;
+    return run(shape, YOCO_MODE_DECODE, Q, K, V, cu_kv_host, kv_len_host, nullptr, part_lse, workspace,
+               workspace_bytes, stream, part_o);
 }
 
 int32_t yoco_xattn_status(const void* workspace, void* stream) {

@@ -38,18 +38,25 @@ __device__ __forceinline__ void combine_body(const CombineParams& p) {
         const int r_local = (h % G) * p.T + t;
         const int slot0 = p.stream_base[stream];
         nseg = p.stream_nseg[stream];
-        if (nseg == 1) return;   // an unsplit stream: the attention kernel wrote the final rows itself
+        // an unsplit stream: the attention kernel wrote the final rows itself (unless told not to)
+        if (nseg == 1 && !p.merge_unsplit) return;
         o_base = ((int64_t)slot0 * p.rows_per_stream + r_local) * p.d;
         o_stride = (int64_t)p.rows_per_stream * p.d;
         lse_base = (int64_t)slot0 * p.rows_per_stream + r_local;
         lse_stride = p.rows_per_stream;
     } else {
-        // public layout: [rows][S][d]
         nseg = p.S;
-        o_base = row * p.S * p.d;
-        o_stride = p.d;
-        lse_base = row * p.S;
-        lse_stride = 1;
+        if (p.piece_major) {     // [S][rows][d]
+            o_base = row * p.d;
+            o_stride = p.rows * p.d;
+            lse_base = row;
+            lse_stride = p.rows;
+        } else {                 // [rows][S][d]
+            o_base = row * p.S * p.d;
+            o_stride = p.d;
+            lse_base = row * p.S;
+            lse_stride = 1;
+        }
     }
 
     float m = -INFINITY;
@@ -57,10 +64,14 @@ __device__ __forceinline__ void combine_body(const CombineParams& p) {
 #pragma unroll
     for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
 
-    __nv_bfloat16* out = p.O + row * p.d;
+    __nv_bfloat16* out = p.O ? p.O + row * p.d : nullptr;
+    float* out32 = p.O_f32 ? p.O_f32 + row * p.d : nullptr;
     if (m == -INFINITY) {   // no piece carries weight (also nseg == 0); the same for every warp of the row
         if (sub == 0) {
-            for (int e = lane; e < p.d; e += 32) out[e] = __float2bfloat16(0.f);
+            for (int e = lane; e < p.d; e += 32) {
+                if (out32) out32[e] = 0.f;
+                else out[e] = __float2bfloat16(0.f);
+            }
             if (p.lse && lane == 0) p.lse[row] = -INFINITY;
         }
         return;
@@ -113,7 +124,9 @@ __device__ __forceinline__ void combine_body(const CombineParams& p) {
     }
 #pragma unroll
     for (int blk = 0; blk < 2; ++blk) {
-        if (e0 + blk * 128 < p.d) {
+        if (e0 + blk * 128 < p.d && out32) {
+            *reinterpret_cast<float4*>(out32 + e0 + blk * 128) = acc[blk];
+        } else if (e0 + blk * 128 < p.d) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(acc[blk].x, acc[blk].y), hi = __floats2bfloat162_rn(acc[blk].z, acc[blk].w);
             uint2 pk;
             pk.x = *reinterpret_cast<uint32_t*>(&lo);

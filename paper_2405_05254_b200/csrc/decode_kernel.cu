@@ -297,7 +297,7 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
             }
         }
         named_barrier_sync(1, kConsumerWarps * 32);
-        const bool final_out = seg.stream_nseg == 1;
+        const bool final_out = seg.stream_nseg == 1 && !p.force_partial;
         for (int idx = threadIdx.x; idx < n_rows * D; idx += kConsumerWarps * 32) {
             const int r = idx / D, col = idx - r * D;
             float M = -INFINITY;

@@ -40,8 +40,14 @@ struct CombineParams {
     const int32_t* stream_nseg; // [B*Hkv] slots of each stream
     const float* part_o;
     const float* part_lse;      // natural log, -inf = empty
-    __nv_bfloat16* O;
+    __nv_bfloat16* O;           // [rows, d] bf16 result, or null when O_f32 is given
     float* lse;                 // may be null
+    float* O_f32;               // [rows, d] fp32 result instead of O (a partial result that another
+                                // merge will consume: key-range sharding across GPUs)
+    int32_t merge_unsplit;      // internal layout: also copy rows whose stream has a single piece
+                                // (set when the attention kernel was told to write no final rows)
+    int32_t piece_major;        // public layout is [S][rows][d] / [S][rows] (as an all-gather over S
+                                // ranks leaves it) instead of [rows][S][d] / [rows][S]
 };
 // inline_tab (host, may be null): stream tables passed as kernel parameters instead of
 // p.stream_base / p.stream_nseg.  after_attention: launched right behind the attention kernel of
@@ -64,6 +70,7 @@ struct DecodeParams {
     int32_t rows_per_stream;    // G * T (<= 16)
     int32_t d;
     int32_t window;             // sliding window C, 0 = none
+    int32_t force_partial;      // write every segment to its partial slot, even of an unsplit stream
 };
 // tmK / tmV: 2-D tensor maps over the [rows, d] view of K and V, box {64, kDecodeTileN},
 // 128-byte swizzle.
