@@ -251,6 +251,51 @@ def measure_window(dev, peak_gbs, name="swa"):
             "l2": "the windows of one call total more than L2 (K+V of the windows > 126 MB)"}
 
 
+def measure_key_range_shard(dev, w, K, V, Q, shards=8):
+    """What one GPU of an S-way key-range-sharded cache does per layer call, measured on this GPU:
+    the partial decode over 1/S of the keys (a view of the resident cache: pointer offset plus head
+    stride, no copy) and the merge of S gathered partials.  The exchange itself (an all-gather of
+    rows x (d + 1) fp32 per rank) needs S GPUs and is not part of this number."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd, shard
+    N = int(w.kv_len[0])
+    off, cnt = shard.key_range_shards([N], shards)
+    n_local = int(cnt[0, 0])
+    rows = w.B * w.Hq
+    shape = bd.make_shape(1, w.Hq, w.Hkv, w.d, 1, kv_head_stride=N * w.d, max_kv_len=n_local)
+    lens = np.array([n_local], dtype=np.int32)
+    cu = np.array([0, N], dtype=np.int32)
+    ws = torch.empty(bd.yoco_xattn_workspace_size(shape, lens, bd.MODE_DECODE), dtype=torch.uint8, device=dev)
+    all_o = torch.zeros((shards, rows, w.d), dtype=torch.float32, device=dev)
+    all_l = torch.zeros((shards, rows), dtype=torch.float32, device=dev)
+    O = torch.empty(rows * w.d, dtype=torch.bfloat16, device=dev)
+
+    def partial(r):
+        o = int(off[r, 0]) * w.d
+        bd.yoco_xattn_decode_partial(shape, Q, K[o:], V[o:], cu, lens, all_o[r], all_l[r], ws)
+
+    for r in range(shards):           # fills every slot once, so that the merge below has real inputs
+        partial(r if int(cnt[r, 0]) == n_local else 0)
+    assert bd.yoco_xattn_status(ws) == 0
+    n = 30
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    ev[0].record()
+    for k in range(n):
+        partial(k % (shards - 1) if shards > 1 else 0)
+    ev[1].record()
+    for _ in range(n):
+        bd.yoco_xattn_combine_gathered(all_o, all_l, O, None)
+    ev[2].record()
+    torch.cuda.synchronize()
+    part_us, merge_us = ev[0].elapsed_time(ev[1]) * 1e3 / n, ev[1].elapsed_time(ev[2]) * 1e3 / n
+    shard_bytes = 2 * w.Hkv * n_local * w.d * 2
+    return {"shards": shards, "keys_per_shard": n_local, "partial_call_us": part_us, "merge_us": merge_us,
+            "shard_kv_bytes": shard_bytes, "partial_call_gbs": shard_bytes / part_us / 1e3,
+            "exchange_bytes_per_rank": rows * (w.d + 1) * 4,
+            "note": "one GPU's share of an S-way key-range-sharded layer call; the all-gather of the partials "
+                    "needs S GPUs and is not included"}
+
+
 def run_ours(args):
     import torch
     from paper_2405_05254_b200 import binding as bd
@@ -399,6 +444,8 @@ def run_ours(args):
                                        "every attention kernel",
                          "traffic": traffic},
         }
+        if world == 1 and w.B == 1 and w.T == 1 and not args.no_shard:
+            line["key_range_shard"] = measure_key_range_shard(dev, w, K, V, Qd[0])
         if world == 1 and not args.no_chunk:
             del K, V
             torch.cuda.empty_cache()
@@ -424,6 +471,7 @@ def main():
     ap.add_argument("--workload", default="1m", choices=["1m", "128k", "3b_32k", "ragged", "tiny"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-chunk", action="store_true", help="skip the extra measurement of the chunk path")
+    ap.add_argument("--no-shard", action="store_true", help="skip the key-range-shard measurement")
     ap.add_argument("--no-window", action="store_true", help="skip the sliding-window decode measurement")
     ap.add_argument("--only-chunk", action="store_true", help="measure the chunk path alone")
     ap.add_argument("--chunk-workload", default="chunk", choices=["chunk", "chunk_32k"])
