@@ -202,6 +202,42 @@ int32_t yoco_xattn_decode_partial(const yoco_xattn_shape* shape, const void* Q, 
                                   float* part_o, float* part_lse, void* workspace,
                                   size_t workspace_bytes, void* stream);
 
+/* ---- Writing the cache (Section 2.2, first cross-decoder equation) -------------------------
+ *   K^ = LN(X) W_K,  V^ = LN(X) W_V,  LN = RMSNorm (Section 2.1), no bias:
+ *   LN(x) = x * g / sqrt(mean_k(x_k^2) + eps)
+ * X holds the self-decoder's output for the T new tokens of every sequence; the rows produced are
+ * stored at positions [N_i - T, N_i) of the packed head-major caches described above, where the
+ * attention calls of the cross-decoder layers then find them (kv_len counts them already). */
+typedef struct yoco_kv_append_shape {
+    int32_t B;               /* sequences (<= 512)                                        */
+    int32_t Hkv;             /* KV heads; Hkv * d must be a multiple of 128               */
+    int32_t d;               /* head dimension: 64 or 128                                 */
+    int32_t T;               /* new tokens per sequence                                   */
+    int32_t d_model;         /* width of X; multiple of 128                               */
+    float   eps;             /* >= 0, used as given (the paper prints none; 1e-6 is usual) */
+    int64_t kv_head_stride;  /* as in yoco_xattn_shape                                    */
+} yoco_kv_append_shape;
+
+/* Folds the RMSNorm gain into a projection weight once per model (weights do not change between
+ * calls):  Wg[k, n] = g[k] * W[k, n], one rounding to bf16.  g [d_model], W and Wg [d_model, n_out]
+ * row-major bf16, all device; Wg may not alias W. */
+int32_t yoco_kv_fold_gain(int64_t d_model, int64_t n_out, const void* g, const void* W, void* Wg,
+                          void* stream);
+
+/* Computes the new cache rows and stores them.  X [B*T, d_model] bf16 (sequence-major, the T
+ * tokens of a sequence consecutive); Wgk, Wgv [d_model, Hkv*d] bf16 = gain-folded W_K, W_V (see
+ * yoco_kv_fold_gain); K, V: the packed caches (device, written in place, 16-byte aligned);
+ * cu_kv_host [B+1] or NULL (tight packing), kv_len_host [B]: host, N_i >= T including the new
+ * tokens.  Rows outside [N_i - T, N_i) are not touched.  Uses no workspace and only enqueues work.
+ * A bounded device-side wait that ran out is reported by yoco_kv_append_status. */
+int32_t yoco_kv_append(const yoco_kv_append_shape* shape, const void* X, const void* Wgk, const void* Wgv,
+                       void* K, void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
+                       void* stream);
+
+/* Synchronises `stream`; returns YOCO_OK or YOCO_ERR_TIMEOUT if an append kernel on the current
+ * device gave up a wait since the last call of this function (which clears the record). */
+int32_t yoco_kv_append_status(void* stream);
+
 /* Synchronises `stream`, reads the status word that the last decode/chunk call
  * using `workspace` left, returns it (YOCO_OK or YOCO_ERR_TIMEOUT). */
 int32_t yoco_xattn_status(const void* workspace, void* stream);

@@ -26,6 +26,11 @@ class Shape(ctypes.Structure):
                 ("window", ctypes.c_int32)]
 
 
+class KvAppendShape(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("d", ctypes.c_int32), ("T", ctypes.c_int32),
+                ("d_model", ctypes.c_int32), ("eps", ctypes.c_float), ("kv_head_stride", ctypes.c_int64)]
+
+
 class Segment(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("group", "b", "c", "k_begin", "k_end", "slot")]
 
@@ -68,6 +73,11 @@ def lib() -> ctypes.CDLL:
         L.yoco_xattn_combine.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
         L.yoco_xattn_combine_gathered.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
         L.yoco_xattn_decode_partial.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.yoco_kv_fold_gain.argtypes = [i64, i64, vp, vp, vp, vp]
+        L.yoco_kv_append.argtypes = [ctypes.POINTER(KvAppendShape), vp, vp, vp, vp, vp, vp, vp, vp]
+        L.yoco_kv_append_status.argtypes = [vp]
+        for name in ("yoco_kv_fold_gain", "yoco_kv_append", "yoco_kv_append_status"):
+            getattr(L, name).restype = i32
         L.yoco_xattn_status.argtypes = [vp, vp]
         L.yoco_xattn_profile_enable.argtypes = [i32]
         L.yoco_xattn_profile_collect.argtypes = [vp, i32, vp]
@@ -176,6 +186,30 @@ def yoco_xattn_decode_partial(shape: Shape, Q, K, V, cu_kv, kv_len, part_o, part
                                          workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     if rc != OK:
         raise YocoError(rc, "yoco_xattn_decode_partial")
+
+
+def yoco_kv_fold_gain(g, W, Wg, stream=None) -> None:
+    """Wg = g[:, None] * W rounded to bf16 (W, Wg: [d_model, n_out] bf16 device tensors)."""
+    d_model, n_out = W.shape
+    rc = lib().yoco_kv_fold_gain(d_model, n_out, _ptr(g), _ptr(W), _ptr(Wg), _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_kv_fold_gain")
+
+
+def yoco_kv_append(shape: KvAppendShape, X, Wgk, Wgv, K, V, cu_kv, kv_len, stream=None) -> None:
+    """Enqueue K^ = RMSNorm(X) W_K, V^ = RMSNorm(X) W_V and store the rows at the last T positions
+    of every sequence in the packed caches K, V (in place)."""
+    keep_cu, p_cu = _host_i32(cu_kv)
+    keep_len, p_len = _host_i32(kv_len)
+    rc = lib().yoco_kv_append(ctypes.byref(shape), _ptr(X), _ptr(Wgk), _ptr(Wgv), _ptr(K), _ptr(V), p_cu, p_len,
+                              _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_kv_append")
+
+
+def yoco_kv_append_status(stream=None) -> int:
+    """Synchronise the stream; 0 unless an append kernel gave up a bounded wait since the last call."""
+    return int(lib().yoco_kv_append_status(_stream_ptr(stream)))
 
 
 def yoco_xattn_status(workspace, stream=None) -> int:

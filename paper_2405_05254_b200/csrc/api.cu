@@ -50,6 +50,7 @@ int32_t device_state(DeviceState** out) {
         YOCO_CUDA_TRY(decode_kernel_setup());
         YOCO_CUDA_TRY(chunk_kernel_setup());
         YOCO_CUDA_TRY(chunk_pair_kernel_setup());
+        YOCO_CUDA_TRY(kv_append_kernel_setup());
         st.ready = true;
     }
     *out = &st;
@@ -448,6 +449,74 @@ int32_t yoco_xattn_decode_partial(const yoco_xattn_shape* shape, const void* Q, 
     if (shape->T != 1 || shape->window != 0) return YOCO_ERR_UNSUPPORTED;
     return run(shape, YOCO_MODE_DECODE, Q, K, V, cu_kv_host, kv_len_host, nullptr, part_lse, workspace,
                workspace_bytes, stream, part_o);
+}
+
+int32_t yoco_kv_fold_gain(int64_t d_model, int64_t n_out, const void* g, const void* W, void* Wg, void* stream) {
+    if (d_model < 0 || n_out < 0) return YOCO_ERR_INVALID_ARG;
+    if (d_model == 0 || n_out == 0) return YOCO_OK;
+    if (!g || !W || !Wg || W == Wg) return YOCO_ERR_INVALID_ARG;
+    YOCO_CUDA_TRY(launch_fold_gain(static_cast<const __nv_bfloat16*>(g), static_cast<const __nv_bfloat16*>(W),
+                                   static_cast<__nv_bfloat16*>(Wg), d_model, n_out,
+                                   reinterpret_cast<cudaStream_t>(stream)));
+    return YOCO_OK;
+}
+
+int32_t yoco_kv_append(const yoco_kv_append_shape* shape, const void* X, const void* Wgk, const void* Wgv,
+                       void* K, void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host, void* stream) {
+    if (!shape) return YOCO_ERR_INVALID_ARG;
+    const yoco_kv_append_shape& s = *shape;
+    if (s.B < 0 || s.Hkv <= 0 || s.d <= 0 || s.T <= 0 || s.d_model <= 0 || s.kv_head_stride < 0 || !(s.eps >= 0.f))
+        return YOCO_ERR_INVALID_ARG;
+    if ((s.d != 64 && s.d != 128) || s.d_model % 128 != 0 || (s.Hkv * s.d) % 128 != 0 ||
+        s.kv_head_stride % s.d != 0 || s.B > kAppendMaxSequences || (int64_t)s.B * s.T >= (1ll << 31))
+        return YOCO_ERR_UNSUPPORTED;
+    if (s.B == 0) return YOCO_OK;
+    if (!X || !Wgk || !Wgv || !K || !V || !kv_len_host) return YOCO_ERR_INVALID_ARG;
+    if (!aligned(X, 16) || !aligned(Wgk, 16) || !aligned(Wgv, 16) || !aligned(K, 16) || !aligned(V, 16))
+        return YOCO_ERR_INVALID_ARG;
+    DeviceState* dev = nullptr;
+    int32_t rc = device_state(&dev);
+    if (rc != YOCO_OK) return rc;
+
+    KvAppendTables tab;
+    std::memset(&tab, 0, sizeof tab);
+    int64_t tok = 0;
+    for (int i = 0; i < s.B; ++i) {
+        const int64_t n = kv_len_host[i];
+        if (n < s.T) return YOCO_ERR_INVALID_ARG;
+        const int64_t head_rows = s.kv_head_stride ? s.kv_head_stride / s.d : n;
+        if (head_rows < n) return YOCO_ERR_INVALID_ARG;
+        if (cu_kv_host) {
+            if (cu_kv_host[i] < 0 || cu_kv_host[i + 1] < cu_kv_host[i]) return YOCO_ERR_INVALID_ARG;
+            tok = cu_kv_host[i];
+        }
+        const int64_t row0 = tok * s.Hkv + (n - s.T);
+        if (row0 + (int64_t)(s.Hkv - 1) * head_rows + s.T >= (1ll << 31)) return YOCO_ERR_UNSUPPORTED;
+        tab.row0[i] = (int32_t)row0;
+        tab.head_rows[i] = (int32_t)head_rows;
+        if (!cu_kv_host) tok += head_rows;
+    }
+    KvAppendParams p{};
+    p.K = static_cast<__nv_bfloat16*>(K);
+    p.V = static_cast<__nv_bfloat16*>(V);
+    p.M = s.B * s.T;
+    p.T = s.T;
+    p.d = s.d;
+    p.d_model = s.d_model;
+    p.n_half = s.Hkv * s.d;
+    p.eps = s.eps;
+    CUtensorMap tmX, tmWk, tmWv;
+    if ((rc = make_map_2d(&tmX, X, p.M, s.d_model, 128)) != YOCO_OK) return rc;
+    if ((rc = make_map_2d(&tmWk, Wgk, s.d_model, p.n_half, 128)) != YOCO_OK) return rc;
+    if ((rc = make_map_2d(&tmWv, Wgv, s.d_model, p.n_half, 128)) != YOCO_OK) return rc;
+    YOCO_CUDA_TRY(launch_kv_append(p, tab, tmX, tmWk, tmWv, reinterpret_cast<cudaStream_t>(stream)));
+    return YOCO_OK;
+}
+
+int32_t yoco_kv_append_status(void* stream) {
+    int32_t word = 0;
+    YOCO_CUDA_TRY(read_and_clear_kv_append_status(&word, reinterpret_cast<cudaStream_t>(stream)));
+    return word == kStatusOk ? YOCO_OK : YOCO_ERR_TIMEOUT;
 }
 
 int32_t yoco_xattn_status(const void* workspace, void* stream) {

@@ -109,4 +109,27 @@ cudaError_t launch_chunk_pair(const ChunkParams& p, const CUtensorMap& tmQ, cons
                               const CUtensorMap& tmV, int num_groups, cudaStream_t stream);
 cudaError_t chunk_pair_kernel_setup();
 
+// ---- writing the cache: K^ = RMSNorm(X) W_K, V^ = RMSNorm(X) W_V appended head-major ------------
+constexpr int kAppendMaxSequences = 512;
+struct KvAppendParams {
+    __nv_bfloat16* K;           // packed head-major caches
+    __nv_bfloat16* V;
+    int32_t M;                  // B * T tokens
+    int32_t T, d, d_model;
+    int32_t n_half;             // Hkv * d: output columns of K^ (those of V^ follow)
+    float eps;
+};
+struct KvAppendTables {         // per sequence, as kernel parameters
+    int32_t row0[kAppendMaxSequences];       // cache row (units of d elements) of (head 0, key N_i - T)
+    int32_t head_rows[kAppendMaxSequences];  // rows between two heads of the sequence
+};
+// tmX: [M, d_model] box {64, 128}; tmWk / tmWv: gain-folded weights [d_model, Hkv*d] box {64, 128};
+// 128-byte swizzle.  Grid = (2*Hkv*d/128, ceil(M/128)).
+cudaError_t launch_kv_append(const KvAppendParams& p, const KvAppendTables& tab, const CUtensorMap& tmX,
+                             const CUtensorMap& tmWk, const CUtensorMap& tmWv, cudaStream_t stream);
+cudaError_t launch_fold_gain(const __nv_bfloat16* g, const __nv_bfloat16* W, __nv_bfloat16* Wg, int64_t d_model,
+                             int64_t n_out, cudaStream_t stream);
+cudaError_t read_and_clear_kv_append_status(int32_t* word, cudaStream_t stream);
+cudaError_t kv_append_kernel_setup();
+
 }  // namespace yoco

@@ -1,0 +1,240 @@
+// Writing the shared cache: K^ = RMSNorm(X) W_K, V^ = RMSNorm(X) W_V for the T new tokens of every
+// sequence, stored straight into the head-major cache rows [N_i - T, N_i) that the cross-decoder
+// attention reads.
+//
+// RMSNorm(x) = x * r * g with r = 1 / sqrt(mean(x^2) + eps).  The gain g is folded into the weights
+// once (fold_gain_kernel: Wg = g (.) W, weights do not change between calls) and r is a per-row
+// scalar, so the product is a plain GEMM X Wg whose rows are scaled by r at the end:
+//   one CTA = 128 tokens x 128 output channels (one KV head of K^ or of V^ when d = 128), K loop
+//   over d_model in steps of 128 through a three-stage TMA ring, tcgen05.mma with the accumulator
+//   in tensor memory.  While a stage of X sits in shared memory the epilogue warps add up the
+//   squares of their rows from it, so X is read once and there is no separate normalisation pass.
+// Roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer (whole warp walks, one elected lane
+// issues), warps 2-5 row statistics during the loop, then scale / round to bf16 / scatter.
+// Every wait is bounded and reports through the status word.
+#include <algorithm>
+
+#include "kernels.h"
+#include "ptx.cuh"
+#include "tcgen05.cuh"
+
+namespace yoco {
+
+// Status word of the append kernel (it takes no workspace): 0, or the code of a bounded wait that
+// ran out.  Sticky until read_and_clear_kv_append_status().
+__device__ int32_t g_kv_append_status;
+
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 128;
+constexpr int kThreads = 192;
+constexpr int HALF_BYTES = 128 * 128;            // 128 rows x 64 bf16: one swizzled half tile
+constexpr int TILE_BYTES = 2 * HALF_BYTES;       // an X tile [128 tokens, 128 k] or a W tile [128 k, 128 n]
+constexpr int STAGES = 3;
+constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+constexpr int OFF_BAR = STAGES * STAGE_BYTES;
+constexpr int SMEM_BYTES = OFF_BAR + (2 * STAGES + 1) * 8 + 16;
+constexpr uint32_t TMEM_COLS = 128;
+
+__global__ void __launch_bounds__(kThreads, 1)
+kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmWk,
+                 const __grid_constant__ CUtensorMap tmWv, const KvAppendParams p,
+                 const __grid_constant__ KvAppendTables tab) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + OFF_BAR);   // [STAGES] tile pair has landed
+    uint64_t* empty = full + STAGES;                                // [STAGES] MMA and row sums are done with it
+    uint64_t* acc_full = empty + STAGES;                            // accumulator complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * BN;          // first output column (K^ columns, then V^ columns)
+    const int m0 = blockIdx.y * BM;          // first token
+    const int KT = p.d_model / BK;
+    const Abort ab{abort_flag, &g_kv_append_status};
+    const bool aligned_ok = (smem_u32(smem) & 1023u) == 0;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = aligned_ok ? 0 : 1;
+        if (!aligned_ok) atomicExch(&g_kv_append_status, kStatusTimeout + 1);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1 + 4);     // one tcgen05.commit + four row-sum warps
+        }
+        mbar_init(acc_full, 1);
+        mbar_fence_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_acc = *tmem_slot;
+
+    if (warp == 0) {
+        // ======================================= TMA producer ================================
+        if (lane == 0 && aligned_ok) {
+            const bool is_v = n0 >= p.n_half;
+            const CUtensorMap* tmW = is_v ? &tmWv : &tmWk;
+            const int nw = n0 - (is_v ? p.n_half : 0);
+            tma_prefetch_desc(&tmX);
+            tma_prefetch_desc(tmW);
+            for (int kt = 0; kt < KT; ++kt) {
+                const uint32_t s = kt % STAGES, ph = (kt / STAGES) & 1u;
+                if (!wait_or_abort(&empty[s], ph ^ 1u, ab)) break;
+                uint8_t* a = smem + s * STAGE_BYTES;
+                uint8_t* b = a + TILE_BYTES;
+                mbar_expect_tx(&full[s], STAGE_BYTES);
+                for (int h = 0; h < 2; ++h) {
+                    tma_load_2d(a + h * HALF_BYTES, &tmX, kt * BK + h * 64, m0, &full[s]);
+                    tma_load_2d(b + h * HALF_BYTES, tmW, nw + h * 64, kt * BK, &full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ======================================= MMA issuer ==================================
+        if (aligned_ok) {
+            constexpr uint32_t idesc = make_idesc(BN, true);
+            const uint32_t sbase = smem_u32(smem);
+            bool ok = true;
+            for (int kt = 0; kt < KT && ok; ++kt) {
+                const uint32_t s = kt % STAGES, ph = (kt / STAGES) & 1u;
+                if (!(ok = warp_wait(&full[s], ph, ab))) break;
+                tc_fence_after();
+                const uint32_t a_lo = desc_lo(sbase + s * STAGE_BYTES, 16);
+                const uint32_t b_lo = desc_lo(sbase + s * STAGE_BYTES + TILE_BYTES, BK * 128);
+                if (elect_one()) {
+#pragma unroll
+                    for (int ks = 0; ks < BK / 16; ++ks) {
+                        const uint32_t a_off = ((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4;
+                        const uint32_t b_off = (uint32_t)(ks * 16 * 128) >> 4;
+                        umma_ss(tmem_acc, desc_from_lo(a_lo + a_off, 1024), desc_from_lo(b_lo + b_off, 1024), idesc,
+                                (kt > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    umma_commit(&empty[s]);
+                    if (kt == KT - 1) umma_commit(acc_full);
+                }
+                __syncwarp();
+            }
+        }
+    } else {
+        // ============================ row statistics, then epilogue ==========================
+        const int quad = warp & 3;                     // TMEM lane quadrant this warp may access
+        const int row = quad * 32 + lane;              // token row inside the tile
+        const int m = m0 + row;
+        bool ok = aligned_ok;
+        float ss = 0.f;                                // sum of squares of this token's hidden state
+        for (int kt = 0; kt < KT; ++kt) {
+            if (!ok) continue;
+            const uint32_t s = kt % STAGES, ph = (kt / STAGES) & 1u;
+            if (!(ok = warp_wait(&full[s], ph, ab))) continue;
+            const uint8_t* a = smem + s * STAGE_BYTES + row * 128;
+            float part[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    // the swizzle only permutes the 16-byte chunks of a row: any order will do, and
+                    // starting each thread at a different chunk spreads the banks
+                    const uint4 v = *reinterpret_cast<const uint4*>(a + h * HALF_BYTES + (((c + row) & 7) << 4));
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float lo = __uint_as_float(w[q] << 16), hi = __uint_as_float(w[q] & 0xFFFF0000u);
+                        part[q] = fmaf(lo, lo, part[q]);
+                        part[q] = fmaf(hi, hi, part[q]);
+                    }
+                }
+            ss += (part[0] + part[1]) + (part[2] + part[3]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[s]);
+        }
+        if (ok) ok = warp_wait(acc_full, 0u, ab);
+        if (ok) {
+            tc_fence_after();
+            const float r = 1.f / sqrtf(ss / (float)p.d_model + p.eps);
+            const int i = m / p.T, t = m - i * p.T;
+            const bool valid = m < p.M;
+            const int64_t row0 = valid ? (int64_t)tab.row0[i] + t : 0;
+            const int head_rows = valid ? tab.head_rows[i] : 0;
+#pragma unroll
+            for (int cb = 0; cb < BN / 32; ++cb) {
+                float o[32];
+                tmem_ld32(tmem_acc + ((uint32_t)(quad * 32) << 16) + cb * 32, o);
+                tmem_wait_ld();
+                if (valid) {
+                    const int n = n0 + cb * 32;
+                    const bool is_v = n >= p.n_half;
+                    const int nn = n - (is_v ? p.n_half : 0);
+                    const int c = nn / p.d, e = nn - c * p.d;
+                    __nv_bfloat16* dst = (is_v ? p.V : p.K) + (row0 + (int64_t)c * head_rows) * p.d + e;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint4 pk;
+                        pk.x = pack_bf16x2(o[q * 8 + 0] * r, o[q * 8 + 1] * r);
+                        pk.y = pack_bf16x2(o[q * 8 + 2] * r, o[q * 8 + 3] * r);
+                        pk.z = pack_bf16x2(o[q * 8 + 4] * r, o[q * 8 + 5] * r);
+                        pk.w = pack_bf16x2(o[q * 8 + 6] * r, o[q * 8 + 7] * r);
+                        *reinterpret_cast<uint4*>(dst + q * 8) = pk;
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_acc, TMEM_COLS);
+    }
+}
+
+// Wg[k, n] = g[k] * W[k, n]: the product of two bf16 values is exact in fp32, one rounding to bf16.
+__global__ void fold_gain_kernel(const __nv_bfloat16* __restrict__ g, const __nv_bfloat16* __restrict__ W,
+                                 __nv_bfloat16* __restrict__ Wg, int64_t d_model, int64_t n_out) {
+    const int64_t total = d_model * n_out;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t k = idx / n_out;
+        Wg[idx] = __float2bfloat16(__bfloat162float(g[k]) * __bfloat162float(W[idx]));
+    }
+}
+
+}  // namespace
+
+cudaError_t read_and_clear_kv_append_status(int32_t* word, cudaStream_t stream) {
+    cudaError_t e = cudaMemcpyFromSymbolAsync(word, g_kv_append_status, sizeof(int32_t), 0, cudaMemcpyDeviceToHost, stream);
+    if (e != cudaSuccess) return e;
+    if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return e;
+    if (*word == 0) return cudaSuccess;
+    const int32_t zero = 0;
+    e = cudaMemcpyToSymbolAsync(g_kv_append_status, &zero, sizeof zero, 0, cudaMemcpyHostToDevice, stream);
+    return e != cudaSuccess ? e : cudaStreamSynchronize(stream);
+}
+
+cudaError_t kv_append_kernel_setup() {
+    return cudaFuncSetAttribute(kv_append_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+}
+
+cudaError_t launch_kv_append(const KvAppendParams& p, const KvAppendTables& tab, const CUtensorMap& tmX,
+                             const CUtensorMap& tmWk, const CUtensorMap& tmWv, cudaStream_t stream) {
+    if (p.M <= 0) return cudaSuccess;
+    dim3 grid((unsigned)(2 * p.n_half / BN), (unsigned)((p.M + BM - 1) / BM));
+    kv_append_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(tmX, tmWk, tmWv, p, tab);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fold_gain(const __nv_bfloat16* g, const __nv_bfloat16* W, __nv_bfloat16* Wg, int64_t d_model,
+                             int64_t n_out, cudaStream_t stream) {
+    const int64_t total = d_model * n_out;
+    if (total <= 0) return cudaSuccess;
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 8);
+    fold_gain_kernel<<<blocks, 256, 0, stream>>>(g, W, Wg, d_model, n_out);
+    return cudaGetLastError();
+}
+
+}  // namespace yoco
