@@ -296,6 +296,53 @@ def measure_key_range_shard(dev, w, K, V, Q, shards=8):
                     "needs S GPUs and is not included"}
 
 
+def measure_kv_append(dev, peaks, hbm_peak):
+    """The step that writes the cache, on the shapes of the benchmark configs: a 2 x 512-token
+    prefill chunk (a dense contraction: tensor roofline) and one new token (the two weight
+    matrices are streamed once: HBM roofline).  d_model = Hq * d = 4,096."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    Hkv, d, d_model = 8, 128, 4096
+    n_out = Hkv * d
+    to_dev = lambda a: torch.from_numpy(a.reshape(-1).view(np.int16)).to(dev).view(torch.bfloat16)  # noqa: E731
+    Wgk = to_dev(si.normal_bf16(7, 42, d_model * n_out, mult=d_model ** -0.5)).view(d_model, n_out)
+    Wgv = to_dev(si.normal_bf16(7, 43, d_model * n_out, mult=d_model ** -0.5)).view(d_model, n_out)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    out = {}
+    for name, B, T, N in (("chunk", 2, 512, 4096), ("decode", 1, 1, 4096)):
+        X = to_dev(si.normal_bf16(7, 40, B * T * d_model))
+        K = torch.zeros(B * Hkv * N * d, dtype=torch.bfloat16, device=dev)
+        V = torch.zeros_like(K)
+        shape = bd.KvAppendShape(B, Hkv, d, T, d_model, 1e-6, 0)
+        lens = np.full(B, N, dtype=np.int32)
+        for _ in range(3):
+            bd.yoco_kv_append(shape, X, Wgk, Wgv, K, V, None, lens)
+        assert bd.yoco_kv_append_status() == 0
+        n, total = 20, 0.0
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for k in range(n):
+            flush.fill_(k)                       # weights (16.8 MB) would otherwise stay in L2
+            e0.record()
+            bd.yoco_kv_append(shape, X, Wgk, Wgv, K, V, None, lens)
+            e1.record()
+            torch.cuda.synchronize()
+            total += e0.elapsed_time(e1)
+        us = total * 1e3 / n
+        flop = 2.0 * B * T * d_model * 2 * n_out
+        wbytes = 2 * d_model * n_out * 2 + B * T * (d_model + 2 * n_out) * 2
+        if name == "chunk":
+            burst = float(peaks.get("bf16_tflops", 1590.0))
+            out[name] = {"workload": f"B={B} T={T} d_model={d_model} Hkv={Hkv} d={d}", "call_us": us, "flop": flop,
+                         "bound": "tensor", "achieved": flop / us / 1e6, "unit": "TFLOP/s", "peak": burst,
+                         "frac": flop / us / 1e6 / burst}
+        else:
+            out[name] = {"workload": f"B={B} T={T} d_model={d_model} Hkv={Hkv} d={d}", "call_us": us,
+                         "algorithmic_bytes": wbytes, "bound": "hbm", "achieved": wbytes / us / 1e3, "unit": "GB/s",
+                         "peak": hbm_peak, "frac": wbytes / us / 1e3 / hbm_peak}
+    out["l2"] = "L2 flushed before every timed call (512 MB write); time includes the launch (event pair around one call)"
+    return out
+
+
 def run_ours(args):
     import torch
     from paper_2405_05254_b200 import binding as bd
@@ -450,6 +497,8 @@ def run_ours(args):
             del K, V
             torch.cuda.empty_cache()
             line["chunk"] = measure_chunk(dev, peaks, args.chunk_workload)
+        if world == 1 and not args.no_append:
+            line["kv_append"] = measure_kv_append(dev, peaks, peak)
         if world == 1 and not args.no_window:
             line["sliding_window"] = measure_window(dev, peak)
         if world == 1 and not args.no_cpu_baseline:
@@ -471,6 +520,7 @@ def main():
     ap.add_argument("--workload", default="1m", choices=["1m", "128k", "3b_32k", "ragged", "tiny"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-chunk", action="store_true", help="skip the extra measurement of the chunk path")
+    ap.add_argument("--no-append", action="store_true", help="skip the cache-writing (K/V projection) measurement")
     ap.add_argument("--no-shard", action="store_true", help="skip the key-range-shard measurement")
     ap.add_argument("--no-window", action="store_true", help="skip the sliding-window decode measurement")
     ap.add_argument("--only-chunk", action="store_true", help="measure the chunk path alone")
