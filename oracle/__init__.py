@@ -42,6 +42,11 @@ def _load():
         lib.oracle_xattn_rows.argtypes = common + [i64, ptr, ptr, ptr, ptr, ptr]
         lib.oracle_xattn_split_merge.argtypes = common + [i32, ptr, ptr, ptr]
         lib.oracle_combine.argtypes = [i64, i32, i32, ptr, ptr, ptr, ptr]
+        lib.oracle_xattn_fp8.argtypes = [i32, i32, i32, i32, i32, f64, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i64, i32,
+                                         ptr, ptr]
+        lib.oracle_xattn_fp8.restype = i32
+        lib.oracle_e4m3_to_f64.argtypes = [ctypes.c_uint8]
+        lib.oracle_e4m3_to_f64.restype = f64
         for f in (lib.oracle_xattn, lib.oracle_xattn_rows, lib.oracle_xattn_split_merge,
                   lib.oracle_combine, lib.oracle_num_threads):
             f.restype = i32
@@ -142,3 +147,31 @@ def combine(part_o, part_lse):
     if rc:
         raise ValueError(f"oracle_combine failed ({rc})")
     return O, LSE
+
+
+def e4m3_to_f64(byte: int) -> float:
+    """Value of one FP8 E4M3 byte (the oracle's own decoder)."""
+    return float(_load().oracle_e4m3_to_f64(int(byte) & 0xFF))
+
+
+def xattn_fp8(Q, K8, V8, k_scale, v_scale, cu, kv_len, *, B, Hq, Hkv, d, T, scale=0.0, kv_head_stride=0, window=0):
+    """The same definition over an 8-bit cache: K8, V8 are uint8 E4M3 bytes in the packed head-major
+    layout, k_scale / v_scale fp32 [Hkv]; an element's value is scale[c] * e4m3(byte)."""
+    Q = np.ascontiguousarray(Q, dtype=np.uint16)
+    K8 = np.ascontiguousarray(K8, dtype=np.uint8).reshape(-1)
+    V8 = np.ascontiguousarray(V8, dtype=np.uint8).reshape(-1)
+    k_scale = np.ascontiguousarray(k_scale, dtype=np.float32)
+    v_scale = np.ascontiguousarray(v_scale, dtype=np.float32)
+    cu = np.ascontiguousarray(cu, dtype=np.int32)
+    kv_len = np.ascontiguousarray(kv_len, dtype=np.int32)
+    if Q.size != B * Hq * T * d or k_scale.size != Hkv or v_scale.size != Hkv:
+        raise ValueError("Q must hold B*Hq*T*d values and the scales Hkv values each")
+    _check_extent(K8, V8, cu, kv_len, Hkv, d, kv_head_stride)
+    O = np.empty((B, Hq, T, d), dtype=np.float64)
+    LSE = np.empty((B, Hq, T), dtype=np.float64)
+    rc = _load().oracle_xattn_fp8(B, Hq, Hkv, d, T, float(scale), _p(Q), _p(K8), _p(V8), _p(k_scale), _p(v_scale),
+                                  _p(cu), _p(kv_len), int(kv_head_stride), int(window), _p(O), _p(LSE))
+    if rc:
+        raise ValueError(f"oracle_xattn_fp8 failed ({rc})")
+    return O, LSE
+

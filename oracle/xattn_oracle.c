@@ -35,6 +35,11 @@
  * being kv_head_stride elements (0 means tight: N_i * d).
  *   element(i, c, j, e) = cu[i] * Hkv * d + c * head_stride_i + j * d + e
  *
+ * Optional 8-bit cache (Section 1 sizes the cache at 8 bits per value): K and V may be given
+ * as FP8 E4M3 bytes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; exponent field 0 is
+ * subnormal m/8 * 2^-6; 0x7F / 0xFF are NaN; no infinities) with one fp32 scale per KV head:
+ * the value of an element is scale[c] * e4m3(byte).  Everything else is unchanged.
+ *
  * Pins (tests/test_oracle_pins.py): single key, identical keys -> prefix means,
  * permutation invariance, split + merge = unsplit, brute force without max
  * subtraction, two-key logistic closed form, affine map of V, key shift,
@@ -75,7 +80,32 @@ typedef struct {
     const int32_t *kv_len;
     int64_t kv_head_stride;
     int32_t window;
+    /* 8-bit cache: when K8 is set, K and V above are unused */
+    const uint8_t *K8, *V8;
+    const float *k_scale, *v_scale;   /* [Hkv] */
 } problem_t;
+
+/* FP8 E4M3 byte -> value, from the format's definition. */
+double oracle_e4m3_to_f64(uint8_t b)
+{
+    int sign = b >> 7, ex = (b >> 3) & 15, man = b & 7;
+    double v;
+    if (ex == 15 && man == 7) return NAN;
+    if (ex == 0) v = ldexp((double)man / 8.0, -6);
+    else v = ldexp(1.0 + (double)man / 8.0, ex - 7);
+    return sign ? -v : v;
+}
+
+/* Element idx (in elements from the start of the packed buffer) of K (which = 0) or V (1). */
+static double kv_val(const problem_t *p, int which, int c, int64_t idx)
+{
+    if (p->K8) {
+        const uint8_t *buf = which ? p->V8 : p->K8;
+        const float *sc = which ? p->v_scale : p->k_scale;
+        return (double)sc[c] * oracle_e4m3_to_f64(buf[idx]);
+    }
+    return bf16_bits_to_f64((which ? p->V : p->K)[idx]);
+}
 
 static int64_t kv_base(const problem_t *p, int i, int c)
 {
@@ -112,8 +142,7 @@ static void row_over_range(const problem_t *p, int i, int h, int t,
     const int G = p->Hq / p->Hkv;
     const int c = h / G;
     const uint16_t *q = p->Q + (((int64_t)i * p->Hq + h) * p->T + t) * d;
-    const uint16_t *Kc = p->K + kv_base(p, i, c);
-    const uint16_t *Vc = p->V + kv_base(p, i, c);
+    const int64_t kvb = kv_base(p, i, c);
 
     for (int e = 0; e < d; ++e) out[e] = 0.0;
     if (j1 <= j0) {
@@ -122,9 +151,8 @@ static void row_over_range(const problem_t *p, int i, int h, int t,
     }
     double m = -INFINITY;
     for (int64_t j = j0; j < j1; ++j) {
-        const uint16_t *k = Kc + j * d;
         double s = 0.0;
-        for (int e = 0; e < d; ++e) s += bf16_bits_to_f64(q[e]) * bf16_bits_to_f64(k[e]);
+        for (int e = 0; e < d; ++e) s += bf16_bits_to_f64(q[e]) * kv_val(p, 0, c, kvb + j * d + e);
         s *= p->scale;
         scores[j - j0] = s;
         if (s > m) m = s;
@@ -133,8 +161,7 @@ static void row_over_range(const problem_t *p, int i, int h, int t,
     for (int64_t j = j0; j < j1; ++j) {
         double w = exp(scores[j - j0] - m);
         denom += w;
-        const uint16_t *v = Vc + j * d;
-        for (int e = 0; e < d; ++e) out[e] += w * bf16_bits_to_f64(v[e]);
+        for (int e = 0; e < d; ++e) out[e] += w * kv_val(p, 1, c, kvb + j * d + e);
     }
     for (int e = 0; e < d; ++e) out[e] /= denom;
     *lse = m + log(denom);
@@ -313,3 +340,41 @@ int oracle_combine(int64_t rows, int32_t S, int32_t d, const float *part_o,
     free(po); free(plse);
     return 0;
 }
+
+/* The same definition over an 8-bit cache: K8, V8 hold E4M3 bytes in the packed head-major
+ * layout (strides in elements as before), k_scale / v_scale one fp32 factor per KV head. */
+int oracle_xattn_fp8(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t T, double scale,
+                     const uint16_t *Q, const uint8_t *K8, const uint8_t *V8,
+                     const float *k_scale, const float *v_scale,
+                     const int32_t *cu, const int32_t *kv_len, int64_t kv_head_stride, int32_t window,
+                     double *O, double *LSE)
+{
+    if (check_shape(B, Hq, Hkv, d, T) || window < 0) return -1;
+    problem_t p = {B, Hq, Hkv, d, T, resolve_scale(scale, d), Q, NULL, NULL, cu, kv_len, kv_head_stride, window,
+                   K8, V8, k_scale, v_scale};
+    int64_t max_len = 1;
+    for (int i = 0; i < B; ++i)
+        if (kv_len[i] > max_len) max_len = kv_len[i];
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *scores = (double *)malloc(sizeof(double) * (size_t)max_len);
+        if (!scores) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for collapse(2) schedule(dynamic, 1)
+        for (int i = 0; i < B; ++i)
+            for (int h = 0; h < Hq; ++h) {
+                if (!scores) continue;
+                for (int t = 0; t < T; ++t) {
+                    int64_t row = ((int64_t)i * Hq + h) * T + t;
+                    row_over_range(&p, i, h, t, first_visible(&p, i, t), visible_keys(&p, i, t), scores,
+                                   O + row * d, LSE + row);
+                }
+            }
+        free(scores);
+    }
+    return failed ? -2 : 0;
+}
+

@@ -73,6 +73,27 @@ def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     return (u >> 16).astype(np.uint16)
 
 
+def e4m3_table() -> np.ndarray:
+    """Values of the 256 FP8 E4M3 codes (1 sign, 4 exponent bits, bias 7, 3 mantissa bits; exponent
+    field 0 subnormal; 0x7F / 0xFF NaN), float64."""
+    code = np.arange(256)
+    ex, man = (code >> 3) & 15, code & 7
+    val = np.where(ex == 0, man / 8.0 * 2.0 ** -6, (1.0 + man / 8.0) * 2.0 ** (ex.astype(np.float64) - 7))
+    val = np.where((ex == 15) & (man == 7), np.nan, val)
+    return np.where(code >= 128, -val, val)
+
+
+def quantize_e4m3(x: np.ndarray) -> np.ndarray:
+    """Nearest E4M3 code of every element of x (float), ties to the even code, saturating at +-448."""
+    pos = e4m3_table()[:127]                               # 0x00 .. 0x7E, ascending
+    mid = (pos[:-1] + pos[1:]) / 2
+    a = np.minimum(np.abs(np.asarray(x, dtype=np.float64)), 448.0)
+    idx = np.searchsorted(mid, a, side="left")             # a == mid[i] -> i (the lower neighbour)
+    tie = (idx < 126) & (a == mid[np.minimum(idx, 125)]) & (idx % 2 == 1)
+    idx = idx + tie
+    return (idx | np.where(np.signbit(x), 128, 0)).astype(np.uint8)
+
+
 @dataclass
 class Workload:
     """One seeded problem instance: shapes, lengths and the packed-layout offsets."""
@@ -116,6 +137,27 @@ class Workload:
 
     def make_v(self) -> np.ndarray:
         return normal_bf16(self.seed, TID_V, self.kv_elems)
+
+    def make_kv_fp8(self):
+        """The same K and V draws stored as an 8-bit cache: (K8, V8, k_scale [Hkv], v_scale [Hkv]) with
+        E4M3 bytes in the packed head-major layout and one scale per KV head, amax / 448 over all
+        sequences, so that value = scale[c] * e4m3(byte)."""
+        out = []
+        for bits in (self.make_k(), self.make_v()):
+            x = bf16_bits_to_f32(bits)
+            amax = np.zeros(self.Hkv, dtype=np.float32)
+            views, off = [], 0
+            for n in self.kv_len:
+                v = x[off:off + self.Hkv * int(n) * self.d].reshape(self.Hkv, int(n), self.d)
+                views.append(v)
+                off += self.Hkv * int(n) * self.d
+                if n:
+                    amax = np.maximum(amax, np.abs(v).max(axis=(1, 2)))
+            scale = np.where(amax > 0, amax / 448.0, 1.0).astype(np.float32)
+            q = np.concatenate([quantize_e4m3(v / scale[:, None, None]).reshape(-1) for v in views]) \
+                if views else np.zeros(0, np.uint8)
+            out.append((q, scale))
+        return out[0][0], out[1][0], out[0][1], out[1][1]
 
 
 def ragged_lengths(seed: int, B: int, lo: int, span: int) -> np.ndarray:
