@@ -180,6 +180,19 @@ int32_t yoco_xattn_chunk(const yoco_xattn_shape* shape, const void* Q, const voi
 int32_t yoco_xattn_combine(int64_t rows, int32_t S, int32_t d, const float* part_o,
                            const float* part_lse, void* O, float* lse, void* stream);
 
+/* Decode over an 8-bit cache (Section 1 sizes the cache at 8 bits per value): K8, V8 hold FP8 E4M3
+ * bytes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities) in the packed
+ * head-major layout described above, one byte per element (offsets and kv_head_stride count
+ * elements as before), and the value of an element of KV head c is k_scale[c] * e4m3(byte)
+ * (v_scale[c] for V).  k_scale_host, v_scale_host: host [Hkv], finite and > 0.  Q, O, lse,
+ * workspace, lengths, offsets, window and the result are as for yoco_xattn_decode (Q and O stay
+ * bf16); |Q| must stay below 65504, it is widened to fp16 for the products.  d = 128 only,
+ * Hkv <= 64.  Half the bytes per key are streamed, so the same bandwidth serves twice the keys. */
+int32_t yoco_xattn_decode_fp8(const yoco_xattn_shape* shape, const void* Q, const void* K8, const void* V8,
+                              const float* k_scale_host, const float* v_scale_host,
+                              const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
 /* The same merge for pieces laid out piece-major: part_o [S, rows, d], part_lse [S, rows] -- what
  * an all-gather over S ranks leaves when every rank contributes its [rows, d] partial result and
  * its [rows] log-sum-exp.  Otherwise as yoco_xattn_combine. */

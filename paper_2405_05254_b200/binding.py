@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.yoco_xattn_combine.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
         L.yoco_xattn_combine_gathered.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
         L.yoco_xattn_decode_partial.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.yoco_xattn_decode_fp8.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.yoco_xattn_decode_fp8.restype = i32
         L.yoco_kv_fold_gain.argtypes = [i64, i64, vp, vp, vp, vp]
         L.yoco_kv_append.argtypes = [ctypes.POINTER(KvAppendShape), vp, vp, vp, vp, vp, vp, vp, vp]
         L.yoco_kv_append_status.argtypes = [vp]
@@ -186,6 +188,21 @@ def yoco_xattn_decode_partial(shape: Shape, Q, K, V, cu_kv, kv_len, part_o, part
                                          workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     if rc != OK:
         raise YocoError(rc, "yoco_xattn_decode_partial")
+
+
+def yoco_xattn_decode_fp8(shape: Shape, Q, K8, V8, k_scale, v_scale, cu_kv, kv_len, O, lse, workspace,
+                          stream=None) -> None:
+    """Decode over an FP8 E4M3 cache (uint8 device tensors) with per-head scales (host float32 [Hkv])."""
+    keep_cu, p_cu = _host_i32(cu_kv)
+    keep_len, p_len = _host_i32(kv_len)
+    ks = np.ascontiguousarray(k_scale, dtype=np.float32)
+    vs = np.ascontiguousarray(v_scale, dtype=np.float32)
+    rc = lib().yoco_xattn_decode_fp8(ctypes.byref(shape), _ptr(Q), _ptr(K8), _ptr(V8),
+                                     ctypes.c_void_p(ks.ctypes.data), ctypes.c_void_p(vs.ctypes.data), p_cu, p_len,
+                                     _ptr(O), _ptr(lse), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_decode_fp8")
 
 
 def yoco_kv_fold_gain(g, W, Wg, stream=None) -> None:

@@ -51,6 +51,7 @@ int32_t device_state(DeviceState** out) {
         YOCO_CUDA_TRY(chunk_kernel_setup());
         YOCO_CUDA_TRY(chunk_pair_kernel_setup());
         YOCO_CUDA_TRY(kv_append_kernel_setup());
+        YOCO_CUDA_TRY(decode_fp8_kernel_setup());
         st.ready = true;
     }
     *out = &st;
@@ -165,6 +166,28 @@ int32_t make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int32_t d,
     return YOCO_OK;
 }
 
+// 2-D byte map over a row-major [rows, 128] matrix of FP8 values, box {128, box_rows}, 128-byte swizzle.
+int32_t make_map_2d_u8(CUtensorMap* map, const void* base, int64_t rows, int32_t box_rows) {
+    EncodeTiledFn enc;
+    int32_t rc = get_encoder(&enc);
+    if (rc != YOCO_OK) return rc;
+    cuuint64_t gdim[2] = {128u, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {128u};
+    cuuint32_t box[2] = {128u, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+    return YOCO_OK;
+}
+
+// per-head scales of an 8-bit cache (host pointers)
+struct Fp8Scales {
+    const float* k_scale;
+    const float* v_scale;
+};
+
 // ---- optional per-launch timing of the attention kernel -------------------------------------
 struct Profiler {
     std::vector<cudaEvent_t> events;   // pairs: before / after the attention kernel
@@ -188,7 +211,8 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 
 int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const void* K, const void* V,
             const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
-            void* workspace, size_t workspace_bytes, void* stream_v, float* part_out = nullptr) {
+            void* workspace, size_t workspace_bytes, void* stream_v, float* part_out = nullptr,
+            const Fp8Scales* fp8 = nullptr) {
     // part_out != null: the result is a partial one (fp32 rows + their LSE in `lse`, no bf16 O)
     if (!shape) return YOCO_ERR_INVALID_ARG;
     int32_t rc = validate_shape(*shape, mode);
@@ -234,8 +258,13 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
         if (prof) YOCO_CUDA_TRY(cudaEventRecord(ev, stream));
         if (mode == YOCO_MODE_DECODE) {
             CUtensorMap tmK, tmV;
-            if ((rc = make_map_2d(&tmK, K, plan.kv_rows_extent, shape->d, kDecodeTileN)) != YOCO_OK) return rc;
-            if ((rc = make_map_2d(&tmV, V, plan.kv_rows_extent, shape->d, kDecodeTileN)) != YOCO_OK) return rc;
+            if (fp8) {
+                if ((rc = make_map_2d_u8(&tmK, K, plan.kv_rows_extent, kDecodeTileN)) != YOCO_OK) return rc;
+                if ((rc = make_map_2d_u8(&tmV, V, plan.kv_rows_extent, kDecodeTileN)) != YOCO_OK) return rc;
+            } else {
+                if ((rc = make_map_2d(&tmK, K, plan.kv_rows_extent, shape->d, kDecodeTileN)) != YOCO_OK) return rc;
+                if ((rc = make_map_2d(&tmV, V, plan.kv_rows_extent, shape->d, kDecodeTileN)) != YOCO_OK) return rc;
+            }
             DecodeParams p{};
             p.Q = static_cast<const __nv_bfloat16*>(Q);
             p.O = static_cast<__nv_bfloat16*>(O);
@@ -251,8 +280,20 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             p.d = shape->d;
             p.window = shape->window;
             p.force_partial = part_out ? 1 : 0;
-            YOCO_CUDA_TRY(launch_decode(p, tmK, tmV, plan.info.num_groups, stream,
-                                        inline_tables ? &ready->decode_tab : nullptr));
+            if (fp8) {
+                DecodeFp8Params p8{};
+                p8.base = p;
+                p8.Hkv = shape->Hkv;
+                for (int c = 0; c < shape->Hkv; ++c) {
+                    p8.score_scale_log2[c] = scale * fp8->k_scale[c] * 1.4426950408889634f;
+                    p8.v_scale[c] = fp8->v_scale[c];
+                }
+                YOCO_CUDA_TRY(launch_decode_fp8(p8, tmK, tmV, plan.info.num_groups, stream,
+                                                inline_tables ? &ready->decode_tab : nullptr));
+            } else {
+                YOCO_CUDA_TRY(launch_decode(p, tmK, tmV, plan.info.num_groups, stream,
+                                            inline_tables ? &ready->decode_tab : nullptr));
+            }
         } else {
             CUtensorMap tmQ, tmK, tmV;
             const int64_t q_rows = (int64_t)shape->B * shape->Hq * shape->T;
@@ -449,6 +490,21 @@ int32_t yoco_xattn_decode_partial(const yoco_xattn_shape* shape, const void* Q, 
     if (shape->T != 1 || shape->window != 0) return YOCO_ERR_UNSUPPORTED;
     return run(shape, YOCO_MODE_DECODE, Q, K, V, cu_kv_host, kv_len_host, nullptr, part_lse, workspace,
                workspace_bytes, stream, part_o);
+}
+
+int32_t yoco_xattn_decode_fp8(const yoco_xattn_shape* shape, const void* Q, const void* K8, const void* V8,
+                              const float* k_scale_host, const float* v_scale_host, const int32_t* cu_kv_host,
+                              const int32_t* kv_len_host, void* O, float* lse, void* workspace,
+                              size_t workspace_bytes, void* stream) {
+    if (!shape || !k_scale_host || !v_scale_host) return YOCO_ERR_INVALID_ARG;
+    if (shape->d != 128 || shape->Hkv > kFp8MaxHeads) return YOCO_ERR_UNSUPPORTED;
+    for (int c = 0; c < shape->Hkv; ++c)
+        if (!(k_scale_host[c] > 0.f) || !(v_scale_host[c] > 0.f) || !std::isfinite(k_scale_host[c]) ||
+            !std::isfinite(v_scale_host[c]))
+            return YOCO_ERR_INVALID_ARG;
+    const Fp8Scales sc{k_scale_host, v_scale_host};
+    return run(shape, YOCO_MODE_DECODE, Q, K8, V8, cu_kv_host, kv_len_host, O, lse, workspace, workspace_bytes,
+               stream, nullptr, &sc);
 }
 
 int32_t yoco_kv_fold_gain(int64_t d_model, int64_t n_out, const void* g, const void* W, void* Wg, void* stream) {

@@ -82,6 +82,20 @@ cudaError_t launch_decode(const DecodeParams& p, const CUtensorMap& tmK, const C
 cudaError_t decode_kernel_setup();
 
 
+// ---- decode over an 8-bit (FP8 E4M3) cache, head dimension 128 ---------------------------------
+constexpr int kFp8MaxHeads = 64;
+struct DecodeFp8Params {
+    DecodeParams base;                    // as for the bf16 kernel; base.scale_log2 is unused
+    int32_t Hkv;
+    float score_scale_log2[kFp8MaxHeads]; // per KV head: softmax scale * k_scale[c] * log2(e)
+    float v_scale[kFp8MaxHeads];          // per KV head
+};
+// tmK / tmV: 2-D uint8 tensor maps over the [rows, 128] byte view of K and V, box {128, 64},
+// 128-byte swizzle.
+cudaError_t launch_decode_fp8(const DecodeFp8Params& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                              int num_groups, cudaStream_t stream, const DecodeInlineTables* inline_tab);
+cudaError_t decode_fp8_kernel_setup();
+
 struct ChunkParams {
     __nv_bfloat16* O;           // [B*Hq*T, d]
     float* lse;                 // [B*Hq*T] or null
