@@ -343,6 +343,49 @@ def measure_kv_append(dev, peaks, hbm_peak):
     return out
 
 
+def measure_fp8_cache(dev, w, Q, peak_gbs):
+    """The headline decode over an 8-bit cache of the same length (FP8 E4M3 bytes, per-head scales):
+    half the bytes per key.  The bytes are random valid codes drawn on the device (timing does not
+    depend on the values; parity is covered by the tests)."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    n = w.kv_elems
+    gen = torch.Generator(device=dev).manual_seed(1234)
+    K8 = (torch.randint(0, 127, (n,), dtype=torch.uint8, device=dev, generator=gen)
+          + 128 * torch.randint(0, 2, (n,), dtype=torch.uint8, device=dev, generator=gen))
+    V8 = K8.flip(0).contiguous()
+    ks = np.full(w.Hkv, 1.0 / 64, dtype=np.float32)
+    vs = np.full(w.Hkv, 1.0 / 64, dtype=np.float32)
+    shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(w.kv_len.max()))
+    ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_DECODE), dtype=torch.uint8, device=dev)
+    O = torch.empty(w.B * w.Hq * w.T * w.d, dtype=torch.bfloat16, device=dev)
+
+    def call():
+        bd.yoco_xattn_decode_fp8(shape, Q, K8, V8, ks, vs, w.cu, w.kv_len, O, None, ws)
+
+    for _ in range(3):
+        call()
+    assert bd.yoco_xattn_status(ws) == 0 and bool(torch.isfinite(O.float()).all())
+    reps = 20
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    call_us = e0.elapsed_time(e1) * 1e3 / reps
+    bd.yoco_xattn_profile_enable(reps)
+    for _ in range(reps):
+        call()
+    k_us = float(bd.yoco_xattn_profile_collect(reps).mean()) * 1e3
+    bd.yoco_xattn_profile_enable(0)
+    nbytes = 2 * n
+    return {"workload": f"{w.name} with an FP8 E4M3 cache: kv_len={int(w.kv_len.max())}, K8 + V8 = {nbytes} bytes",
+            "algorithmic_bytes_per_launch": nbytes, "kernel_us": k_us, "call_us": call_us,
+            "us_per_token_layer": call_us / w.B, "bound": "hbm", "achieved": nbytes / k_us / 1e3, "unit": "GB/s",
+            "peak": peak_gbs, "frac": nbytes / k_us / 1e3 / peak_gbs}
+
+
 def run_ours(args):
     import torch
     from paper_2405_05254_b200 import binding as bd
@@ -491,6 +534,8 @@ def run_ours(args):
                                        "every attention kernel",
                          "traffic": traffic},
         }
+        if world == 1 and w.d == 128 and not args.no_fp8:
+            line["fp8_cache"] = measure_fp8_cache(dev, w, Qd[0], peak)
         if world == 1 and w.B == 1 and w.T == 1 and not args.no_shard:
             line["key_range_shard"] = measure_key_range_shard(dev, w, K, V, Qd[0])
         if world == 1 and not args.no_chunk:
@@ -520,6 +565,7 @@ def main():
     ap.add_argument("--workload", default="1m", choices=["1m", "128k", "3b_32k", "ragged", "tiny"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-chunk", action="store_true", help="skip the extra measurement of the chunk path")
+    ap.add_argument("--no-fp8", action="store_true", help="skip the decode over an 8-bit cache")
     ap.add_argument("--no-append", action="store_true", help="skip the cache-writing (K/V projection) measurement")
     ap.add_argument("--no-shard", action="store_true", help="skip the key-range-shard measurement")
     ap.add_argument("--no-window", action="store_true", help="skip the sliding-window decode measurement")
