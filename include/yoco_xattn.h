@@ -180,7 +180,7 @@ int32_t yoco_xattn_chunk(const yoco_xattn_shape* shape, const void* Q, const voi
 int32_t yoco_xattn_combine(int64_t rows, int32_t S, int32_t d, const float* part_o,
                            const float* part_lse, void* O, float* lse, void* stream);
 
-/* Decode over an 8-bit cache (Section 1 sizes the cache at 8 bits per value): K8, V8 hold FP8 E4M3
+/* Decode over an 8-bit cache (Section 1 assumes 8-bit K/V quantisation when it sizes a cache): K8, V8 hold FP8 E4M3
  * bytes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities) in the packed
  * head-major layout described above, one byte per element (offsets and kv_head_stride count
  * elements as before), and the value of an element of KV head c is k_scale[c] * e4m3(byte)

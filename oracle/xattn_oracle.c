@@ -35,7 +35,7 @@
  * being kv_head_stride elements (0 means tight: N_i * d).
  *   element(i, c, j, e) = cu[i] * Hkv * d + c * head_stride_i + j * d + e
  *
- * Optional 8-bit cache (Section 1 sizes the cache at 8 bits per value): K and V may be given
+ * Optional 8-bit cache (Section 1 assumes 8-bit K/V quantisation when it sizes a cache): K and V may be given
  * as FP8 E4M3 bytes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; exponent field 0 is
  * subnormal m/8 * 2^-6; 0x7F / 0xFF are NaN; no infinities) with one fp32 scale per KV head:
  * the value of an element is scale[c] * e4m3(byte).  Everything else is unchanged.
