@@ -44,9 +44,9 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)", {}
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of decode_kernel<128, 8> per launch from the ncu capture
+# dram__bytes_read.sum + dram__bytes_write.sum of decode_kernel_inline<128, 8> per launch from the ncu capture
 # summarised in profiles/decode_kernel_128k_ncu_full.md (mean of two launches, 128K-token case).
-NCU_DECODE_DRAM_BYTES = 540852736
+NCU_DECODE_DRAM_BYTES = 541321984
 NCU_DECODE_KV_BYTES = 536870912
 
 
