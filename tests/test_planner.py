@@ -17,7 +17,7 @@ def declared_symbols():
     for fn in os.listdir(os.path.join(ROOT, "include")):
         if fn.endswith(".h"):
             src = open(os.path.join(ROOT, "include", fn)).read()
-            names |= set(re.findall(r"\b(yoco_xattn_[a-z_0-9]+)\s*\(", src))
+            names |= set(re.findall(r"\b(yoco_(?:xattn|kv)_[a-z_0-9]+)\s*\(", src))
     return sorted(names)
 
 
@@ -25,7 +25,9 @@ def test_library_exports_every_declared_symbol():
     L = bd.lib()
     syms = declared_symbols()
     assert {"yoco_xattn_decode", "yoco_xattn_chunk", "yoco_xattn_combine", "yoco_xattn_plan",
-            "yoco_xattn_workspace_size", "yoco_xattn_status", "yoco_xattn_strerror"} <= set(syms)
+            "yoco_xattn_workspace_size", "yoco_xattn_status", "yoco_xattn_strerror", "yoco_xattn_decode_partial",
+            "yoco_xattn_combine_gathered", "yoco_xattn_decode_fp8", "yoco_kv_append", "yoco_kv_fold_gain",
+            "yoco_kv_append_status"} <= set(syms)
     for s in syms:
         assert hasattr(L, s), f"{s} is declared in include/ but not exported"
 
@@ -205,3 +207,31 @@ def test_negative_window_is_rejected():
     with pytest.raises(bd.YocoError) as e:
         bd.yoco_xattn_plan(shape, [100], 148, bd.MODE_DECODE)
     assert e.value.code == bd.ERR_INVALID_ARG
+
+
+def test_new_entry_points_validate_arguments_before_touching_cuda():
+    """Shape and pointer errors of the later entry points come back as codes on a box without a GPU."""
+    L = bd.lib()
+    p = ctypes.c_void_p
+    ok_shape = bd.KvAppendShape(1, 8, 128, 1, 4096, 1e-6, 0)
+    lens = np.array([4], dtype=np.int32)
+    pl = p(lens.ctypes.data)
+    assert L.yoco_kv_append(None, p(16), p(16), p(16), p(16), p(16), None, pl, None) == bd.ERR_INVALID_ARG
+    for bad in (bd.KvAppendShape(1, 8, 128, 1, 4000, 1e-6, 0),        # d_model not a multiple of 128
+                bd.KvAppendShape(1, 8, 96, 1, 4096, 1e-6, 0),         # head size
+                bd.KvAppendShape(600, 8, 128, 1, 4096, 1e-6, 0)):     # too many sequences for the parameter table
+        assert L.yoco_kv_append(ctypes.byref(bad), p(16), p(16), p(16), p(16), p(16), None, pl, None) == bd.ERR_UNSUPPORTED
+    neg = bd.KvAppendShape(1, 8, 128, 1, 4096, -1.0, 0)
+    assert L.yoco_kv_append(ctypes.byref(neg), p(16), p(16), p(16), p(16), p(16), None, pl, None) == bd.ERR_INVALID_ARG
+    assert L.yoco_kv_append(ctypes.byref(ok_shape), None, p(16), p(16), p(16), p(16), None, pl, None) == bd.ERR_INVALID_ARG
+    assert L.yoco_kv_fold_gain(-1, 8, p(16), p(16), p(32), None) == bd.ERR_INVALID_ARG
+    assert L.yoco_kv_fold_gain(8, 8, p(16), p(32), p(32), None) == bd.ERR_INVALID_ARG      # Wg aliases W
+    shape = bd.make_shape(1, 8, 8, 64, 1, max_kv_len=64)
+    ones = np.ones(8, dtype=np.float32)
+    po = p(ones.ctypes.data)
+    assert L.yoco_xattn_decode_fp8(ctypes.byref(shape), p(16), p(16), p(16), po, po, None, None, p(16), None, p(256), 1 << 20,
+                                   None) == bd.ERR_UNSUPPORTED                             # d = 64
+    shape2 = bd.make_shape(1, 8, 8, 128, 2, max_kv_len=64)
+    assert L.yoco_xattn_decode_partial(ctypes.byref(shape2), p(16), p(16), p(16), None, None, p(16), p(16), p(256),
+                                       1 << 20, None) == bd.ERR_UNSUPPORTED                # T = 2
+    assert L.yoco_xattn_combine_gathered(4, 0, 128, None, None, None, None, None) == bd.ERR_INVALID_ARG
