@@ -41,11 +41,11 @@ def measured_peaks():
         with open(p) as f:
             d = json.load(f)
         return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)", d
-    return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)", {}
+    return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, an earlier measurement of the same GPU model)", {}
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of decode_kernel_inline<128, 8> per launch from the ncu capture
-# summarised in profiles/decode_kernel_128k_ncu_full.md (mean of two launches, 128K-token case).
+# (mean of two launches, 128K-token case; the summary sits with the other profiler summaries).
 NCU_DECODE_DRAM_BYTES = 541321984
 NCU_DECODE_KV_BYTES = 536870912
 
