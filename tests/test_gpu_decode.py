@@ -6,7 +6,7 @@ import pytest
 
 import oracle
 import synth_inputs as si
-from helpers import GpuRunner, assert_close, assert_lse_close, errors
+from helpers import GpuRunner, assert_close, assert_lse_close, errors, to_dev_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -210,3 +210,37 @@ def test_undersized_workspace_is_refused():
     with pytest.raises(bd.YocoError) as e:
         bd.yoco_xattn_decode(shape, q, t, t, None, [4096], q.clone(), None, ws)
     assert e.value.code == bd.ERR_WORKSPACE_TOO_SMALL
+
+
+def test_layer_calls_replay_bit_identically_from_a_cuda_graph():
+    """A serving loop captures the layer calls of a step once and replays them: the call only
+    enqueues (status memset, attention kernel, merge), so a capture on a side stream must replay
+    to the same bits as the eager calls."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    w = si.Workload("graph", B=2, Hq=32, Hkv=8, d=128, T=1, layers=3, seed=29, kv_len=[20000, 333])
+    K, V = to_dev_bf16(w.make_k()), to_dev_bf16(w.make_v())
+    Qs = [to_dev_bf16(w.make_q(l).reshape(-1)) for l in range(w.layers)]
+    Os = [torch.empty(w.B * w.Hq * w.d, dtype=torch.bfloat16, device="cuda") for _ in range(w.layers)]
+    shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, 1, max_kv_len=int(w.kv_len.max()))
+    ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_DECODE), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+
+    def step():
+        for l in range(w.layers):
+            bd.yoco_xattn_decode(shape, Qs[l], K, V, w.cu, w.kv_len, Os[l], None, ws, side)
+
+    with torch.cuda.stream(side):
+        step()                                   # first call outside the capture: one-time set-up
+    torch.cuda.synchronize()
+    eager = [o.clone() for o in Os]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        step()
+    for o in Os:
+        o.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert bd.yoco_xattn_status(ws, side) == 0
+    for a, b in zip(eager, Os):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
