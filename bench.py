@@ -386,6 +386,48 @@ def measure_fp8_cache(dev, w, Q, peak_gbs):
             "peak": peak_gbs, "frac": nbytes / k_us / 1e3 / peak_gbs}
 
 
+def measure_other_configs(dev, peak_gbs):
+    """Layer-call time of the decode path on the other decode configurations (tiny, 32K with a cold and a
+    warm L2, the ragged batch of 16), for the record; not part of the default run."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    out = {}
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    for name in ("tiny", "3b_32k", "ragged"):
+        w = si.workload(name)
+        to_dev = lambda a: torch.from_numpy(a.reshape(-1).view(np.int16)).to(dev).view(torch.bfloat16)  # noqa: E731
+        K, V = to_dev(w.make_k()), to_dev(w.make_v())
+        Qs = [to_dev(w.make_q(l)) for l in range(w.layers)]
+        O = torch.empty(w.B * w.Hq * w.T * w.d, dtype=torch.bfloat16, device=dev)
+        shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(w.kv_len.max()))
+        ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_DECODE), dtype=torch.uint8, device=dev)
+        for l in range(3):
+            bd.yoco_xattn_decode(shape, Qs[l % w.layers], K, V, w.cu, w.kv_len, O, None, ws)
+        assert bd.yoco_xattn_status(ws) == 0
+        n = 26
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for k in range(n):
+            bd.yoco_xattn_decode(shape, Qs[k % w.layers], K, V, w.cu, w.kv_len, O, None, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        warm_us = e0.elapsed_time(e1) * 1e3 / n
+        cold = 0.0
+        for k in range(10):
+            flush.fill_(k)
+            e0.record()
+            bd.yoco_xattn_decode(shape, Qs[k % w.layers], K, V, w.cu, w.kv_len, O, None, ws)
+            e1.record()
+            torch.cuda.synchronize()
+            cold += e0.elapsed_time(e1) * 1e3 / 10
+        out[name] = {"workload": f"B={w.B} Hq={w.Hq} Hkv={w.Hkv} d={w.d} T={w.T} tokens={w.total_tokens}",
+                     "kv_bytes_per_call": w.kv_bytes, "back_to_back_call_us": warm_us, "cold_l2_call_us": cold,
+                     "back_to_back_gbs": w.kv_bytes / warm_us / 1e3, "cold_l2_gbs": w.kv_bytes / cold / 1e3,
+                     "us_per_token_layer": warm_us / w.B, "frac_of_measured_hbm_cold": w.kv_bytes / cold / 1e3 / peak_gbs}
+        del K, V
+    return out
+
+
 def run_ours(args):
     import torch
     from paper_2405_05254_b200 import binding as bd
@@ -546,6 +588,8 @@ def run_ours(args):
             line["kv_append"] = measure_kv_append(dev, peaks, peak)
         if world == 1 and not args.no_window:
             line["sliding_window"] = measure_window(dev, peak)
+        if world == 1 and args.all_configs:
+            line["other_configs"] = measure_other_configs(dev, peak)
         if world == 1 and not args.no_cpu_baseline:
             gbs, dt, sample, cores = oracle_sample_rate(w, Qh, Kh, Vh)
             line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
@@ -565,6 +609,8 @@ def main():
     ap.add_argument("--workload", default="1m", choices=["1m", "128k", "3b_32k", "ragged", "tiny"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-chunk", action="store_true", help="skip the extra measurement of the chunk path")
+    ap.add_argument("--all-configs", action="store_true",
+                    help="also time a layer call on the tiny, 32K and ragged configurations")
     ap.add_argument("--no-fp8", action="store_true", help="skip the decode over an 8-bit cache")
     ap.add_argument("--no-append", action="store_true", help="skip the cache-writing (K/V projection) measurement")
     ap.add_argument("--no-shard", action="store_true", help="skip the key-range-shard measurement")
