@@ -2,7 +2,8 @@
 // KV head (value = scale[c] * e4m3(byte)), head dimension 128.  Same structure as the bf16 decode
 // kernel (one CTA per contiguous range of the flat (stream, key tile) space, a TMA producer warp,
 // four consumer warps with their own online-softmax state), but a 64-key tile is 8 KB per tensor,
-// so the same HBM bandwidth streams twice as many keys.
+// so the same HBM bandwidth streams twice as many keys, and each consumer warp takes whole tiles
+// in turn (instead of a quarter of every tile) so that its fixed latencies are paid per 64 keys.
 //
 // The bytes are widened to fp16 in registers (cvt.rn.f16x2.e4m3x2 is exact) and the small
 // products run as m16n8k16 fp16 MMAs with fp32 accumulation; Q is converted bf16 -> fp16 once per
@@ -35,6 +36,7 @@ struct Cfg8 {
     static constexpr int BUDGET = 113 * 1024;     // two CTAs per SM
     static constexpr int STAGES_FIT = (BUDGET - MERGE_O_BYTES - MERGE_ML_BYTES - 128) / STAGE_BYTES;
     static constexpr int STAGES = STAGES_FIT > 5 ? 5 : STAGES_FIT;
+    static_assert(STAGES >= kConsumerWarps, "every consumer warp needs a tile in flight");
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + MERGE_O_BYTES + MERGE_ML_BYTES + 128;
     static_assert(STAGES >= 2, "need at least a double buffer");
 };
@@ -89,7 +91,7 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], kConsumerWarps);
+            mbar_init(&empty_bar[s], 1);                 // released by the one warp that read the tile
         }
         mbar_fence_init();
     }
@@ -123,10 +125,14 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
     }
 
     // ----------------------------------- consumers ---------------------------------------
+    // Each consumer warp takes WHOLE tiles, round robin (tile number mod 4): per tile a warp then runs
+    // one softmax for 64 keys instead of one per 16, which matters here because at half the bytes
+    // per key the chain of dependent latencies per tile (products, shuffles, exponentials), not
+    // the memory, would otherwise set the pace.  A tile is released by the one warp that read it.
     const int g = lane >> 2, tq = lane & 3;
     const int n_rows = p.rows_per_stream;
     // row address this lane supplies to ldmatrix.x4: matrix (lane >> 3) = (chunk pair member, key half)
-    const int ld_key = warp * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);   // key row inside the tile
+    const int ld_key16 = ((lane >> 3) & 1) * 8 + (lane & 7);            // key row inside a 16-key group
     const int ld_chunk = lane >> 4;                                      // 0: first chunk of the pair, 1: second
     uint32_t it = 0;
     bool ok = true;
@@ -164,124 +170,134 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
             for (int h = 0; h < 2; ++h) o[c][h][0] = o[c][h][1] = o[c][h][2] = o[c][h][3] = 0.f;
 
         for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += TILE_N, ++it) {
-            if (!ok) continue;
+            if (!ok || (int)(it % kConsumerWarps) != warp) continue;       // not this warp's tile
             const uint32_t stage = it % STAGES, round = it / STAGES;
             if (!mbar_wait(&full_bar[stage], round & 1u)) {
                 atomicExch(p.status, kStatusTimeout);
                 ok = false;
                 continue;
             }
-            const int kw = k0 + warp * 16;          // first key of this warp's slice
-            if (kw < seg.k_end) {
-                const uint32_t kbase = smem_u32(stage_mem + stage * STAGE_BYTES);
-                const uint32_t vbase = kbase + TENSOR_BYTES;
-                const uint32_t ld_row = ld_key * 128;
+            const uint32_t kbase = smem_u32(stage_mem + stage * STAGE_BYTES);
+            const uint32_t vbase = kbase + TENSOR_BYTES;
 
-                // ---- S = Q K^T for 16 keys (two n-tiles of 8 keys), two reduction steps per ldmatrix ----
-                float s[2][4];
+            // ---- S = Q K^T for 64 keys: four 16-key groups, two n-tiles of 8 keys each ----
+            float s[8][4];
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+            for (int nt = 0; nt < 8; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+#pragma unroll
+            for (int kg = 0; kg < 4; ++kg) {
+                const int key = kg * 16 + ld_key16;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int chunk = 2 * j + ld_chunk;
                     uint32_t r0, r1, r2, r3;   // (keys 0-7, chunk 2j) (keys 8-15, 2j) (keys 0-7, 2j+1) (keys 8-15, 2j+1)
-                    ldmatrix_x4(kbase + ld_row + (((chunk ^ ld_key) & 7) << 4), r0, r1, r2, r3);
-                    mma_f16_16816(s[0], qa[2 * j], e4m3x2_to_f16x2(r0), e4m3x2_to_f16x2(r0 >> 16));
-                    mma_f16_16816(s[1], qa[2 * j], e4m3x2_to_f16x2(r1), e4m3x2_to_f16x2(r1 >> 16));
-                    mma_f16_16816(s[0], qa[2 * j + 1], e4m3x2_to_f16x2(r2), e4m3x2_to_f16x2(r2 >> 16));
-                    mma_f16_16816(s[1], qa[2 * j + 1], e4m3x2_to_f16x2(r3), e4m3x2_to_f16x2(r3 >> 16));
+                    ldmatrix_x4(kbase + key * 128 + (((chunk ^ key) & 7) << 4), r0, r1, r2, r3);
+                    mma_f16_16816(s[2 * kg], qa[2 * j], e4m3x2_to_f16x2(r0), e4m3x2_to_f16x2(r0 >> 16));
+                    mma_f16_16816(s[2 * kg + 1], qa[2 * j], e4m3x2_to_f16x2(r1), e4m3x2_to_f16x2(r1 >> 16));
+                    mma_f16_16816(s[2 * kg], qa[2 * j + 1], e4m3x2_to_f16x2(r2), e4m3x2_to_f16x2(r2 >> 16));
+                    mma_f16_16816(s[2 * kg + 1], qa[2 * j + 1], e4m3x2_to_f16x2(r3), e4m3x2_to_f16x2(r3 >> 16));
                 }
-                // ---- scale, mask (causal edge, sequence end, window start), online softmax ----
-                const bool need_mask = kw + 16 > n_full || (p.window > 0 && kw < seg.n_kv - p.window);
-                int lo0 = -1, lo1 = -1;
-                if (need_mask && p.window > 0) {
-                    lo0 = n_full + (g % p.T) - p.window;
-                    lo1 = n_full + ((g + 8) % p.T) - p.window;
-                }
+            }
+            // ---- scale, mask (causal edge, sequence end, window start), online softmax ----
+            const bool need_mask = k0 + TILE_N > n_full || (p.window > 0 && k0 < seg.n_kv - p.window);
+            int lo0 = -1, lo1 = -1;
+            if (need_mask && p.window > 0) {
+                lo0 = n_full + (g % p.T) - p.window;
+                lo1 = n_full + ((g + 8) % p.T) - p.window;
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt)
+            for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        float v = s[nt][e] * sscale;
-                        if (need_mask) {
-                            const int j = kw + nt * 8 + tq * 2 + (e & 1);
-                            v = (j < ((e & 2) ? vis1 : vis0) && j >= ((e & 2) ? lo1 : lo0)) ? v : -INFINITY;
-                        }
-                        s[nt][e] = v;
+                for (int e = 0; e < 4; ++e) {
+                    float v = s[nt][e] * sscale;
+                    if (need_mask) {
+                        const int j = k0 + nt * 8 + tq * 2 + (e & 1);
+                        v = (j < ((e & 2) ? vis1 : vis0) && j >= ((e & 2) ? lo1 : lo0)) ? v : -INFINITY;
                     }
-                float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-                const float mn0 = fmaxf(m0, mx0);
-                const float ms0 = mn0 == -INFINITY ? 0.f : mn0;
-                const float alpha0 = exp2f(m0 - ms0);
-                m0 = mn0;
-                float alpha1 = 1.f, ms1 = 0.f;
+                    s[nt][e] = v;
+                    if (e & 2) mx1 = fmaxf(mx1, v);
+                    else mx0 = fmaxf(mx0, v);
+                }
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+            const float mn0 = fmaxf(m0, mx0);
+            const float ms0 = mn0 == -INFINITY ? 0.f : mn0;
+            const float alpha0 = exp2f(m0 - ms0);
+            m0 = mn0;
+            float alpha1 = 1.f, ms1 = 0.f;
+            if (ROWS == 16) {
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+                const float mn1 = fmaxf(m1, mx1);
+                ms1 = mn1 == -INFINITY ? 0.f : mn1;
+                alpha1 = exp2f(m1 - ms1);
+                m1 = mn1;
+            }
+            // P in [0, 1], rounded to fp16, as the A operands of the four 16-key reduction steps
+            uint32_t pa[4][4];
+            float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+            for (int kg = 0; kg < 4; ++kg) {
+                const float p00 = exp2f(s[2 * kg][0] - ms0), p01 = exp2f(s[2 * kg][1] - ms0);
+                const float p10 = exp2f(s[2 * kg + 1][0] - ms0), p11 = exp2f(s[2 * kg + 1][1] - ms0);
+                sum0 += (p00 + p01) + (p10 + p11);
+                pa[kg][0] = pack_f16x2(p00, p01);
+                pa[kg][2] = pack_f16x2(p10, p11);
                 if (ROWS == 16) {
-                    float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
-                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-                    const float mn1 = fmaxf(m1, mx1);
-                    ms1 = mn1 == -INFINITY ? 0.f : mn1;
-                    alpha1 = exp2f(m1 - ms1);
-                    m1 = mn1;
+                    const float q00 = exp2f(s[2 * kg][2] - ms1), q01 = exp2f(s[2 * kg][3] - ms1);
+                    const float q10 = exp2f(s[2 * kg + 1][2] - ms1), q11 = exp2f(s[2 * kg + 1][3] - ms1);
+                    sum1 += (q00 + q01) + (q10 + q11);
+                    pa[kg][1] = pack_f16x2(q00, q01);
+                    pa[kg][3] = pack_f16x2(q10, q11);
+                } else {
+                    pa[kg][1] = pa[kg][3] = 0u;
                 }
-                uint32_t pa[4];      // P in [0, 1], rounded to fp16, as the A operand of O += P V
-                {
-                    const float p00 = exp2f(s[0][0] - ms0), p01 = exp2f(s[0][1] - ms0);
-                    const float p10 = exp2f(s[1][0] - ms0), p11 = exp2f(s[1][1] - ms0);
-                    l0 = l0 * alpha0 + ((p00 + p01) + (p10 + p11));
-                    pa[0] = pack_f16x2(p00, p01);
-                    pa[2] = pack_f16x2(p10, p11);
-                    if (ROWS == 16) {
-                        const float q00 = exp2f(s[0][2] - ms1), q01 = exp2f(s[0][3] - ms1);
-                        const float q10 = exp2f(s[1][2] - ms1), q11 = exp2f(s[1][3] - ms1);
-                        l1 = l1 * alpha1 + ((q00 + q01) + (q10 + q11));
-                        pa[1] = pack_f16x2(q00, q01);
-                        pa[3] = pack_f16x2(q10, q11);
-                    } else {
-                        pa[1] = pa[3] = 0u;
+            }
+            l0 = l0 * alpha0 + sum0;
+            l1 = l1 * alpha1 + sum1;
+            if (__any_sync(0xffffffffu, alpha0 != 1.f || alpha1 != 1.f)) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        o[c][h][0] *= alpha0; o[c][h][1] *= alpha0;
+                        o[c][h][2] *= alpha1; o[c][h][3] *= alpha1;
                     }
-                }
-                if (__any_sync(0xffffffffu, alpha0 != 1.f || alpha1 != 1.f)) {
+            }
+            // ---- rows past the end of the sequence may hold anything (an FP8 NaN included):
+            //      zero them so that 0 * garbage cannot produce NaN in O += P V ----
+            if (k0 + TILE_N > seg.n_kv) {
+                const int first_bad = max(seg.n_kv - k0, 0);          // 0..63
+                uint8_t* vrow = stage_mem + stage * STAGE_BYTES + TENSOR_BYTES;
+                if (lane < 8)
+                    for (int r = first_bad; r < TILE_N; ++r)
+                        *reinterpret_cast<uint4*>(vrow + r * 128 + lane * 16) = make_uint4(0u, 0u, 0u, 0u);
+                __syncwarp();
+            }
+            // ---- O += P V.  The transposed ldmatrix hands this lane, for keys 2 tq and 2 tq + 1,
+            //      the two channels 16 c + 2 g and 16 c + 2 g + 1: the even channels of a chunk
+            //      form one n-tile, the odd ones the other ----
 #pragma unroll
-                    for (int c = 0; c < 8; ++c)
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            o[c][h][0] *= alpha0; o[c][h][1] *= alpha0;
-                            o[c][h][2] *= alpha1; o[c][h][3] *= alpha1;
-                        }
-                }
-                // ---- rows past the end of the sequence may hold anything (an FP8 NaN included):
-                //      zero them so that 0 * garbage cannot produce NaN in O += P V ----
-                if (kw + 16 > seg.n_kv) {
-                    const int first_bad = max(seg.n_kv - kw, 0);          // 0..15
-                    uint8_t* vrow = stage_mem + stage * STAGE_BYTES + TENSOR_BYTES;
-                    if (lane < 8)
-                        for (int r = first_bad; r < 16; ++r)
-                            *reinterpret_cast<uint4*>(vrow + (warp * 16 + r) * 128 + lane * 16) = make_uint4(0u, 0u, 0u, 0u);
-                    __syncwarp();
-                }
-                // ---- O += P V.  The transposed ldmatrix hands this lane, for keys 2 tq and 2 tq + 1,
-                //      the two channels 16 c + 2 g and 16 c + 2 g + 1: the even channels of a chunk
-                //      form one n-tile, the odd ones the other ----
+            for (int kg = 0; kg < 4; ++kg) {
+                const int key = kg * 16 + ld_key16;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int chunk = 2 * j + ld_chunk;
                     uint32_t r0, r1, r2, r3;   // (keys 0-7, chunk 2j) (keys 8-15, 2j) (keys 0-7, 2j+1) (keys 8-15, 2j+1)
-                    ldmatrix_x4_trans(vbase + ld_row + (((chunk ^ ld_key) & 7) << 4), r0, r1, r2, r3);
+                    ldmatrix_x4_trans(vbase + key * 128 + (((chunk ^ key) & 7) << 4), r0, r1, r2, r3);
                     // bytes [k0 c0, k0 c1, k1 c0, k1 c1] -> [k0 c0, k1 c0 | k0 c1, k1 c1]
                     r0 = __byte_perm(r0, 0u, 0x3120);
                     r1 = __byte_perm(r1, 0u, 0x3120);
                     r2 = __byte_perm(r2, 0u, 0x3120);
                     r3 = __byte_perm(r3, 0u, 0x3120);
-                    mma_f16_16816(o[2 * j][0], pa, e4m3x2_to_f16x2(r0), e4m3x2_to_f16x2(r1));
-                    mma_f16_16816(o[2 * j][1], pa, e4m3x2_to_f16x2(r0 >> 16), e4m3x2_to_f16x2(r1 >> 16));
-                    mma_f16_16816(o[2 * j + 1][0], pa, e4m3x2_to_f16x2(r2), e4m3x2_to_f16x2(r3));
-                    mma_f16_16816(o[2 * j + 1][1], pa, e4m3x2_to_f16x2(r2 >> 16), e4m3x2_to_f16x2(r3 >> 16));
+                    mma_f16_16816(o[2 * j][0], pa[kg], e4m3x2_to_f16x2(r0), e4m3x2_to_f16x2(r1));
+                    mma_f16_16816(o[2 * j][1], pa[kg], e4m3x2_to_f16x2(r0 >> 16), e4m3x2_to_f16x2(r1 >> 16));
+                    mma_f16_16816(o[2 * j + 1][0], pa[kg], e4m3x2_to_f16x2(r2), e4m3x2_to_f16x2(r3));
+                    mma_f16_16816(o[2 * j + 1][1], pa[kg], e4m3x2_to_f16x2(r2 >> 16), e4m3x2_to_f16x2(r3 >> 16));
                 }
-                if (kw + 16 > seg.n_kv) fence_proxy_async_smem();   // generic writes before TMA reuse
             }
+            if (k0 + TILE_N > seg.n_kv) fence_proxy_async_smem();   // generic writes before TMA reuse
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[stage]);
         }
