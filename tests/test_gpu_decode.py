@@ -244,3 +244,34 @@ def test_layer_calls_replay_bit_identically_from_a_cuda_graph():
     assert bd.yoco_xattn_status(ws, side) == 0
     for a, b in zip(eager, Os):
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+def test_calls_on_two_streams_with_their_own_workspaces_do_not_interfere():
+    """Two serving streams, different problems, interleaved calls: each has its own workspace, the
+    plan cache and the launches must keep them apart."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    ws_list, outs, refs, streams = [], [], [], [torch.cuda.Stream(), torch.cuda.Stream()]
+    probs = [si.Workload("s0", B=1, Hq=32, Hkv=8, d=128, T=1, layers=2, seed=71, kv_len=[30000]),
+             si.Workload("s1", B=3, Hq=8, Hkv=2, d=64, T=2, layers=2, seed=72, kv_len=[5000, 77, 1300])]
+    state = []
+    for w in probs:
+        K, V = to_dev_bf16(w.make_k()), to_dev_bf16(w.make_v())
+        Qs = [to_dev_bf16(w.make_q(l).reshape(-1)) for l in range(w.layers)]
+        Os = [torch.empty(w.B * w.Hq * w.T * w.d, dtype=torch.bfloat16, device="cuda") for _ in range(w.layers)]
+        shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(w.kv_len.max()))
+        ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_DECODE), dtype=torch.uint8, device="cuda")
+        state.append((w, K, V, Qs, Os, shape, ws))
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for l in range(2):
+            for (w, K, V, Qs, Os, shape, ws), st in zip(state, streams):
+                bd.yoco_xattn_decode(shape, Qs[l], K, V, w.cu, w.kv_len, Os[l], None, ws, st)
+    torch.cuda.synchronize()
+    for (w, K, V, Qs, Os, shape, ws), st in zip(state, streams):
+        assert bd.yoco_xattn_status(ws, st) == 0
+        for l in range(2):
+            o_ref, _ = oracle.xattn(w.make_q(l), w.make_k(), w.make_v(), w.cu, w.kv_len, B=w.B, Hq=w.Hq, Hkv=w.Hkv,
+                                    d=w.d, T=w.T)
+            got = si.bf16_bits_to_f32(Os[l].view(torch.int16).cpu().numpy().view(np.uint16)).astype(np.float64)
+            assert_close(got.reshape(o_ref.shape), o_ref, f"{w.name} layer {l}")
