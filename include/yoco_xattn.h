@@ -247,6 +247,15 @@ int32_t yoco_kv_append(const yoco_kv_append_shape* shape, const void* X, const v
                        void* K, void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
                        void* stream);
 
+/* The same step writing an 8-bit cache: every new row is divided by its KV head's scale and stored as
+ * FP8 E4M3 bytes (round to nearest even, saturating at +-448) in the byte caches K8, V8 that
+ * yoco_xattn_decode_fp8 reads (same packed layout, one byte per element).  k_scale_host, v_scale_host:
+ * host [Hkv], finite and > 0, chosen by the caller (for instance the largest magnitude expected / 448);
+ * Hkv <= 64.  Otherwise as yoco_kv_append. */
+int32_t yoco_kv_append_fp8(const yoco_kv_append_shape* shape, const void* X, const void* Wgk, const void* Wgv,
+                           void* K8, void* V8, const float* k_scale_host, const float* v_scale_host,
+                           const int32_t* cu_kv_host, const int32_t* kv_len_host, void* stream);
+
 /* Synchronises `stream`; returns YOCO_OK or YOCO_ERR_TIMEOUT if an append kernel on the current
  * device gave up a wait since the last call of this function (which clears the record). */
 int32_t yoco_kv_append_status(void* stream);

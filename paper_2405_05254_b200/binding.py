@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.yoco_xattn_decode_fp8.restype = i32
         L.yoco_kv_fold_gain.argtypes = [i64, i64, vp, vp, vp, vp]
         L.yoco_kv_append.argtypes = [ctypes.POINTER(KvAppendShape), vp, vp, vp, vp, vp, vp, vp, vp]
+        L.yoco_kv_append_fp8.argtypes = [ctypes.POINTER(KvAppendShape), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.yoco_kv_append_fp8.restype = i32
         L.yoco_kv_append_status.argtypes = [vp]
         for name in ("yoco_kv_fold_gain", "yoco_kv_append", "yoco_kv_append_status"):
             getattr(L, name).restype = i32
@@ -222,6 +224,20 @@ def yoco_kv_append(shape: KvAppendShape, X, Wgk, Wgv, K, V, cu_kv, kv_len, strea
                               _stream_ptr(stream))
     if rc != OK:
         raise YocoError(rc, "yoco_kv_append")
+
+
+def yoco_kv_append_fp8(shape: KvAppendShape, X, Wgk, Wgv, K8, V8, k_scale, v_scale, cu_kv, kv_len, stream=None) -> None:
+    """As yoco_kv_append, but the rows are stored as FP8 E4M3 bytes (uint8 caches) after division by the
+    per-head scales (host float32 [Hkv])."""
+    keep_cu, p_cu = _host_i32(cu_kv)
+    keep_len, p_len = _host_i32(kv_len)
+    ks = np.ascontiguousarray(k_scale, dtype=np.float32)
+    vs = np.ascontiguousarray(v_scale, dtype=np.float32)
+    rc = lib().yoco_kv_append_fp8(ctypes.byref(shape), _ptr(X), _ptr(Wgk), _ptr(Wgv), _ptr(K8), _ptr(V8),
+                                  ctypes.c_void_p(ks.ctypes.data), ctypes.c_void_p(vs.ctypes.data), p_cu, p_len,
+                                  _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_kv_append_fp8")
 
 
 def yoco_kv_append_status(stream=None) -> int:

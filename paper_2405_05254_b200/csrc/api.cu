@@ -517,8 +517,10 @@ int32_t yoco_kv_fold_gain(int64_t d_model, int64_t n_out, const void* g, const v
     return YOCO_OK;
 }
 
-int32_t yoco_kv_append(const yoco_kv_append_shape* shape, const void* X, const void* Wgk, const void* Wgv,
-                       void* K, void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host, void* stream) {
+namespace {
+int32_t kv_append_impl(const yoco_kv_append_shape* shape, const void* X, const void* Wgk, const void* Wgv, void* K,
+                       void* V, const float* k_scale_host, const float* v_scale_host, bool fp8,
+                       const int32_t* cu_kv_host, const int32_t* kv_len_host, void* stream) {
     if (!shape) return YOCO_ERR_INVALID_ARG;
     const yoco_kv_append_shape& s = *shape;
     if (s.B < 0 || s.Hkv <= 0 || s.d <= 0 || s.T <= 0 || s.d_model <= 0 || s.kv_head_stride < 0 || !(s.eps >= 0.f))
@@ -565,8 +567,33 @@ int32_t yoco_kv_append(const yoco_kv_append_shape* shape, const void* X, const v
     if ((rc = make_map_2d(&tmX, X, p.M, s.d_model, 128)) != YOCO_OK) return rc;
     if ((rc = make_map_2d(&tmWk, Wgk, s.d_model, p.n_half, 128)) != YOCO_OK) return rc;
     if ((rc = make_map_2d(&tmWv, Wgv, s.d_model, p.n_half, 128)) != YOCO_OK) return rc;
-    YOCO_CUDA_TRY(launch_kv_append(p, tab, tmX, tmWk, tmWv, reinterpret_cast<cudaStream_t>(stream)));
+    KvAppendScales sc{};
+    if (fp8) {
+        if (!k_scale_host || !v_scale_host) return YOCO_ERR_INVALID_ARG;
+        if (s.Hkv > kFp8MaxHeads) return YOCO_ERR_UNSUPPORTED;
+        for (int c = 0; c < s.Hkv; ++c) {
+            if (!(k_scale_host[c] > 0.f) || !(v_scale_host[c] > 0.f) || !std::isfinite(k_scale_host[c]) ||
+                !std::isfinite(v_scale_host[c]))
+                return YOCO_ERR_INVALID_ARG;
+            sc.inv_k[c] = 1.f / k_scale_host[c];
+            sc.inv_v[c] = 1.f / v_scale_host[c];
+        }
+    }
+    YOCO_CUDA_TRY(launch_kv_append(p, tab, tmX, tmWk, tmWv, reinterpret_cast<cudaStream_t>(stream), fp8 ? &sc : nullptr));
     return YOCO_OK;
+}
+}  // namespace
+
+int32_t yoco_kv_append(const yoco_kv_append_shape* shape, const void* X, const void* Wgk, const void* Wgv,
+                       void* K, void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host, void* stream) {
+    return kv_append_impl(shape, X, Wgk, Wgv, K, V, nullptr, nullptr, false, cu_kv_host, kv_len_host, stream);
+}
+
+int32_t yoco_kv_append_fp8(const yoco_kv_append_shape* shape, const void* X, const void* Wgk, const void* Wgv,
+                           void* K8, void* V8, const float* k_scale_host, const float* v_scale_host,
+                           const int32_t* cu_kv_host, const int32_t* kv_len_host, void* stream) {
+    return kv_append_impl(shape, X, Wgk, Wgv, K8, V8, k_scale_host, v_scale_host, true, cu_kv_host, kv_len_host,
+                          stream);
 }
 
 int32_t yoco_kv_append_status(void* stream) {

@@ -139,8 +139,14 @@ struct KvAppendTables {         // per sequence, as kernel parameters
 };
 // tmX: [M, d_model] box {64, 128}; tmWk / tmWv: gain-folded weights [d_model, Hkv*d] box {64, 128};
 // 128-byte swizzle.  Grid = (2*Hkv*d/128, ceil(M/128)).
+struct KvAppendScales {         // 8-bit cache: reciprocal of the per-head scales (value = scale * e4m3(byte))
+    float inv_k[kFp8MaxHeads];
+    float inv_v[kFp8MaxHeads];
+};
+// fp8_scales (host, may be null): store FP8 E4M3 bytes instead of bf16.
 cudaError_t launch_kv_append(const KvAppendParams& p, const KvAppendTables& tab, const CUtensorMap& tmX,
-                             const CUtensorMap& tmWk, const CUtensorMap& tmWv, cudaStream_t stream);
+                             const CUtensorMap& tmWk, const CUtensorMap& tmWv, cudaStream_t stream,
+                             const KvAppendScales* fp8_scales = nullptr);
 cudaError_t launch_fold_gain(const __nv_bfloat16* g, const __nv_bfloat16* W, __nv_bfloat16* Wg, int64_t d_model,
                              int64_t n_out, cudaStream_t stream);
 cudaError_t read_and_clear_kv_append_status(int32_t* word, cudaStream_t stream);

@@ -12,6 +12,8 @@
 // Roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer (whole warp walks, one elected lane
 // issues), warps 2-5 row statistics during the loop, then scale / round to bf16 / scatter.
 // Every wait is bounded and reports through the status word.
+#include <cuda_fp8.h>
+
 #include <algorithm>
 
 #include "kernels.h"
@@ -36,10 +38,13 @@ constexpr int OFF_BAR = STAGES * STAGE_BYTES;
 constexpr int SMEM_BYTES = OFF_BAR + (2 * STAGES + 1) * 8 + 16;
 constexpr uint32_t TMEM_COLS = 128;
 
+// FP8 = false: rows stored as bf16.  FP8 = true: rows divided by the head's scale and stored as FP8
+// E4M3 bytes (round to nearest even, saturating at +-448), one byte per element.
+template <bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmWk,
                  const __grid_constant__ CUtensorMap tmWv, const KvAppendParams p,
-                 const __grid_constant__ KvAppendTables tab) {
+                 const __grid_constant__ KvAppendTables tab, const __grid_constant__ KvAppendScales sc) {
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + OFF_BAR);   // [STAGES] tile pair has landed
     uint64_t* empty = full + STAGES;                                // [STAGES] MMA and row sums are done with it
@@ -169,6 +174,24 @@ kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                     const bool is_v = n >= p.n_half;
                     const int nn = n - (is_v ? p.n_half : 0);
                     const int c = nn / p.d, e = nn - c * p.d;
+                    if (FP8) {
+                        const float rs = r * (is_v ? sc.inv_v[c] : sc.inv_k[c]);
+                        uint8_t* dst8 = reinterpret_cast<uint8_t*>(is_v ? p.V : p.K) + (row0 + (int64_t)c * head_rows) * p.d + e;
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const uint32_t lo = __nv_cvt_float2_to_fp8x2(
+                                    make_float2(o[q * 16 + k * 4 + 0] * rs, o[q * 16 + k * 4 + 1] * rs), __NV_SATFINITE, __NV_E4M3);
+                                const uint32_t hi = __nv_cvt_float2_to_fp8x2(
+                                    make_float2(o[q * 16 + k * 4 + 2] * rs, o[q * 16 + k * 4 + 3] * rs), __NV_SATFINITE, __NV_E4M3);
+                                w[k] = lo | (hi << 16);
+                            }
+                            *reinterpret_cast<uint4*>(dst8 + q * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                        continue;
+                    }
                     __nv_bfloat16* dst = (is_v ? p.V : p.K) + (row0 + (int64_t)c * head_rows) * p.d + e;
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
@@ -217,14 +240,22 @@ cudaError_t read_and_clear_kv_append_status(int32_t* word, cudaStream_t stream) 
 }
 
 cudaError_t kv_append_kernel_setup() {
-    return cudaFuncSetAttribute(kv_append_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(kv_append_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(kv_append_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
 }
 
 cudaError_t launch_kv_append(const KvAppendParams& p, const KvAppendTables& tab, const CUtensorMap& tmX,
-                             const CUtensorMap& tmWk, const CUtensorMap& tmWv, cudaStream_t stream) {
+                             const CUtensorMap& tmWk, const CUtensorMap& tmWv, cudaStream_t stream,
+                             const KvAppendScales* fp8_scales) {
     if (p.M <= 0) return cudaSuccess;
     dim3 grid((unsigned)(2 * p.n_half / BN), (unsigned)((p.M + BM - 1) / BM));
-    kv_append_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(tmX, tmWk, tmWv, p, tab);
+    if (fp8_scales) {
+        kv_append_kernel<true><<<grid, kThreads, SMEM_BYTES, stream>>>(tmX, tmWk, tmWv, p, tab, *fp8_scales);
+    } else {
+        KvAppendScales none{};
+        kv_append_kernel<false><<<grid, kThreads, SMEM_BYTES, stream>>>(tmX, tmWk, tmWv, p, tab, none);
+    }
     return cudaGetLastError();
 }
 

@@ -27,7 +27,7 @@ def test_library_exports_every_declared_symbol():
     assert {"yoco_xattn_decode", "yoco_xattn_chunk", "yoco_xattn_combine", "yoco_xattn_plan",
             "yoco_xattn_workspace_size", "yoco_xattn_status", "yoco_xattn_strerror", "yoco_xattn_decode_partial",
             "yoco_xattn_combine_gathered", "yoco_xattn_decode_fp8", "yoco_kv_append", "yoco_kv_fold_gain",
-            "yoco_kv_append_status"} <= set(syms)
+            "yoco_kv_append_status", "yoco_kv_append_fp8"} <= set(syms)
     for s in syms:
         assert hasattr(L, s), f"{s} is declared in include/ but not exported"
 
