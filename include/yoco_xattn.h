@@ -79,7 +79,8 @@ typedef struct yoco_xattn_shape {
 /* One unit of work: a contiguous key range of one (sequence, KV head) stream,
  * executed by CTA group `group`; its partial result goes to slot `slot`. */
 typedef struct yoco_xattn_segment {
-    int32_t group;      /* CTA group that streams this range                              */
+    int32_t group;      /* work item: CTA group g, or with sub_items > 1 piece r of
+                           group g as r * num_groups + g                                  */
     int32_t b;          /* sequence                                                       */
     int32_t c;          /* KV head                                                        */
     int32_t k_begin;    /* first key (multiple of tile_n)                                 */
@@ -102,6 +103,8 @@ typedef struct yoco_xattn_plan_info {
     int32_t needs_combine;   /* 0 when every stream has exactly one segment               */
     int64_t total_tiles;     /* sum over streams of ceil(N_i / tile_n)                    */
     int64_t workspace_bytes; /* what decode/chunk need for this problem                   */
+    int32_t sub_items;       /* decode: pieces a group's range is cut into (1, 2 or 4)    */
+    int32_t num_slots;       /* partial-result slots the workspace holds                  */
 } yoco_xattn_plan_info;
 
 /* Split-count / tile heuristic (host only, integers only, deterministic).
@@ -109,12 +112,25 @@ typedef struct yoco_xattn_plan_info {
  * num_groups contiguous ranges of equal tile count (+-1); a range that crosses a
  * stream boundary becomes several segments.  num_groups = min(total_tiles,
  * sm_count * groups_per_sm(mode)).  sm_count > 0 must be given (pure host call).
+ * Decode plans whose groups are long (>= 40 tiles) cut every group's range once more, into
+ * sub_items pieces of decreasing size (yoco_xattn_sub_bound): the SMs of a GPU do not all
+ * stream at the same rate, so CTA g runs piece 0 of its own group and the remaining pieces
+ * are handed out, in item order, to whichever CTA is free.  The pieces, their slots and the
+ * merge order are fixed here, so the result is the same whoever runs a piece; segments_out
+ * then lists the pieces.  (yoco_xattn_decode_fp8 and yoco_xattn_decode_static run with
+ * sub_items = 1.)
  * kv_len_host: [B] or NULL (every N_i = shape->max_kv_len).
  * segments_out: optional array of `capacity` entries; at most `capacity` are written,
  * info->num_segments tells how many exist.  */
 int32_t yoco_xattn_plan(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
                         int32_t sm_count, int32_t mode, yoco_xattn_plan_info* info,
                         yoco_xattn_segment* segments_out, int32_t capacity);
+
+/* First tile, counted inside a group of n_tiles key tiles, of piece r of sub_items
+ * (r = 0 .. sub_items; sub_items in {1, 2, 4}): piece r covers tiles [bound(r), bound(r+1))
+ * with bound(r) = n_tiles * c(r) / 64 rounded down, c = 0, 52, 64 for two pieces and
+ * 0, 44, 54, 61, 64 for four.  Returns -1 for other arguments.  Pure host. */
+int64_t yoco_xattn_sub_bound(int64_t n_tiles, int32_t sub_items, int32_t r);
 
 /* Workspace bytes for decode/chunk on this problem.  sm_count = 0 queries the
  * current CUDA device (then YOCO_ERR_CUDA is possible).  Pure host otherwise. */

@@ -39,7 +39,8 @@ class PlanInfo(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("mode", "tile_n", "tile_m", "m_tiles", "num_groups", "num_ctas", "num_streams",
                  "num_segments", "max_splits", "needs_combine")] + \
-               [("total_tiles", ctypes.c_int64), ("workspace_bytes", ctypes.c_int64)]
+               [("total_tiles", ctypes.c_int64), ("workspace_bytes", ctypes.c_int64),
+                ("sub_items", ctypes.c_int32), ("num_slots", ctypes.c_int32)]
 
 
 class YocoError(RuntimeError):
@@ -77,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.yoco_xattn_decode_fp8.restype = i32
         L.yoco_kv_fold_gain.argtypes = [i64, i64, vp, vp, vp, vp]
         L.yoco_kv_append.argtypes = [ctypes.POINTER(KvAppendShape), vp, vp, vp, vp, vp, vp, vp, vp]
+        L.yoco_xattn_sub_bound.argtypes = [ctypes.c_int64, i32, i32]
+        L.yoco_xattn_sub_bound.restype = ctypes.c_int64
         L.yoco_kv_append_fp8.argtypes = [ctypes.POINTER(KvAppendShape), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.yoco_kv_append_fp8.restype = i32
         L.yoco_kv_append_status.argtypes = [vp]
@@ -224,6 +227,10 @@ def yoco_kv_append(shape: KvAppendShape, X, Wgk, Wgv, K, V, cu_kv, kv_len, strea
                               _stream_ptr(stream))
     if rc != OK:
         raise YocoError(rc, "yoco_kv_append")
+
+
+def yoco_xattn_sub_bound(n_tiles: int, sub_items: int, r: int) -> int:
+    return int(lib().yoco_xattn_sub_bound(n_tiles, sub_items, r))
 
 
 def yoco_kv_append_fp8(shape: KvAppendShape, X, Wgk, Wgv, K8, V8, k_scale, v_scale, cu_kv, kv_len, stream=None) -> None:

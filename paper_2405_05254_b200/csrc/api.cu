@@ -61,11 +61,11 @@ int32_t device_state(DeviceState** out) {
 // ---- plan cache ---------------------------------------------------------------------------
 struct PlanKey {
     yoco_xattn_shape shape;
-    int32_t sm_count, mode;
+    int32_t sm_count, mode, max_sub;
     std::vector<int32_t> lens, cu;
     bool operator==(const PlanKey& o) const {
         return std::memcmp(&shape, &o.shape, sizeof shape) == 0 && sm_count == o.sm_count &&
-               mode == o.mode && lens == o.lens && cu == o.cu;
+               mode == o.mode && max_sub == o.max_sub && lens == o.lens && cu == o.cu;
     }
 };
 // A cached plan with the launch-ready forms of its tables.
@@ -86,12 +86,13 @@ constexpr size_t kPlanCacheEntries = 16;
 // Looks the plan up (most recently used first) or makes it.  The shared pointer keeps the entry
 // alive for the caller even if another thread evicts it from the cache meanwhile.
 int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t* lens, int32_t sm_count,
-                    int32_t mode, std::shared_ptr<const ReadyPlan>& out) {
+                    int32_t mode, int32_t max_sub, std::shared_ptr<const ReadyPlan>& out) {
     PlanKey key;
     std::memset(&key.shape, 0, sizeof key.shape);
     key.shape = s;
     key.sm_count = sm_count;
     key.mode = mode;
+    key.max_sub = max_sub;
     if (lens) key.lens.assign(lens, lens + s.B);
     if (cu) key.cu.assign(cu, cu + s.B + 1);
     {
@@ -104,18 +105,18 @@ int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t*
             }
     }
     auto ready = std::make_shared<ReadyPlan>();
-    int32_t rc = make_plan(s, cu, lens, sm_count, mode, ready->plan);
+    int32_t rc = make_plan(s, cu, lens, sm_count, mode, ready->plan, max_sub);
     if (rc != YOCO_OK) return rc;
     const Plan& plan = ready->plan;
     ready->blob.assign(kWorkspaceHeaderBytes / 4 + plan.table.size(), 0);
     std::copy(plan.table.begin(), plan.table.end(), ready->blob.begin() + kWorkspaceHeaderBytes / 4);
-    ready->fits_inline = mode == YOCO_MODE_DECODE && plan.info.num_segments <= kInlineSegments &&
+    ready->fits_inline = mode == YOCO_MODE_DECODE && plan.coarse_segments <= kInlineSegments &&
                          plan.info.num_groups <= kInlineGroups && plan.info.num_streams <= kInlineStreams;
     if (ready->fits_inline) {
         std::memset(&ready->decode_tab, 0, sizeof ready->decode_tab);
         std::memset(&ready->combine_tab, 0, sizeof ready->combine_tab);
         std::memcpy(ready->decode_tab.seg, plan.table.data() + plan.off_segments,
-                    (size_t)plan.info.num_segments * sizeof(DevSegment));
+                    (size_t)plan.coarse_segments * sizeof(DevSegment));
         std::memcpy(ready->decode_tab.group_begin, plan.table.data() + plan.off_group_begin,
                     (size_t)(plan.info.num_groups + 1) * 4);
         std::memcpy(ready->combine_tab.stream_base, plan.table.data() + plan.off_stream_base,
@@ -212,7 +213,7 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const void* K, const void* V,
             const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
             void* workspace, size_t workspace_bytes, void* stream_v, float* part_out = nullptr,
-            const Fp8Scales* fp8 = nullptr) {
+            const Fp8Scales* fp8 = nullptr, int32_t max_sub = kMaxSubItems) {
     // part_out != null: the result is a partial one (fp32 rows + their LSE in `lse`, no bf16 O)
     if (!shape) return YOCO_ERR_INVALID_ARG;
     int32_t rc = validate_shape(*shape, mode);
@@ -228,7 +229,10 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
     if ((rc = device_state(&dev)) != YOCO_OK) return rc;
 
     std::shared_ptr<const ReadyPlan> ready;
-    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, mode, ready)) != YOCO_OK)
+    // The 8-bit kernel runs one piece per group: it is paced by its own instruction chains, evenly
+    // on every SM, and handing out pieces made it slower (351 us against 331 us at 1M keys).
+    if (fp8) max_sub = 1;
+    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, mode, max_sub, ready)) != YOCO_OK)
         return rc;
     const Plan& plan = ready->plan;
     if ((int64_t)workspace_bytes < plan.info.workspace_bytes) return YOCO_ERR_WORKSPACE_TOO_SMALL;
@@ -280,6 +284,8 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             p.d = shape->d;
             p.window = shape->window;
             p.force_partial = part_out ? 1 : 0;
+            p.sub_items = plan.sub_items;
+            p.work_counter = reinterpret_cast<int32_t*>(ws + kWorkCounterOffset);
             if (fp8) {
                 DecodeFp8Params p8{};
                 p8.base = p;
@@ -334,6 +340,7 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
         c.T = shape->T;
         c.rows_per_stream = plan.rows_per_stream;
         c.max_pieces = plan.info.max_splits;
+        c.sub_items = plan.sub_items;
         c.stream_base = table + plan.off_stream_base;
         c.stream_nseg = table + plan.off_stream_nseg;
         c.part_o = part_o;
@@ -393,6 +400,11 @@ int32_t yoco_xattn_plan(const yoco_xattn_shape* shape, const int32_t* kv_len_hos
     return YOCO_OK;
 }
 
+int64_t yoco_xattn_sub_bound(int64_t n_tiles, int32_t sub_items, int32_t r) {
+    if (n_tiles < 0 || (sub_items != 1 && sub_items != 2 && sub_items != 4)) return -1;
+    return sub_bound(n_tiles, sub_items, r);
+}
+
 int32_t yoco_xattn_workspace_size(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
                                   int32_t sm_count, int32_t mode, size_t* bytes) {
     if (!shape || !bytes || sm_count < 0) return YOCO_ERR_INVALID_ARG;
@@ -427,14 +439,15 @@ int32_t yoco_xattn_decode_static(const yoco_xattn_shape* shape, const void* Q, c
     // size check first, on the host: nothing is enqueued for a problem that does not fit
     DeviceState* dev = nullptr;
     if ((rc = device_state(&dev)) != YOCO_OK) return rc;
+    // one piece per group: the fixed buffer is sized for that
     std::shared_ptr<const ReadyPlan> ready;
-    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, YOCO_MODE_DECODE, ready)) != YOCO_OK)
+    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, YOCO_MODE_DECODE, 1, ready)) != YOCO_OK)
         return rc;
     if ((size_t)ready->plan.info.workspace_bytes > kStaticScratchBytes) return YOCO_ERR_STATIC_SCRATCH_EXCEEDED;
     void* scratch = nullptr;
     if ((rc = static_scratch_address(&scratch)) != YOCO_OK) return rc;
     return run(shape, YOCO_MODE_DECODE, Q, K, V, cu_kv_host, kv_len_host, O, lse, scratch,
-               kStaticScratchBytes, stream);
+               kStaticScratchBytes, stream, nullptr, nullptr, 1);
 }
 
 int32_t yoco_xattn_static_scratch_bytes(void) { return (int32_t)kStaticScratchBytes; }

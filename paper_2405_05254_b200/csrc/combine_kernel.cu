@@ -3,25 +3,29 @@
 //   lse = log sum_s exp(lse_s),   O = sum_s exp(lse_s - lse) * O_s
 //
 // Lanes cover the head dimension with 128-bit loads.  With few pieces per row one warp merges a
-// row; with many (a long sequence cut into dozens of splits) the four warps of a CTA share the
-// pieces of one row, and the loop carries no load-to-branch dependence, so that several pieces are
-// in flight at once: the merge is a chain of dependent memory latencies otherwise.
+// row; with many (a long sequence cut into dozens or hundreds of pieces) the 4 or 32 warps of a
+// CTA share the pieces of one row, and the loop carries no load-to-branch dependence, so that
+// several pieces are in flight at once: the merge is a chain of dependent memory latencies
+// otherwise, and its length is what the launch shape is chosen to bound.
 #include "kernels.h"
 
 namespace yoco {
 
 namespace {
 
-constexpr int kCombineWarps = 4;
+constexpr int kCombineWarps = 4;       // warps per CTA of the small shapes
+constexpr int kCombineWarpsMany = 32;  // one 1024-thread CTA per row when a row has very many pieces
+constexpr int kManyPieces = 64;
 
-template <int WPR>   // warps per output row: 1 or kCombineWarps
+// WPR: warps per output row (1 or WARPS); WARPS: warps per CTA
+template <int WPR, int WARPS>
 __device__ __forceinline__ void combine_body(const CombineParams& p) {
     // When launched behind the attention kernel with programmatic stream serialisation, this
     // grid may start before that kernel has finished: wait for it (and for its writes) here.
     // Without that launch attribute the instruction returns at once.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t row = WPR == 1 ? (int64_t)blockIdx.x * kCombineWarps + warp : (int64_t)blockIdx.x;
+    const int64_t row = WPR == 1 ? (int64_t)blockIdx.x * WARPS + warp : (int64_t)blockIdx.x;
     const int sub = WPR == 1 ? 0 : warp;
     if (row >= p.rows) return;
 
@@ -36,8 +40,10 @@ __device__ __forceinline__ void combine_body(const CombineParams& p) {
         const int G = p.Hq / p.Hkv;
         const int stream = b * p.Hkv + h / G;
         const int r_local = (h % G) * p.T + t;
-        const int slot0 = p.stream_base[stream];
-        nseg = p.stream_nseg[stream];
+        // every table entry stands for sub_items consecutive slots (the pieces of one segment)
+        const int per = p.sub_items > 1 ? p.sub_items : 1;
+        const int slot0 = p.stream_base[stream] * per;
+        nseg = p.stream_nseg[stream] * per;
         // an unsplit stream: the attention kernel wrote the final rows itself (unless told not to)
         if (nseg == 1 && !p.merge_unsplit) return;
         o_base = ((int64_t)slot0 * p.rows_per_stream + r_local) * p.d;
@@ -106,7 +112,7 @@ __device__ __forceinline__ void combine_body(const CombineParams& p) {
         }
     }
     if (WPR > 1) {
-        __shared__ float4 red[kCombineWarps][2][32];
+        __shared__ float4 red[WARPS][2][32];
         red[warp][0][lane] = acc[0];
         red[warp][1][lane] = acc[1];
         __syncthreads();
@@ -115,7 +121,7 @@ __device__ __forceinline__ void combine_body(const CombineParams& p) {
         for (int blk = 0; blk < 2; ++blk) {
             float4 t = red[0][blk][lane];
 #pragma unroll
-            for (int w2 = 1; w2 < kCombineWarps; ++w2) {
+            for (int w2 = 1; w2 < WARPS; ++w2) {
                 const float4 u = red[w2][blk][lane];
                 t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
             }
@@ -137,17 +143,17 @@ __device__ __forceinline__ void combine_body(const CombineParams& p) {
     if (p.lse && lane == 0) p.lse[row] = m + __logf(denom);
 }
 
-template <int WPR>
-__global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const CombineParams p) { combine_body<WPR>(p); }
+template <int WPR, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32) combine_kernel(const CombineParams p) { combine_body<WPR, WARPS>(p); }
 
 // stream tables as kernel parameters
-template <int WPR>
-__global__ void __launch_bounds__(kCombineWarps * 32)
+template <int WPR, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32)
 combine_kernel_inline(const CombineParams p0, const __grid_constant__ CombineInlineTables tab) {
     CombineParams p = p0;
     p.stream_base = tab.stream_base;
     p.stream_nseg = tab.stream_nseg;
-    combine_body<WPR>(p);
+    combine_body<WPR, WARPS>(p);
 }
 
 }  // namespace
@@ -155,11 +161,13 @@ combine_kernel_inline(const CombineParams p0, const __grid_constant__ CombineInl
 cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream, const CombineInlineTables* inline_tab,
                            bool after_attention) {
     if (p.rows == 0) return cudaSuccess;
-    const bool wide = p.max_pieces > kCombineWarps;      // many pieces per row: one CTA per row
-    const int64_t blocks = wide ? p.rows : (p.rows + kCombineWarps - 1) / kCombineWarps;
+    // pieces per row -> shape: a warp per row; a 4-warp CTA per row; a 32-warp CTA per row
+    const int shape = p.max_pieces > kManyPieces ? 2 : p.max_pieces > kCombineWarps ? 1 : 0;
+    const int warps = shape == 2 ? kCombineWarpsMany : kCombineWarps;
+    const int64_t blocks = shape ? p.rows : (p.rows + kCombineWarps - 1) / kCombineWarps;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks);
-    cfg.blockDim = dim3(kCombineWarps * 32);
+    cfg.blockDim = dim3(warps * 32);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -167,11 +175,15 @@ cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream, const Co
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = after_attention ? 1 : 0;
-    if (inline_tab)
-        return wide ? cudaLaunchKernelEx(&cfg, combine_kernel_inline<kCombineWarps>, p, *inline_tab)
-                    : cudaLaunchKernelEx(&cfg, combine_kernel_inline<1>, p, *inline_tab);
-    return wide ? cudaLaunchKernelEx(&cfg, combine_kernel<kCombineWarps>, p)
-                : cudaLaunchKernelEx(&cfg, combine_kernel<1>, p);
+    if (inline_tab) {
+        if (shape == 2)
+            return cudaLaunchKernelEx(&cfg, combine_kernel_inline<kCombineWarpsMany, kCombineWarpsMany>, p, *inline_tab);
+        if (shape == 1) return cudaLaunchKernelEx(&cfg, combine_kernel_inline<kCombineWarps, kCombineWarps>, p, *inline_tab);
+        return cudaLaunchKernelEx(&cfg, combine_kernel_inline<1, kCombineWarps>, p, *inline_tab);
+    }
+    if (shape == 2) return cudaLaunchKernelEx(&cfg, combine_kernel<kCombineWarpsMany, kCombineWarpsMany>, p);
+    if (shape == 1) return cudaLaunchKernelEx(&cfg, combine_kernel<kCombineWarps, kCombineWarps>, p);
+    return cudaLaunchKernelEx(&cfg, combine_kernel<1, kCombineWarps>, p);
 }
 
 }  // namespace yoco

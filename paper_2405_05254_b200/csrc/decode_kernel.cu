@@ -10,6 +10,13 @@
 // bound by HBM bandwidth; the small matrix products go through mma.sync (bf16 in, fp32
 // accumulate) only to keep the issue slots free for the memory pipeline.
 // Row max / row sum use warp shuffles inside each quad of lanes.
+//
+// Work items: with p.sub_items = R > 1 every group's range is cut into R pieces (plan.h:
+// sub_bound).  CTA g starts with piece 0 of group g; when its producer has issued the last
+// load of an item it takes the next unclaimed one from a global counter and tells the consumer
+// warps through a two-entry queue in shared memory, so the tile ring never drains between
+// items.  Fast SMs thereby take more pieces than slow ones; what a piece computes and where
+// its partial result goes is fixed by the plan.
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -33,7 +40,9 @@ struct Cfg {
     static constexpr int BUDGET = 113 * 1024;
     static constexpr int STAGES_FIT = (BUDGET - MERGE_O_BYTES - MERGE_ML_BYTES - 128) / STAGE_BYTES;
     static constexpr int STAGES = STAGES_FIT > 4 ? 4 : STAGES_FIT;
+    // + ring barriers (<= 64 B), item-queue barriers (32 B), queue entries and give-up flag
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + MERGE_O_BYTES + MERGE_ML_BYTES + 128;
+    static_assert(2 * STAGES * 8 + 4 * 8 + 4 * 4 <= 128, "barrier block");
     static_assert(STAGES >= 2, "need at least a double buffer");
 };
 
@@ -56,9 +65,15 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * C::STAGE_BYTES +
                                                      C::MERGE_O_BYTES + C::MERGE_ML_BYTES);
     uint64_t* empty_bar = full_bar + STAGES;
+    uint64_t* item_full = empty_bar + STAGES;      // [2] producer -> consumers: entry written
+    uint64_t* item_empty = item_full + 2;          // [2] consumers -> producer: entry read
+    volatile int32_t* item_q = reinterpret_cast<volatile int32_t*>(item_empty + 2);   // [2] item ids
+    volatile int32_t* give_up = item_q + 2;        // a consumer warp ran out of patience
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int seg_lo = p.group_begin[blockIdx.x], seg_hi = p.group_begin[blockIdx.x + 1];
+    const int R = p.sub_items > 1 ? p.sub_items : 1;
+    const int n_groups = (int)gridDim.x;
+    const int n_items = n_groups * R;
     // lets a merge kernel queued behind this one be launched early; it still waits for this
     // grid to finish before it reads anything
     asm volatile("griddepcontrol.launch_dependents;");
@@ -72,6 +87,11 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kConsumerWarps);
         }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&item_full[s], 1);
+            mbar_init(&item_empty[s], kConsumerWarps);
+        }
+        *give_up = 0;
         mbar_fence_init();
     }
     __syncthreads();
@@ -83,25 +103,54 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
             tma_prefetch_desc(&tmV);
             uint32_t it = 0;
             bool ok = true;
-            for (int si = seg_lo; si < seg_hi && ok; ++si) {
-                const DevSegment seg = p.segments[si];
-                for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += TILE_N, ++it) {
-                    const uint32_t stage = it % STAGES, round = it / STAGES;
-                    if (!mbar_wait(&empty_bar[stage], (round & 1u) ^ 1u)) {
-                        atomicExch(p.status, kStatusTimeout);
-                        ok = false;
-                        break;
-                    }
-                    uint8_t* kdst = stage_mem + stage * C::STAGE_BYTES;
-                    uint8_t* vdst = kdst + C::TENSOR_BYTES;
-                    mbar_expect_tx(&full_bar[stage], C::STAGE_BYTES);
-                    const int row = seg.kv_row0 + (k0 - seg.k_begin);
+            int item = blockIdx.x;
+            for (uint32_t n = 0; ok; ++n) {
+                // hand the item (or the end mark) to the consumers
+                if (!mbar_wait(&item_empty[n & 1u], ((n >> 1) & 1u) ^ 1u)) {
+                    atomicExch(p.status, kStatusTimeout);
+                    break;
+                }
+                item_q[n & 1u] = item;
+                mbar_arrive(&item_full[n & 1u]);
+                if (item >= n_items) break;
+                const int grp = item % n_groups, piece = item / n_groups;
+                const int seg_lo = p.group_begin[grp], seg_hi = p.group_begin[grp + 1];
+                int t_lo = 0, t_hi = 0x7fffffff, acc = 0;       // the piece's tiles inside the group
+                if (R > 1) {
+                    int n_g = 0;
+                    for (int si = seg_lo; si < seg_hi; ++si)
+                        n_g += (p.segments[si].k_end - p.segments[si].k_begin + TILE_N - 1) / TILE_N;
+                    t_lo = (int)sub_bound(n_g, R, piece);
+                    t_hi = (int)sub_bound(n_g, R, piece + 1);
+                }
+                for (int si = seg_lo; si < seg_hi && ok; ++si) {
+                    const DevSegment seg = p.segments[si];
+                    const int nt = (seg.k_end - seg.k_begin + TILE_N - 1) / TILE_N;
+                    const int s_lo = max(t_lo - acc, 0), s_hi = min(t_hi - acc, nt);
+                    acc += nt;
+                    if (s_lo >= s_hi) continue;
+                    const int k_lo = seg.k_begin + s_lo * TILE_N;
+                    const int k_hi = min(seg.k_begin + s_hi * TILE_N, seg.k_end);
+                    for (int k0 = k_lo; k0 < k_hi; k0 += TILE_N, ++it) {
+                        const uint32_t stage = it % STAGES, round = it / STAGES;
+                        if (!mbar_wait(&empty_bar[stage], (round & 1u) ^ 1u)) {
+                            atomicExch(p.status, kStatusTimeout);
+                            ok = false;
+                            break;
+                        }
+                        uint8_t* kdst = stage_mem + stage * C::STAGE_BYTES;
+                        uint8_t* vdst = kdst + C::TENSOR_BYTES;
+                        mbar_expect_tx(&full_bar[stage], C::STAGE_BYTES);
+                        const int row = seg.kv_row0 + (k0 - seg.k_begin);
 #pragma unroll
-                    for (int h = 0; h < C::HALVES; ++h) {
-                        tma_load_2d(kdst + h * HALF_BYTES, &tmK, h * 64, row, &full_bar[stage]);
-                        tma_load_2d(vdst + h * HALF_BYTES, &tmV, h * 64, row, &full_bar[stage]);
+                        for (int h = 0; h < C::HALVES; ++h) {
+                            tma_load_2d(kdst + h * HALF_BYTES, &tmK, h * 64, row, &full_bar[stage]);
+                            tma_load_2d(vdst + h * HALF_BYTES, &tmV, h * 64, row, &full_bar[stage]);
+                        }
                     }
                 }
+                // all loads of this item are on their way: claim the next one
+                item = R > 1 ? n_groups + atomicAdd(p.work_counter, 1) : n_items;
             }
         }
         return;
@@ -113,8 +162,42 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
     uint32_t it = 0;
     bool ok = true;
 
+    for (uint32_t n_item = 0;; ++n_item) {
+    // the next item from the producer; the four warps must take the same decision, so a warp
+    // that gives up waiting says so before the barrier and all of them leave together
+    if (!mbar_wait(&item_full[n_item & 1u], (n_item >> 1) & 1u)) {
+        atomicExch(p.status, kStatusTimeout);
+        *give_up = 1;
+    }
+    const int item = item_q[n_item & 1u];
+    named_barrier_sync(1, kConsumerWarps * 32);
+    if (*give_up) break;
+    if (lane == 0) mbar_arrive(&item_empty[n_item & 1u]);
+    if (item >= n_items) break;
+    const int grp = item % n_groups, piece = item / n_groups;
+    const int seg_lo = p.group_begin[grp], seg_hi = p.group_begin[grp + 1];
+    int t_lo = 0, t_hi = 0x7fffffff, t_acc = 0;       // the piece's tiles inside the group
+    if (R > 1) {
+        int n_g = 0;
+        for (int si = seg_lo; si < seg_hi; ++si)
+            n_g += (p.segments[si].k_end - p.segments[si].k_begin + TILE_N - 1) / TILE_N;
+        t_lo = (int)sub_bound(n_g, R, piece);
+        t_hi = (int)sub_bound(n_g, R, piece + 1);
+    }
+
     for (int si = seg_lo; si < seg_hi; ++si) {
         const DevSegment seg = p.segments[si];
+        const int seg_tiles = (seg.k_end - seg.k_begin + TILE_N - 1) / TILE_N;
+        const int s_lo = max(t_lo - t_acc, 0), s_hi = min(t_hi - t_acc, seg_tiles);
+        t_acc += seg_tiles;
+        const int slot = seg.slot * R + piece;
+        if (s_lo >= s_hi) {
+            // this piece holds nothing of the segment: its slot must say so to the merge
+            if (R > 1 && threadIdx.x < n_rows) p.part_lse[(int64_t)slot * n_rows + threadIdx.x] = -INFINITY;
+            continue;
+        }
+        const int k_lo = seg.k_begin + s_lo * TILE_N;
+        const int k_hi = min(seg.k_begin + s_hi * TILE_N, seg.k_end);
 
         // Q as the A operand of m16n8k16: rows = (head in group, t), zero beyond n_rows
         uint32_t qa[KSTEPS][4];
@@ -140,7 +223,7 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
 #pragma unroll
         for (int nt = 0; nt < NT_O; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
 
-        for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += TILE_N, ++it) {
+        for (int k0 = k_lo; k0 < k_hi; k0 += TILE_N, ++it) {
             if (!ok) continue;
             const uint32_t stage = it % STAGES, round = it / STAGES;
             if (!mbar_wait(&full_bar[stage], round & 1u)) {
@@ -149,7 +232,7 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
                 continue;
             }
             const int kw = k0 + warp * 16;          // first key of this warp's slice
-            if (kw < seg.k_end) {
+            if (kw < k_hi) {
                 const uint32_t kbase = smem_u32(stage_mem + stage * C::STAGE_BYTES);
                 const uint32_t vbase = kbase + C::TENSOR_BYTES;
 
@@ -297,7 +380,7 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
             }
         }
         named_barrier_sync(1, kConsumerWarps * 32);
-        const bool final_out = seg.stream_nseg == 1 && !p.force_partial;
+        const bool final_out = seg.stream_nseg == 1 && !p.force_partial && R == 1;
         for (int idx = threadIdx.x; idx < n_rows * D; idx += kConsumerWarps * 32) {
             const int r = idx / D, col = idx - r * D;
             float M = -INFINITY;
@@ -318,11 +401,12 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
                 p.O[((int64_t)seg.q_row0 + r) * D + col] = __float2bfloat16(outv);
                 if (p.lse && col == 0) p.lse[seg.q_row0 + r] = lse;
             } else {
-                p.part_o[((int64_t)seg.slot * n_rows + r) * D + col] = outv;
-                if (col == 0) p.part_lse[(int64_t)seg.slot * n_rows + r] = lse;
+                p.part_o[((int64_t)slot * n_rows + r) * D + col] = outv;
+                if (col == 0) p.part_lse[(int64_t)slot * n_rows + r] = lse;
             }
         }
         named_barrier_sync(1, kConsumerWarps * 32);
+    }
     }
 }
 

@@ -36,6 +36,7 @@ struct CombineParams {
     // internal slot-major layout
     int32_t Hq, Hkv, T, rows_per_stream;
     int32_t max_pieces;         // most pieces any row has (S, or the plan's max_splits): picks the launch shape
+    int32_t sub_items;          // internal layout: slots per table entry (0 or 1: one)
     const int32_t* stream_base; // [B*Hkv] first slot of each stream
     const int32_t* stream_nseg; // [B*Hkv] slots of each stream
     const float* part_o;
@@ -71,6 +72,8 @@ struct DecodeParams {
     int32_t d;
     int32_t window;             // sliding window C, 0 = none
     int32_t force_partial;      // write every segment to its partial slot, even of an unsplit stream
+    int32_t sub_items;          // pieces per group (plan.h: sub_bound); slot = segment slot * sub_items + piece
+    int32_t* work_counter;      // zeroed before the launch; hands out the pieces beyond each CTA's first
 };
 // tmK / tmV: 2-D tensor maps over the [rows, d] view of K and V, box {64, kDecodeTileN},
 // 128-byte swizzle.

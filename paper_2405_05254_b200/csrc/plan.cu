@@ -20,7 +20,7 @@ int32_t validate_shape(const yoco_xattn_shape& s, int32_t mode) {
 }
 
 int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const int32_t* kv_len_host,
-                  int32_t sm_count, int32_t mode, Plan& plan) {
+                  int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items) {
     int32_t rc = validate_shape(s, mode);
     if (rc != YOCO_OK) return rc;
     if (sm_count <= 0) return YOCO_ERR_INVALID_ARG;
@@ -111,9 +111,10 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
             flat += nt - t0;
         }
     }
-    int32_t max_splits = 0, needs_combine = 0;
+    const int R = mode == YOCO_MODE_DECODE ? choose_sub_items(total_tiles / num_groups, max_sub_items) : 1;
+    int32_t max_splits = 0, needs_combine = R > 1 ? 1 : 0;
     for (int st = 0; st < num_streams; ++st) {
-        max_splits = std::max(max_splits, stream_nseg[st]);
+        max_splits = std::max(max_splits, stream_nseg[st] * R);
         if (stream_nseg[st] != 1) needs_combine = 1;
     }
     for (auto& d : dev) d.stream_nseg = stream_nseg[d.stream];
@@ -126,6 +127,36 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
         }
         group_begin[num_groups] = (int32_t)k;
     }
+
+    // With R > 1 the public list names the pieces that are executed: piece r of group g is work
+    // item r * num_groups + g and fills slot (segment index) * R + r.  Same walk as the kernel's.
+    if (R > 1) {
+        std::vector<yoco_xattn_segment> pieces;
+        for (int64_t p = 0; p < num_groups; ++p) {
+            int64_t n_g = 0;
+            for (int32_t k = group_begin[p]; k < group_begin[p + 1]; ++k)
+                n_g += (dev[k].k_end - dev[k].k_begin + tile_n - 1) / tile_n;
+            int64_t acc = 0;
+            for (int32_t k = group_begin[p]; k < group_begin[p + 1]; ++k) {
+                const int64_t nt = (dev[k].k_end - dev[k].k_begin + tile_n - 1) / tile_n;
+                for (int r = 0; r < R; ++r) {
+                    const int64_t lo = std::max<int64_t>(sub_bound(n_g, R, r) - acc, 0);
+                    const int64_t hi = std::min<int64_t>(sub_bound(n_g, R, r + 1) - acc, nt);
+                    if (lo >= hi) continue;
+                    yoco_xattn_segment pub = plan.segments[k];
+                    pub.group = (int32_t)(r * num_groups + p);
+                    pub.k_begin = (int32_t)(dev[k].k_begin + lo * tile_n);
+                    pub.k_end = (int32_t)std::min<int64_t>(dev[k].k_begin + hi * tile_n, dev[k].k_end);
+                    pub.slot = dev[k].slot * R + r;
+                    pieces.push_back(pub);
+                }
+                acc += nt;
+            }
+        }
+        plan.segments.swap(pieces);
+    }
+    plan.sub_items = R;
+    plan.coarse_segments = (int32_t)dev.size();
 
     // device blob
     plan.off_segments = 0;
@@ -145,8 +176,9 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     auto align256 = [](int64_t x) { return (x + 255) / 256 * 256; };
     plan.ws_table = kWorkspaceHeaderBytes;
     plan.ws_part_lse = align256(plan.ws_table + (int64_t)plan.table.size() * 4);
-    plan.ws_part_o = align256(plan.ws_part_lse + (int64_t)dev.size() * rows_per_stream * 4);
-    const int64_t ws_end = align256(plan.ws_part_o + (int64_t)dev.size() * rows_per_stream * s.d * 4);
+    const int64_t slots = (int64_t)dev.size() * R;
+    plan.ws_part_o = align256(plan.ws_part_lse + slots * rows_per_stream * 4);
+    const int64_t ws_end = align256(plan.ws_part_o + slots * rows_per_stream * s.d * 4);
 
     yoco_xattn_plan_info& info = plan.info;
     info.mode = mode;
@@ -156,7 +188,9 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     info.num_groups = (int32_t)num_groups;
     info.num_ctas = (int32_t)(num_groups * m_tiles);
     info.num_streams = num_streams;
-    info.num_segments = (int32_t)dev.size();
+    info.num_segments = (int32_t)plan.segments.size();
+    info.sub_items = R;
+    info.num_slots = (int32_t)slots;
     info.max_splits = max_splits;
     info.needs_combine = needs_combine;
     info.total_tiles = total_tiles;

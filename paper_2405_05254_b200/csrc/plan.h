@@ -22,6 +22,40 @@ constexpr int kChunkTileM = 128;      // query rows per tcgen05 tile
 constexpr int kChunkPairTileM = 256;  // rows per CTA when a stream has more than 128 rows: two tiles
                                       // that share every K/V tile in shared memory
 constexpr int kWorkspaceHeaderBytes = 256;
+constexpr int kWorkCounterOffset = 64;  // byte offset of the decode kernel's work counter in the header
+
+// ---- pieces of a decode group ---------------------------------------------------------------
+// SMs do not all stream at the same rate (their share of the memory fabric differs with their
+// place on the die), so equal static shares leave the fast ones idle at the end.  With R > 1 a
+// group's tile range is cut into R pieces of decreasing size; piece 0 is taken by the group's own
+// CTA, the rest are handed out in order to whichever CTA is free.  The pieces are fixed by the plan
+// (integers only), so the result does not depend on who ran what.
+constexpr int kMaxSubItems = 4;
+
+#ifdef __CUDACC__
+#define YOCO_HD __host__ __device__
+#else
+#define YOCO_HD
+#endif
+// First tile (inside a group of n tiles) of piece r of R, r = 0..R; R in {1, 2, 4}.
+YOCO_HD inline int64_t sub_bound(int64_t n, int R, int r) {
+    // cumulative shares in 64ths: a large first piece, then smaller and smaller ones
+    const unsigned c4 = 0x403D362Cu;                       // 44 54 61 64
+    if (r <= 0) return 0;
+    if (r >= R) return n;
+    const int c = R == 4 ? (int)((c4 >> (8 * (r - 1))) & 0xFF) : 52;   // R == 2: 52 | 12
+    return n * c / 64;
+}
+#undef YOCO_HD
+
+// Pieces per group for a decode plan whose groups hold `tiles_per_group` key tiles on average.
+// (Measured on B200, 32 query heads over 8 KV heads: two pieces pay from 128K keys per sequence,
+// four from 256K; eight gained nothing over four at 1M and made the merge longer.)
+inline int choose_sub_items(int64_t tiles_per_group, int max_sub) {
+    int R = tiles_per_group >= 96 ? 4 : tiles_per_group >= 40 ? 2 : 1;
+    while (R > max_sub) R /= 2;
+    return R < 1 ? 1 : R;
+}
 
 // One work segment as the kernels read it (8 x int32 = 32 bytes).
 struct DevSegment {
@@ -45,11 +79,15 @@ struct Plan {
     int64_t ws_table = 0, ws_part_lse = 0, ws_part_o = 0;
     int64_t kv_rows_extent = 0;                  // rows of the [rows, d] K/V view that may be touched
     int32_t rows_per_stream = 0;                 // G * T
+    int32_t sub_items = 1;                       // pieces per group (decode), see sub_bound
+    int32_t coarse_segments = 0;                 // entries of the device segment table; partial slots
+                                                 // = coarse_segments * sub_items
 };
 
 // Returns YOCO_OK or an error code; fills `plan`.  cu_kv_host may be null (tight packing).
+// max_sub_items: upper limit of pieces per decode group (1 = every group is one piece).
 int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const int32_t* kv_len_host,
-                  int32_t sm_count, int32_t mode, Plan& plan);
+                  int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items = kMaxSubItems);
 
 int32_t validate_shape(const yoco_xattn_shape& s, int32_t mode);
 

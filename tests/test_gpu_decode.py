@@ -275,3 +275,57 @@ def test_calls_on_two_streams_with_their_own_workspaces_do_not_interfere():
                                     d=w.d, T=w.T)
             got = si.bf16_bits_to_f32(Os[l].view(torch.int16).cpu().numpy().view(np.uint16)).astype(np.float64)
             assert_close(got.reshape(o_ref.shape), o_ref, f"{w.name} layer {l}")
+
+
+def test_long_ragged_batch_runs_its_groups_in_pieces():
+    """Sequences long enough for the plan to cut every group into pieces, with lengths chosen so
+    that groups straddle stream boundaries (a piece then holds nothing of one of its group's
+    segments and must mark that slot empty).  All rows against the oracle, and the plan says what ran."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    lens = np.array([200001, 130000, 70003], dtype=np.int32)
+    w = si.Workload("pieces", B=3, Hq=8, Hkv=2, d=128, T=1, layers=1, seed=21, kv_len=lens)
+    sm = torch.cuda.get_device_properties(0).multi_processor_count
+    info, segs = bd.yoco_xattn_plan(bd.make_shape(w.B, w.Hq, w.Hkv, w.d, 1), lens, sm, bd.MODE_DECODE)
+    assert info.sub_items == 2 or info.sub_items == 4
+    assert info.num_segments < info.num_slots          # some piece is empty for some segment
+    K, V, Q = w.make_k(), w.make_v(), w.make_q(0)
+    r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, 1, lens, K, V)
+    o, lse, _ = r.run(Q)
+    o_ref, lse_ref = oracle.xattn(Q, K, V, w.cu, lens, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=1)
+    assert_close(o, o_ref, "pieces")
+    assert_lse_close(lse, lse_ref, "pieces")
+
+
+def test_pieces_give_the_same_bits_whoever_runs_them():
+    """Which CTA runs a piece depends on timing; the result must not.  The same call repeated, alone
+    and while another stream keeps the SMs busy with a second problem, is bit-identical every time."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    w = si.Workload("pieces2", B=1, Hq=32, Hkv=8, d=128, T=1, layers=1, seed=22, kv_len=[300000])
+    K, V, Q = w.make_k(), w.make_v(), w.make_q(0)
+    r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, 1, w.kv_len, K, V)
+    sm = torch.cuda.get_device_properties(0).multi_processor_count
+    info, _ = bd.yoco_xattn_plan(r.shape, w.kv_len, sm, bd.MODE_DECODE)
+    assert info.sub_items == 4
+    o0, lse0, O = r.run(Q)
+    ref_bits, ref_lse = O.view(torch.int16).clone(), lse0.copy()
+    o_ref, lse_ref = oracle.xattn(Q, K, V, w.cu, w.kv_len, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=1)
+    assert_close(o0, o_ref, "four pieces")
+    assert_lse_close(lse0, lse_ref, "four pieces")
+    # a second, smaller problem on another stream perturbs who is free when
+    w2 = si.Workload("noise", B=4, Hq=8, Hkv=8, d=128, T=1, layers=1, seed=23, kv_len=[9000, 14000, 300, 7000])
+    r2 = GpuRunner(w2.B, w2.Hq, w2.Hkv, w2.d, 1, w2.kv_len, w2.make_k(), w2.make_v())
+    O2, L2, W2 = r2._buffers(bd.MODE_DECODE)
+    Q2 = to_dev_bf16(w2.make_q(0).reshape(-1))
+    side = torch.cuda.Stream()
+    for rep in range(6):
+        if rep >= 2:
+            with torch.cuda.stream(side):
+                for _ in range(8):
+                    bd.yoco_xattn_decode(r2.shape, Q2, r2.K, r2.V, None, w2.kv_len, O2, L2, W2, stream=side)
+        o, lse, O = r.run(Q)
+        assert torch.equal(O.view(torch.int16), ref_bits), f"repeat {rep} differs"
+        assert np.array_equal(lse, ref_lse)
+    torch.cuda.synchronize()
+    assert bd.yoco_xattn_status(W2) == 0

@@ -58,7 +58,44 @@ def restated_plan(B, Hkv, lens, sm_count, mode, G, T):
                 if a < e:
                     segs.append((p, b, c, (a - lo) * tile_n, min((e - lo) * tile_n, int(lens[b]))))
             flat = hi
-    return groups, m_tiles, segs
+    # decode groups of 40 tiles or more are cut once more, into 2 or 4 pieces of decreasing size
+    R = 1
+    if mode == bd.MODE_DECODE:
+        per = total // groups
+        R = 4 if per >= 96 else 2 if per >= 40 else 1
+    if R > 1:
+        cum = np.concatenate([[0], np.cumsum(SHARES_64THS[R])])
+        assert cum[-1] == 64
+        pieces, acc_of = [], {}
+        n_g = {}
+        for (p, b, c, k0, k1) in segs:
+            n_g[p] = n_g.get(p, 0) + -(-(k1 - k0) // tile_n)
+        for idx, (p, b, c, k0, k1) in enumerate(segs):
+            nt = -(-(k1 - k0) // tile_n)
+            acc = acc_of.get(p, 0)
+            for r in range(R):
+                lo = max(n_g[p] * int(cum[r]) // 64 - acc, 0)
+                hi = min(n_g[p] * int(cum[r + 1]) // 64 - acc, nt)
+                if lo < hi:
+                    pieces.append((r * groups + p, b, c, k0 + lo * tile_n, min(k0 + hi * tile_n, k1), idx * R + r))
+            acc_of[p] = acc + nt
+        return groups, m_tiles, [q[:5] for q in pieces], [q[5] for q in pieces], R, len(segs)
+    return groups, m_tiles, segs, list(range(len(segs))), 1, len(segs)
+
+
+SHARES_64THS = {2: [52, 12], 4: [44, 10, 7, 3]}
+
+
+def test_sub_bound_follows_the_published_shares():
+    for R, shares in SHARES_64THS.items():
+        cum = np.concatenate([[0], np.cumsum(shares)])
+        for n in (0, 1, 7, 63, 64, 443, 16384, 10 ** 9):
+            got = [bd.yoco_xattn_sub_bound(n, R, r) for r in range(R + 1)]
+            assert got == [n * int(c) // 64 for c in cum] and got[0] == 0 and got[-1] == n
+            assert all(x <= y for x, y in zip(got, got[1:]))
+    assert [bd.yoco_xattn_sub_bound(100, 1, r) for r in (0, 1)] == [0, 100]
+    assert bd.yoco_xattn_sub_bound(100, 3, 1) == -1 and bd.yoco_xattn_sub_bound(100, 8, 1) == -1
+    assert bd.yoco_xattn_sub_bound(-1, 2, 1) == -1
 
 
 CASES = [
@@ -80,12 +117,15 @@ def test_plan_partitions_every_stream_exactly(case, sm_count):
     for mode in modes:
         shape = bd.make_shape(case["B"], case["Hq"], case["Hkv"], case["d"], case["T"])
         info, segs = bd.yoco_xattn_plan(shape, case["lens"], sm_count, mode)
-        groups, m_tiles, want = restated_plan(case["B"], case["Hkv"], case["lens"], sm_count, mode, G, case["T"])
+        groups, m_tiles, want, want_slots, R, coarse = restated_plan(case["B"], case["Hkv"], case["lens"], sm_count,
+                                                                     mode, G, case["T"])
         assert info.num_groups == groups and info.m_tiles == m_tiles
         assert info.num_ctas == groups * m_tiles
+        assert info.sub_items == R and info.num_slots == coarse * R
         got = [(s.group, s.b, s.c, s.k_begin, s.k_end) for s in segs]
         assert got == want                                     # integer for integer
-        assert [s.slot for s in segs] == list(range(len(segs)))  # unique, consecutive slots
+        assert [s.slot for s in segs] == want_slots            # unique, ascending, inside the workspace
+        assert all(x < y for x, y in zip(want_slots, want_slots[1:])) and (not segs or segs[-1].slot < info.num_slots)
         # partition: no gap, no overlap, in order
         for b in range(case["B"]):
             for c in range(case["Hkv"]):
@@ -95,16 +135,21 @@ def test_plan_partitions_every_stream_exactly(case, sm_count):
                     assert s.k_begin == pos and s.k_end > s.k_begin and s.k_begin % info.tile_n == 0
                     pos = s.k_end
                 assert pos == case["lens"][b]
-                if mine:
+                if mine and R == 1:
                     assert [s.slot for s in mine] == list(range(mine[0].slot, mine[0].slot + len(mine)))
-        # balance: every group streams the same number of tiles (+-1)
+        # balance: every group streams the same number of tiles (+-1), all its pieces taken together
         tiles = {}
         for s in segs:
-            tiles[s.group] = tiles.get(s.group, 0) + -(-(s.k_end - s.k_begin) // info.tile_n)
+            tiles[s.group % groups] = tiles.get(s.group % groups, 0) + -(-(s.k_end - s.k_begin) // info.tile_n)
         if tiles:
             assert max(tiles.values()) - min(tiles.values()) <= 1
-        assert info.max_splits == max([0] + [sum(1 for s in segs if (s.b, s.c) == bc)
-                                             for bc in {(s.b, s.c) for s in segs}])
+        # slots of one stream: a run of R per coarse segment
+        per_stream = {}
+        for s in segs:
+            per_stream.setdefault((s.b, s.c), set()).add(s.slot // R)
+        assert info.max_splits == R * max([0] + [len(v) for v in per_stream.values()])
+        for v in per_stream.values():
+            assert sorted(v) == list(range(min(v), min(v) + len(v)))
         # determinism
         info2, segs2 = bd.yoco_xattn_plan(shape, case["lens"], sm_count, mode)
         assert bytes(info) == bytes(info2) and [bytes(s) for s in segs] == [bytes(s) for s in segs2]
@@ -115,7 +160,14 @@ def test_one_million_tokens_fills_the_machine_in_one_wave():
     shape = bd.make_shape(1, 32, 8, 128, 1)
     info, segs = bd.yoco_xattn_plan(shape, [1048576], 148, bd.MODE_DECODE)
     assert info.num_groups == 296 and info.total_tiles == 8 * 16384
-    assert info.needs_combine == 1 and info.num_segments <= 296 + 8
+    assert info.needs_combine == 1 and info.sub_items == 4 and info.num_segments == 4 * 296
+    assert info.num_slots == 4 * 296
+    # piece 0 of every group is the large one; the last pieces are 3/64 of the group
+    sizes = {}
+    for s in segs:
+        sizes.setdefault(s.group // 296, []).append(s.k_end - s.k_begin)
+    per_group = 1048576 * 8 / 296
+    assert min(sizes[0]) >= 0.68 * per_group and max(sizes[3]) <= 0.05 * per_group
 
 
 def test_unsplit_streams_need_no_combine():
