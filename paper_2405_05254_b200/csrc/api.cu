@@ -568,6 +568,7 @@ int32_t kv_append_impl(const yoco_kv_append_shape* shape, const void* X, const v
         if (!cu_kv_host) tok += head_rows;
     }
     KvAppendParams p{};
+    p.X = static_cast<const __nv_bfloat16*>(X);
     p.K = static_cast<__nv_bfloat16*>(K);
     p.V = static_cast<__nv_bfloat16*>(V);
     p.M = s.B * s.T;

@@ -129,6 +129,7 @@ cudaError_t chunk_pair_kernel_setup();
 // ---- writing the cache: K^ = RMSNorm(X) W_K, V^ = RMSNorm(X) W_V appended head-major ------------
 constexpr int kAppendMaxSequences = 512;
 struct KvAppendParams {
+    const __nv_bfloat16* X;     // [M, d_model] (the few-token kernel reads it with plain loads)
     __nv_bfloat16* K;           // packed head-major caches
     __nv_bfloat16* V;
     int32_t M;                  // B * T tokens
@@ -141,7 +142,9 @@ struct KvAppendTables {         // per sequence, as kernel parameters
     int32_t head_rows[kAppendMaxSequences];  // rows between two heads of the sequence
 };
 // tmX: [M, d_model] box {64, 128}; tmWk / tmWv: gain-folded weights [d_model, Hkv*d] box {64, 128};
-// 128-byte swizzle.  Grid = (2*Hkv*d/128, ceil(M/128)).
+// 128-byte swizzle.  Grid = (2*Hkv*d/128, ceil(M/128)); with M <= 16 tokens (a decode step) a second
+// kernel streams the weights instead: clusters of CTAs split d_model and add up through
+// distributed shared memory.
 struct KvAppendScales {         // 8-bit cache: reciprocal of the per-head scales (value = scale * e4m3(byte))
     float inv_k[kFp8MaxHeads];
     float inv_v[kFp8MaxHeads];

@@ -216,6 +216,209 @@ kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     }
 }
 
+// ---- a decode step: at most 16 tokens ---------------------------------------------------------
+// With a handful of rows the product is a stream of the two weight matrices (33 MB at d_model 4,096
+// and 2 x 1,024 output channels) and the 128-row tensor-core tile above would leave all but
+// Hkv * d / 64 SMs idle.  Here a CTA owns 64 output channels and 1/S of d_model; the S CTAs of a
+// cluster cover d_model between them, each with its whole weight slab in flight at once (up to four
+// 16 KB TMA boxes), multiply with mma.sync (the tokens are the 16 rows of the A operand, the slab goes
+// through ldmatrix.trans), and add their partial sums and their partial row sums of squares through
+// distributed shared memory: CTA j of the cluster reduces and stores 64 / S of the channels.
+constexpr int SK_THREADS = 128;
+constexpr int SK_COLS = 64;                      // output channels per CTA: one TMA box wide
+constexpr int SK_KBOX = 128;                     // weight rows per TMA box
+constexpr int SK_STAGES = 4;
+constexpr int SK_ROWS = 16;
+constexpr int SK_XSTRIDE = SK_KBOX + 8;          // bf16 elements per X row in shared memory (conflict-free)
+constexpr int SK_OFF_X = SK_STAGES * HALF_BYTES;
+constexpr int SK_OFF_RED = SK_OFF_X + SK_ROWS * SK_XSTRIDE * 2;
+constexpr int SK_OFF_SSQ = SK_OFF_RED + SK_ROWS * SK_COLS * 4;
+constexpr int SK_OFF_BAR = SK_OFF_SSQ + SK_ROWS * 4;
+constexpr int SK_SMEM_BYTES = SK_OFF_BAR + SK_STAGES * 8 + 16;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float ld_cluster_f(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+
+// grid = (Hkv*d / 64, 2 (K^ | V^), S), cluster (1, 1, S); S * n_chunks * 128 = d_model
+template <bool FP8>
+__global__ void __launch_bounds__(SK_THREADS)
+kv_append_small_kernel(const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmWv,
+                       const KvAppendParams p, const __grid_constant__ KvAppendTables tab,
+                       const __grid_constant__ KvAppendScales sc) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem + SK_OFF_X);
+    float* red = reinterpret_cast<float*>(smem + SK_OFF_RED);      // [16][64] partial sums of this CTA
+    float* ssq = reinterpret_cast<float*>(smem + SK_OFF_SSQ);      // [16] partial sums of squares
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + SK_OFF_BAR);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+    const int S = (int)gridDim.z;
+    const int rank = (int)cluster_ctarank();
+    const bool is_v = blockIdx.y != 0;
+    const int col0 = blockIdx.x * SK_COLS;                 // first channel inside K^ (or V^)
+    const int k_slice = p.d_model / S;
+    const int k_base = rank * k_slice;
+    const int n_chunks = k_slice / SK_KBOX;
+    const CUtensorMap* tmW = is_v ? &tmWv : &tmWk;
+    bool ok = (smem_u32(smem) & 1023u) == 0;
+    if (!ok && threadIdx.x == 0) atomicExch(&g_kv_append_status, kStatusTimeout + 1);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < SK_STAGES; ++s) mbar_init(&full[s], 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && ok) {
+        tma_prefetch_desc(tmW);
+        for (int c = 0; c < n_chunks && c < SK_STAGES; ++c) {
+            mbar_expect_tx(&full[c], HALF_BYTES);
+            tma_load_2d(smem + c * HALF_BYTES, tmW, col0, k_base + c * SK_KBOX, &full[c]);
+        }
+    }
+
+    float acc[2][4];
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    float sq = 0.f;                                         // this thread's share of a row's sum of squares
+    const int xr = threadIdx.x >> 3, xc = (threadIdx.x & 7) * 16;   // X staging: row, first of 16 elements
+
+    for (int c = 0; c < n_chunks; ++c) {
+        // X[:, chunk] -> shared memory (rows beyond M are zero), squares on the way
+        {
+            uint4 v0 = make_uint4(0u, 0u, 0u, 0u), v1 = v0;
+            if (xr < p.M) {
+                const uint4* src = reinterpret_cast<const uint4*>(p.X + (int64_t)xr * p.d_model + k_base + c * SK_KBOX + xc);
+                v0 = src[0];
+                v1 = src[1];
+            }
+            const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float a = __uint_as_float(w[j] << 16), b = __uint_as_float(w[j] & 0xFFFF0000u);
+                sq = fmaf(a, a, sq);
+                sq = fmaf(b, b, sq);
+            }
+            uint4* dst = reinterpret_cast<uint4*>(xs + xr * SK_XSTRIDE + xc);
+            dst[0] = v0;
+            dst[1] = v1;
+        }
+        __syncthreads();
+        const int stage = c % SK_STAGES;
+        if (ok && !mbar_wait(&full[stage], (uint32_t)(c / SK_STAGES) & 1u)) {
+            atomicExch(&g_kv_append_status, kStatusTimeout);
+            ok = false;
+        }
+        if (ok) {
+            const uint32_t wbase = smem_u32(smem + stage * HALF_BYTES);
+            const int k_l = ((lane >> 3) & 1) * 8 + (lane & 7);      // ldmatrix row inside a 16-k step
+            const int chunk16 = warp * 2 + (lane >> 4);              // 16-byte column chunk: 8 channels
+#pragma unroll
+            for (int ks = 0; ks < SK_KBOX / 16; ++ks) {
+                uint32_t a[4];
+                const __nv_bfloat16* x0 = xs + g * SK_XSTRIDE + ks * 16 + tq * 2;
+                a[0] = *reinterpret_cast<const uint32_t*>(x0);
+                a[1] = *reinterpret_cast<const uint32_t*>(x0 + 8 * SK_XSTRIDE);
+                a[2] = *reinterpret_cast<const uint32_t*>(x0 + 8);
+                a[3] = *reinterpret_cast<const uint32_t*>(x0 + 8 * SK_XSTRIDE + 8);
+                const int krow = ks * 16 + k_l;
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4_trans(wbase + krow * 128 + (((chunk16 ^ krow) & 7) << 4), b0, b1, b2, b3);
+                mma_bf16_16816(acc[0], a, b0, b1);
+                mma_bf16_16816(acc[1], a, b2, b3);
+            }
+        }
+        __syncthreads();                                    // everyone is done with xs and with the stage
+        if (threadIdx.x == 0 && ok && c + SK_STAGES < n_chunks) {
+            fence_proxy_async_smem();
+            mbar_expect_tx(&full[stage], HALF_BYTES);
+            tma_load_2d(smem + stage * HALF_BYTES, tmW, col0, k_base + (c + SK_STAGES) * SK_KBOX, &full[stage]);
+        }
+    }
+
+    // partial results of this CTA -> its shared memory
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+        const int col = warp * 16 + nt * 8 + tq * 2;
+        *reinterpret_cast<float2*>(red + g * SK_COLS + col) = make_float2(acc[nt][0], acc[nt][1]);
+        *reinterpret_cast<float2*>(red + (g + 8) * SK_COLS + col) = make_float2(acc[nt][2], acc[nt][3]);
+    }
+    sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+    sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+    sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+    if ((threadIdx.x & 7) == 0) ssq[xr] = sq;
+    cluster_sync_all();
+
+    // CTA `rank` adds up and stores channels [rank * cw, (rank + 1) * cw) of the 64, eight per thread
+    const int cw = SK_COLS / S;                             // 8, 16, 32 or 64
+    const int groups = cw / 8;
+    if (threadIdx.x < SK_ROWS * groups) {
+        const int row = threadIdx.x / groups, cg = threadIdx.x - row * groups;
+        const int col = rank * cw + cg * 8;
+        if (row < p.M) {
+            float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            float total_sq = 0.f;
+            const uint32_t red_addr = smem_u32(red + row * SK_COLS + col);
+            const uint32_t ssq_addr = smem_u32(ssq + row);
+            for (int r = 0; r < S; ++r) {
+                const float4 lo = ld_cluster_f4(map_to_rank(red_addr, r));
+                const float4 hi = ld_cluster_f4(map_to_rank(red_addr + 16, r));
+                v[0] += lo.x; v[1] += lo.y; v[2] += lo.z; v[3] += lo.w;
+                v[4] += hi.x; v[5] += hi.y; v[6] += hi.z; v[7] += hi.w;
+                total_sq += ld_cluster_f(map_to_rank(ssq_addr, r));
+            }
+            const float rn = rsqrtf(total_sq / (float)p.d_model + p.eps);
+            const int i = row / p.T, t = row - i * p.T;
+            const int n = col0 + col;                       // channel inside K^ (or V^)
+            const int head = n / p.d, e = n - head * p.d;
+            const int64_t dst_row = (int64_t)tab.row0[i] + t + (int64_t)head * tab.head_rows[i];
+            if (FP8) {
+                const float rs = rn * (is_v ? sc.inv_v[head] : sc.inv_k[head]);
+                uint32_t w[2];
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const uint32_t lo16 = __nv_cvt_float2_to_fp8x2(make_float2(v[4 * j] * rs, v[4 * j + 1] * rs), __NV_SATFINITE, __NV_E4M3);
+                    const uint32_t hi16 = __nv_cvt_float2_to_fp8x2(make_float2(v[4 * j + 2] * rs, v[4 * j + 3] * rs), __NV_SATFINITE, __NV_E4M3);
+                    w[j] = lo16 | (hi16 << 16);
+                }
+                uint8_t* dst8 = reinterpret_cast<uint8_t*>(is_v ? p.V : p.K) + dst_row * p.d + e;
+                *reinterpret_cast<uint2*>(dst8) = make_uint2(w[0], w[1]);
+            } else {
+                uint4 pk;
+                pk.x = pack_bf16x2(v[0] * rn, v[1] * rn);
+                pk.y = pack_bf16x2(v[2] * rn, v[3] * rn);
+                pk.z = pack_bf16x2(v[4] * rn, v[5] * rn);
+                pk.w = pack_bf16x2(v[6] * rn, v[7] * rn);
+                *reinterpret_cast<uint4*>((is_v ? p.V : p.K) + dst_row * p.d + e) = pk;
+            }
+        }
+    }
+    cluster_sync_all();                                     // nobody leaves while its memory is being read
+}
+
 // Wg[k, n] = g[k] * W[k, n]: the product of two bf16 values is exact in fp32, one rounding to bf16.
 __global__ void fold_gain_kernel(const __nv_bfloat16* __restrict__ g, const __nv_bfloat16* __restrict__ W,
                                  __nv_bfloat16* __restrict__ Wg, int64_t d_model, int64_t n_out) {
@@ -242,13 +445,38 @@ cudaError_t read_and_clear_kv_append_status(int32_t* word, cudaStream_t stream) 
 cudaError_t kv_append_kernel_setup() {
     cudaError_t e = cudaFuncSetAttribute(kv_append_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(kv_append_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if ((e = cudaFuncSetAttribute(kv_append_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) != cudaSuccess)
+        return e;
+    if ((e = cudaFuncSetAttribute(kv_append_small_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  SK_SMEM_BYTES)) != cudaSuccess)
+        return e;
+    return cudaFuncSetAttribute(kv_append_small_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SK_SMEM_BYTES);
 }
 
 cudaError_t launch_kv_append(const KvAppendParams& p, const KvAppendTables& tab, const CUtensorMap& tmX,
                              const CUtensorMap& tmWk, const CUtensorMap& tmWv, cudaStream_t stream,
                              const KvAppendScales* fp8_scales) {
     if (p.M <= 0) return cudaSuccess;
+    if (p.M <= SK_ROWS && p.n_half % SK_COLS == 0 && p.d_model % SK_KBOX == 0) {
+        // a decode step: stream the weights with clusters that split d_model
+        int S = 8;
+        while (S > 1 && p.d_model % (S * SK_KBOX) != 0) S /= 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(p.n_half / SK_COLS), 2u, (unsigned)S);
+        cfg.blockDim = dim3(SK_THREADS);
+        cfg.dynamicSmemBytes = SK_SMEM_BYTES;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 1;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = (unsigned)S;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        KvAppendScales none{};
+        if (fp8_scales) return cudaLaunchKernelEx(&cfg, kv_append_small_kernel<true>, tmWk, tmWv, p, tab, *fp8_scales);
+        return cudaLaunchKernelEx(&cfg, kv_append_small_kernel<false>, tmWk, tmWv, p, tab, none);
+    }
     dim3 grid((unsigned)(2 * p.n_half / BN), (unsigned)((p.M + BM - 1) / BM));
     if (fp8_scales) {
         kv_append_kernel<true><<<grid, kThreads, SMEM_BYTES, stream>>>(tmX, tmWk, tmWv, p, tab, *fp8_scales);

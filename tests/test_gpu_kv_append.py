@@ -66,6 +66,10 @@ def run_append(seed, B, T, d_model, Hkv, d, lens, eps=1e-6, cap=0):
     (3, 40, 3072, 8, 128, [40, 1000, 77]),        # the paper's width, tokens straddle tiles and sequences
     (2, 200, 1024, 2, 64, [200, 513]),            # d = 64: one output tile covers two heads
     (16, 1, 512, 4, 128, list(range(1, 17))),     # a row of the tile per sequence
+    (5, 3, 1536, 2, 64, [3, 70, 1000, 64, 5]),    # 15 tokens: the few-token kernel, three chunks per CTA, d = 64
+    (1, 1, 8192, 8, 128, [4097]),                 # one token, wide model: a CTA reuses its weight stages
+    (4, 4, 4096, 8, 128, [4, 100, 5000, 64]),     # 16 tokens of four sequences
+    (17, 1, 1024, 4, 128, list(range(1, 18))),    # 17 tokens: one more than the few-token kernel takes
 ])
 def test_append_matches_the_oracle_and_touches_nothing_else(B, T, d_model, Hkv, d, lens):
     run_append(80, B, T, d_model, Hkv, d, lens)
@@ -73,6 +77,7 @@ def test_append_matches_the_oracle_and_touches_nothing_else(B, T, d_model, Hkv, 
 
 def test_append_into_a_cache_with_spare_capacity_and_another_eps():
     run_append(81, 2, 9, 1024, 8, 128, [100, 9], eps=1e-2, cap=128)
+    run_append(81, 3, 2, 1024, 8, 128, [100, 2, 128], eps=1e-2, cap=128)     # six tokens: the few-token kernel
 
 
 def test_attention_over_a_cache_written_on_the_gpu():
@@ -163,6 +168,8 @@ def run_append_fp8(seed, B, T, d_model, Hkv, d, lens, cap=0):
     (2, 1, 4096, 8, 128, [300, 1]),
     (3, 40, 3072, 8, 128, [40, 1000, 77]),
     (2, 200, 1024, 2, 64, [200, 513]),
+    (5, 3, 1536, 2, 64, [3, 70, 1000, 64, 5]),    # the few-token kernel
+    (1, 1, 8192, 8, 128, [4097]),
 ])
 def test_fp8_append_writes_the_nearest_codes(B, T, d_model, Hkv, d, lens):
     run_append_fp8(83, B, T, d_model, Hkv, d, lens)
