@@ -253,12 +253,12 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
 __device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
     float4 v;
     asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ float ld_cluster_f(uint32_t addr) {
     float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr));
     return v;
 }
 
@@ -383,12 +383,24 @@ kv_append_small_kernel(const __grid_constant__ CUtensorMap tmWk, const __grid_co
             float total_sq = 0.f;
             const uint32_t red_addr = smem_u32(red + row * SK_COLS + col);
             const uint32_t ssq_addr = smem_u32(ssq + row);
-            for (int r = 0; r < S; ++r) {
-                const float4 lo = ld_cluster_f4(map_to_rank(red_addr, r));
-                const float4 hi = ld_cluster_f4(map_to_rank(red_addr + 16, r));
-                v[0] += lo.x; v[1] += lo.y; v[2] += lo.z; v[3] += lo.w;
-                v[4] += hi.x; v[5] += hi.y; v[6] += hi.z; v[7] += hi.w;
-                total_sq += ld_cluster_f(map_to_rank(ssq_addr, r));
+            // all remote loads first, then the sums: a load-add-load chain would pay S round trips
+            float4 lo[8], hi[8];
+            float part_sq[8];
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                if (r < S) {
+                    lo[r] = ld_cluster_f4(map_to_rank(red_addr, r));
+                    hi[r] = ld_cluster_f4(map_to_rank(red_addr + 16, r));
+                    part_sq[r] = ld_cluster_f(map_to_rank(ssq_addr, r));
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                if (r < S) {
+                    v[0] += lo[r].x; v[1] += lo[r].y; v[2] += lo[r].z; v[3] += lo[r].w;
+                    v[4] += hi[r].x; v[5] += hi[r].y; v[6] += hi[r].z; v[7] += hi[r].w;
+                    total_sq += part_sq[r];
+                }
             }
             const float rn = rsqrtf(total_sq / (float)p.d_model + p.eps);
             const int i = row / p.T, t = row - i * p.T;
