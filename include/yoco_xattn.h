@@ -112,7 +112,8 @@ typedef struct yoco_xattn_plan_info {
  * num_groups contiguous ranges of equal tile count (+-1); a range that crosses a
  * stream boundary becomes several segments.  num_groups = min(total_tiles,
  * sm_count * groups_per_sm(mode)).  sm_count > 0 must be given (pure host call).
- * Decode plans whose groups are long (>= 40 tiles) cut every group's range once more, into
+ * Decode plans whose groups are long (>= 40 tiles) and made of long runs (at most two segments
+ * per group on average) cut every group's range once more, into
  * sub_items pieces of decreasing size (yoco_xattn_sub_bound): the SMs of a GPU do not all
  * stream at the same rate, so CTA g runs piece 0 of its own group and the remaining pieces
  * are handed out, in item order, to whichever CTA is free.  The pieces, their slots and the

@@ -111,7 +111,11 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
             flat += nt - t0;
         }
     }
-    const int R = mode == YOCO_MODE_DECODE ? choose_sub_items(total_tiles / num_groups, max_sub_items) : 1;
+    // Pieces pay when a group is one long run of a stream.  When groups are chains of short streams
+    // (more than two segments per group on average) most streams are not split at all and are written
+    // without a merge; pieces would split every one of them.
+    int R = mode == YOCO_MODE_DECODE ? choose_sub_items(total_tiles / num_groups, max_sub_items) : 1;
+    if ((int64_t)dev.size() > 2 * num_groups) R = 1;
     int32_t max_splits = 0, needs_combine = R > 1 ? 1 : 0;
     for (int st = 0; st < num_streams; ++st) {
         max_splits = std::max(max_splits, stream_nseg[st] * R);
