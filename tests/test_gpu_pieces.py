@@ -26,6 +26,10 @@ def plan_of(w, window=0, stride=0):
     ("four pieces, ragged", dict(B=4, Hq=8, Hkv=8, d=128, T=1, kv_len=[90001, 64, 120000, 31000]), 4),
     ("four pieces, two rows per head, G = 2", dict(B=2, Hq=16, Hkv=8, d=128, T=2, kv_len=[150003, 95000]), 4),
     ("two pieces, d = 64, 16 rows", dict(B=3, Hq=32, Hkv=2, d=64, T=1, kv_len=[200000, 1, 230007]), 2),
+    # 200 streams and ~490 segments: too many for the kernel-parameter tables, so the work tables and the
+    # work counter live in the workspace
+    ("two pieces, tables in the workspace", dict(B=25, Hq=8, Hkv=8, d=128, T=1,
+                                                 kv_len=[4000 + 137 * i for i in range(25)]), 2),
 ])
 def test_ragged_batches_in_pieces_match_the_oracle(name, kw, pieces):
     w = si.Workload("pieces", layers=1, seed=31, **kw)
