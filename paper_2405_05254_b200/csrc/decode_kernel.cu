@@ -163,250 +163,250 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
     bool ok = true;
 
     for (uint32_t n_item = 0;; ++n_item) {
-    // the next item from the producer; the four warps must take the same decision, so a warp
-    // that gives up waiting says so before the barrier and all of them leave together
-    if (!mbar_wait(&item_full[n_item & 1u], (n_item >> 1) & 1u)) {
-        atomicExch(p.status, kStatusTimeout);
-        *give_up = 1;
-    }
-    const int item = item_q[n_item & 1u];
-    named_barrier_sync(1, kConsumerWarps * 32);
-    if (*give_up) break;
-    if (lane == 0) mbar_arrive(&item_empty[n_item & 1u]);
-    if (item >= n_items) break;
-    const int grp = item % n_groups, piece = item / n_groups;
-    const int seg_lo = p.group_begin[grp], seg_hi = p.group_begin[grp + 1];
-    int t_lo = 0, t_hi = 0x7fffffff, t_acc = 0;       // the piece's tiles inside the group
-    if (R > 1) {
-        int n_g = 0;
-        for (int si = seg_lo; si < seg_hi; ++si)
-            n_g += (p.segments[si].k_end - p.segments[si].k_begin + TILE_N - 1) / TILE_N;
-        t_lo = (int)sub_bound(n_g, R, piece);
-        t_hi = (int)sub_bound(n_g, R, piece + 1);
-    }
-
-    for (int si = seg_lo; si < seg_hi; ++si) {
-        const DevSegment seg = p.segments[si];
-        const int seg_tiles = (seg.k_end - seg.k_begin + TILE_N - 1) / TILE_N;
-        const int s_lo = max(t_lo - t_acc, 0), s_hi = min(t_hi - t_acc, seg_tiles);
-        t_acc += seg_tiles;
-        const int slot = seg.slot * R + piece;
-        if (s_lo >= s_hi) {
-            // this piece holds nothing of the segment: its slot must say so to the merge
-            if (R > 1 && threadIdx.x < n_rows) p.part_lse[(int64_t)slot * n_rows + threadIdx.x] = -INFINITY;
-            continue;
+        // the next item from the producer; the four warps must take the same decision, so a warp
+        // that gives up waiting says so before the barrier and all of them leave together
+        if (!mbar_wait(&item_full[n_item & 1u], (n_item >> 1) & 1u)) {
+            atomicExch(p.status, kStatusTimeout);
+            *give_up = 1;
         }
-        const int k_lo = seg.k_begin + s_lo * TILE_N;
-        const int k_hi = min(seg.k_begin + s_hi * TILE_N, seg.k_end);
-
-        // Q as the A operand of m16n8k16: rows = (head in group, t), zero beyond n_rows
-        uint32_t qa[KSTEPS][4];
-        {
-            const __nv_bfloat16* q0 = p.Q + ((int64_t)seg.q_row0 + g) * D + tq * 2;
-            const __nv_bfloat16* q1 = q0 + 8 * D;
-            const bool v0 = g < n_rows, v1 = ROWS == 16 && (g + 8) < n_rows;
-#pragma unroll
-            for (int ks = 0; ks < KSTEPS; ++ks) {
-                qa[ks][0] = v0 ? ld_global_u32(q0 + ks * 16) : 0u;
-                qa[ks][1] = v1 ? ld_global_u32(q1 + ks * 16) : 0u;
-                qa[ks][2] = v0 ? ld_global_u32(q0 + ks * 16 + 8) : 0u;
-                qa[ks][3] = v1 ? ld_global_u32(q1 + ks * 16 + 8) : 0u;
-            }
+        const int item = item_q[n_item & 1u];
+        named_barrier_sync(1, kConsumerWarps * 32);
+        if (*give_up) break;
+        if (lane == 0) mbar_arrive(&item_empty[n_item & 1u]);
+        if (item >= n_items) break;
+        const int grp = item % n_groups, piece = item / n_groups;
+        const int seg_lo = p.group_begin[grp], seg_hi = p.group_begin[grp + 1];
+        int t_lo = 0, t_hi = 0x7fffffff, t_acc = 0;       // the piece's tiles inside the group
+        if (R > 1) {
+            int n_g = 0;
+            for (int si = seg_lo; si < seg_hi; ++si)
+                n_g += (p.segments[si].k_end - p.segments[si].k_begin + TILE_N - 1) / TILE_N;
+            t_lo = (int)sub_bound(n_g, R, piece);
+            t_hi = (int)sub_bound(n_g, R, piece + 1);
         }
-        // causal limits: row t sees keys j < n_kv - T + 1 + t
-        const int n_full = seg.n_kv - p.T + 1;
-        const int vis0 = min(seg.n_kv, max(0, n_full + (g % p.T)));
-        const int vis1 = min(seg.n_kv, max(0, n_full + ((g + 8) % p.T)));
 
-        float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-        float o[NT_O][4];
-#pragma unroll
-        for (int nt = 0; nt < NT_O; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-
-        for (int k0 = k_lo; k0 < k_hi; k0 += TILE_N, ++it) {
-            if (!ok) continue;
-            const uint32_t stage = it % STAGES, round = it / STAGES;
-            if (!mbar_wait(&full_bar[stage], round & 1u)) {
-                atomicExch(p.status, kStatusTimeout);
-                ok = false;
+        for (int si = seg_lo; si < seg_hi; ++si) {
+            const DevSegment seg = p.segments[si];
+            const int seg_tiles = (seg.k_end - seg.k_begin + TILE_N - 1) / TILE_N;
+            const int s_lo = max(t_lo - t_acc, 0), s_hi = min(t_hi - t_acc, seg_tiles);
+            t_acc += seg_tiles;
+            const int slot = seg.slot * R + piece;
+            if (s_lo >= s_hi) {
+                // this piece holds nothing of the segment: its slot must say so to the merge
+                if (R > 1 && threadIdx.x < n_rows) p.part_lse[(int64_t)slot * n_rows + threadIdx.x] = -INFINITY;
                 continue;
             }
-            const int kw = k0 + warp * 16;          // first key of this warp's slice
-            if (kw < k_hi) {
-                const uint32_t kbase = smem_u32(stage_mem + stage * C::STAGE_BYTES);
-                const uint32_t vbase = kbase + C::TENSOR_BYTES;
+            const int k_lo = seg.k_begin + s_lo * TILE_N;
+            const int k_hi = min(seg.k_begin + s_hi * TILE_N, seg.k_end);
 
-                // ---- S = Q K^T for 16 keys (two n-tiles of 8 keys) ----
-                float s[2][4];
+            // Q as the A operand of m16n8k16: rows = (head in group, t), zero beyond n_rows
+            uint32_t qa[KSTEPS][4];
+            {
+                const __nv_bfloat16* q0 = p.Q + ((int64_t)seg.q_row0 + g) * D + tq * 2;
+                const __nv_bfloat16* q1 = q0 + 8 * D;
+                const bool v0 = g < n_rows, v1 = ROWS == 16 && (g + 8) < n_rows;
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-                {
-                    const int key_l = warp * 16 + (lane >> 4) * 8 + (lane & 7);
-                    const int sel = (lane >> 3) & 1;
-                    const uint32_t rowaddr = kbase + key_l * 128;
-#pragma unroll
-                    for (int ks = 0; ks < KSTEPS; ++ks) {
-                        const int c = 2 * ks + sel;
-                        const uint32_t addr =
-                            rowaddr + (c >> 3) * HALF_BYTES + ((((c & 7) ^ key_l) & 7) << 4);
-                        uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4(addr, b0, b1, b2, b3);
-                        mma_bf16_16816(s[0], qa[ks], b0, b1);
-                        mma_bf16_16816(s[1], qa[ks], b2, b3);
-                    }
+                for (int ks = 0; ks < KSTEPS; ++ks) {
+                    qa[ks][0] = v0 ? ld_global_u32(q0 + ks * 16) : 0u;
+                    qa[ks][1] = v1 ? ld_global_u32(q1 + ks * 16) : 0u;
+                    qa[ks][2] = v0 ? ld_global_u32(q0 + ks * 16 + 8) : 0u;
+                    qa[ks][3] = v1 ? ld_global_u32(q1 + ks * 16 + 8) : 0u;
                 }
-                // ---- scale, mask, online softmax ----
-                // sliding window: the row at position i = n_kv - T + t keeps i - C < j, i.e.
-                // j >= i - C + 1 = n_full + t - C; the highest such bound of any row is n_kv - C
-                const bool need_mask = kw + 16 > n_full || (p.window > 0 && kw < seg.n_kv - p.window);
-                // window start of the two rows this lane holds (no window: below every key)
-                int lo0 = -1, lo1 = -1;
-                if (need_mask && p.window > 0) {
-                    lo0 = n_full + (g % p.T) - p.window;
-                    lo1 = n_full + ((g + 8) % p.T) - p.window;
+            }
+            // causal limits: row t sees keys j < n_kv - T + 1 + t
+            const int n_full = seg.n_kv - p.T + 1;
+            const int vis0 = min(seg.n_kv, max(0, n_full + (g % p.T)));
+            const int vis1 = min(seg.n_kv, max(0, n_full + ((g + 8) % p.T)));
+
+            float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+            float o[NT_O][4];
+#pragma unroll
+            for (int nt = 0; nt < NT_O; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+
+            for (int k0 = k_lo; k0 < k_hi; k0 += TILE_N, ++it) {
+                if (!ok) continue;
+                const uint32_t stage = it % STAGES, round = it / STAGES;
+                if (!mbar_wait(&full_bar[stage], round & 1u)) {
+                    atomicExch(p.status, kStatusTimeout);
+                    ok = false;
+                    continue;
                 }
+                const int kw = k0 + warp * 16;          // first key of this warp's slice
+                if (kw < k_hi) {
+                    const uint32_t kbase = smem_u32(stage_mem + stage * C::STAGE_BYTES);
+                    const uint32_t vbase = kbase + C::TENSOR_BYTES;
+
+                    // ---- S = Q K^T for 16 keys (two n-tiles of 8 keys) ----
+                    float s[2][4];
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt)
+                    for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+                    {
+                        const int key_l = warp * 16 + (lane >> 4) * 8 + (lane & 7);
+                        const int sel = (lane >> 3) & 1;
+                        const uint32_t rowaddr = kbase + key_l * 128;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        float v = s[nt][e] * p.scale_log2;
-                        if (need_mask) {
-                            const int j = kw + nt * 8 + tq * 2 + (e & 1);
-                            v = (j < ((e & 2) ? vis1 : vis0) && j >= ((e & 2) ? lo1 : lo0)) ? v : -INFINITY;
+                        for (int ks = 0; ks < KSTEPS; ++ks) {
+                            const int c = 2 * ks + sel;
+                            const uint32_t addr =
+                                rowaddr + (c >> 3) * HALF_BYTES + ((((c & 7) ^ key_l) & 7) << 4);
+                            uint32_t b0, b1, b2, b3;
+                            ldmatrix_x4(addr, b0, b1, b2, b3);
+                            mma_bf16_16816(s[0], qa[ks], b0, b1);
+                            mma_bf16_16816(s[1], qa[ks], b2, b3);
                         }
-                        s[nt][e] = v;
                     }
-                float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-                const float mn0 = fmaxf(m0, mx0);
-                const float ms0 = mn0 == -INFINITY ? 0.f : mn0;
-                const float alpha0 = exp2f(m0 - ms0);
-                m0 = mn0;
-                float alpha1 = 1.f, ms1 = 0.f;
-                if (ROWS == 16) {
-                    float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
-                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-                    const float mn1 = fmaxf(m1, mx1);
-                    ms1 = mn1 == -INFINITY ? 0.f : mn1;
-                    alpha1 = exp2f(m1 - ms1);
-                    m1 = mn1;
-                }
-                uint32_t pa[4];
-                {
-                    const float p00 = exp2f(s[0][0] - ms0), p01 = exp2f(s[0][1] - ms0);
-                    const float p10 = exp2f(s[1][0] - ms0), p11 = exp2f(s[1][1] - ms0);
-                    l0 = l0 * alpha0 + ((p00 + p01) + (p10 + p11));
-                    pa[0] = pack_bf16x2(p00, p01);
-                    pa[2] = pack_bf16x2(p10, p11);
+                    // ---- scale, mask, online softmax ----
+                    // sliding window: the row at position i = n_kv - T + t keeps i - C < j, i.e.
+                    // j >= i - C + 1 = n_full + t - C; the highest such bound of any row is n_kv - C
+                    const bool need_mask = kw + 16 > n_full || (p.window > 0 && kw < seg.n_kv - p.window);
+                    // window start of the two rows this lane holds (no window: below every key)
+                    int lo0 = -1, lo1 = -1;
+                    if (need_mask && p.window > 0) {
+                        lo0 = n_full + (g % p.T) - p.window;
+                        lo1 = n_full + ((g + 8) % p.T) - p.window;
+                    }
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            float v = s[nt][e] * p.scale_log2;
+                            if (need_mask) {
+                                const int j = kw + nt * 8 + tq * 2 + (e & 1);
+                                v = (j < ((e & 2) ? vis1 : vis0) && j >= ((e & 2) ? lo1 : lo0)) ? v : -INFINITY;
+                            }
+                            s[nt][e] = v;
+                        }
+                    float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+                    const float mn0 = fmaxf(m0, mx0);
+                    const float ms0 = mn0 == -INFINITY ? 0.f : mn0;
+                    const float alpha0 = exp2f(m0 - ms0);
+                    m0 = mn0;
+                    float alpha1 = 1.f, ms1 = 0.f;
                     if (ROWS == 16) {
-                        const float q00 = exp2f(s[0][2] - ms1), q01 = exp2f(s[0][3] - ms1);
-                        const float q10 = exp2f(s[1][2] - ms1), q11 = exp2f(s[1][3] - ms1);
-                        l1 = l1 * alpha1 + ((q00 + q01) + (q10 + q11));
-                        pa[1] = pack_bf16x2(q00, q01);
-                        pa[3] = pack_bf16x2(q10, q11);
-                    } else {
-                        pa[1] = pa[3] = 0u;
+                        float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+                        const float mn1 = fmaxf(m1, mx1);
+                        ms1 = mn1 == -INFINITY ? 0.f : mn1;
+                        alpha1 = exp2f(m1 - ms1);
+                        m1 = mn1;
                     }
-                }
-                if (__any_sync(0xffffffffu, alpha0 != 1.f || alpha1 != 1.f)) {
-#pragma unroll
-                    for (int nt = 0; nt < NT_O; ++nt) {
-                        o[nt][0] *= alpha0; o[nt][1] *= alpha0;
-                        o[nt][2] *= alpha1; o[nt][3] *= alpha1;
-                    }
-                }
-                // ---- rows past the end of the sequence may hold anything: zero them so that
-                //      0 * garbage cannot produce NaN in O += P V ----
-                if (kw + 16 > seg.n_kv) {
-                    const int first_bad = max(seg.n_kv - kw, 0);          // 0..15
-                    uint8_t* vrow = stage_mem + stage * C::STAGE_BYTES + C::TENSOR_BYTES;
-                    for (int r = first_bad; r < 16; ++r) {
-                        const int key_l = warp * 16 + r;
-                        for (int b = lane * 16; b < C::HALVES * 128; b += 512) {
-                            const int h = b >> 7, off = b & 127;
-                            *reinterpret_cast<uint4*>(vrow + h * HALF_BYTES + key_l * 128 + off) =
-                                make_uint4(0u, 0u, 0u, 0u);
+                    uint32_t pa[4];
+                    {
+                        const float p00 = exp2f(s[0][0] - ms0), p01 = exp2f(s[0][1] - ms0);
+                        const float p10 = exp2f(s[1][0] - ms0), p11 = exp2f(s[1][1] - ms0);
+                        l0 = l0 * alpha0 + ((p00 + p01) + (p10 + p11));
+                        pa[0] = pack_bf16x2(p00, p01);
+                        pa[2] = pack_bf16x2(p10, p11);
+                        if (ROWS == 16) {
+                            const float q00 = exp2f(s[0][2] - ms1), q01 = exp2f(s[0][3] - ms1);
+                            const float q10 = exp2f(s[1][2] - ms1), q11 = exp2f(s[1][3] - ms1);
+                            l1 = l1 * alpha1 + ((q00 + q01) + (q10 + q11));
+                            pa[1] = pack_bf16x2(q00, q01);
+                            pa[3] = pack_bf16x2(q10, q11);
+                        } else {
+                            pa[1] = pa[3] = 0u;
                         }
                     }
-                    __syncwarp();
-                }
-                // ---- O += P V ----
-                {
-                    const int key_l = warp * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
-                    const int sel = lane >> 4;
-                    const uint32_t rowaddr = vbase + key_l * 128;
+                    if (__any_sync(0xffffffffu, alpha0 != 1.f || alpha1 != 1.f)) {
 #pragma unroll
-                    for (int nt = 0; nt < NT_O; nt += 2) {
-                        const int c = nt + sel;
-                        const uint32_t addr =
-                            rowaddr + (c >> 3) * HALF_BYTES + ((((c & 7) ^ key_l) & 7) << 4);
-                        uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4_trans(addr, b0, b1, b2, b3);
-                        mma_bf16_16816(o[nt], pa, b0, b1);
-                        mma_bf16_16816(o[nt + 1], pa, b2, b3);
+                        for (int nt = 0; nt < NT_O; ++nt) {
+                            o[nt][0] *= alpha0; o[nt][1] *= alpha0;
+                            o[nt][2] *= alpha1; o[nt][3] *= alpha1;
+                        }
+                    }
+                    // ---- rows past the end of the sequence may hold anything: zero them so that
+                    //      0 * garbage cannot produce NaN in O += P V ----
+                    if (kw + 16 > seg.n_kv) {
+                        const int first_bad = max(seg.n_kv - kw, 0);          // 0..15
+                        uint8_t* vrow = stage_mem + stage * C::STAGE_BYTES + C::TENSOR_BYTES;
+                        for (int r = first_bad; r < 16; ++r) {
+                            const int key_l = warp * 16 + r;
+                            for (int b = lane * 16; b < C::HALVES * 128; b += 512) {
+                                const int h = b >> 7, off = b & 127;
+                                *reinterpret_cast<uint4*>(vrow + h * HALF_BYTES + key_l * 128 + off) =
+                                    make_uint4(0u, 0u, 0u, 0u);
+                            }
+                        }
+                        __syncwarp();
+                    }
+                    // ---- O += P V ----
+                    {
+                        const int key_l = warp * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+                        const int sel = lane >> 4;
+                        const uint32_t rowaddr = vbase + key_l * 128;
+#pragma unroll
+                        for (int nt = 0; nt < NT_O; nt += 2) {
+                            const int c = nt + sel;
+                            const uint32_t addr =
+                                rowaddr + (c >> 3) * HALF_BYTES + ((((c & 7) ^ key_l) & 7) << 4);
+                            uint32_t b0, b1, b2, b3;
+                            ldmatrix_x4_trans(addr, b0, b1, b2, b3);
+                            mma_bf16_16816(o[nt], pa, b0, b1);
+                            mma_bf16_16816(o[nt + 1], pa, b2, b3);
+                        }
+                    }
+                    if (kw + 16 > seg.n_kv) fence_proxy_async_smem();   // generic writes before TMA reuse
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[stage]);
+            }
+
+            // ---- merge the four warps' states, write the final rows or this segment's partial ----
+            l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+            l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+            if (ROWS == 16) {
+                l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+                l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+            }
+            {
+                float* mo = merge_o + (warp * ROWS) * D;
+#pragma unroll
+                for (int nt = 0; nt < NT_O; ++nt) {
+                    *reinterpret_cast<float2*>(mo + g * D + nt * 8 + tq * 2) = make_float2(o[nt][0], o[nt][1]);
+                    if (ROWS == 16)
+                        *reinterpret_cast<float2*>(mo + (g + 8) * D + nt * 8 + tq * 2) =
+                            make_float2(o[nt][2], o[nt][3]);
+                }
+                if (tq == 0) {
+                    merge_ml[(warp * ROWS + g) * 2] = m0;
+                    merge_ml[(warp * ROWS + g) * 2 + 1] = l0;
+                    if (ROWS == 16) {
+                        merge_ml[(warp * ROWS + g + 8) * 2] = m1;
+                        merge_ml[(warp * ROWS + g + 8) * 2 + 1] = l1;
                     }
                 }
-                if (kw + 16 > seg.n_kv) fence_proxy_async_smem();   // generic writes before TMA reuse
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[stage]);
-        }
-
-        // ---- merge the four warps' states, write the final rows or this segment's partial ----
-        l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-        l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-        if (ROWS == 16) {
-            l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-            l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-        }
-        {
-            float* mo = merge_o + (warp * ROWS) * D;
+            named_barrier_sync(1, kConsumerWarps * 32);
+            const bool final_out = seg.stream_nseg == 1 && !p.force_partial && R == 1;
+            for (int idx = threadIdx.x; idx < n_rows * D; idx += kConsumerWarps * 32) {
+                const int r = idx / D, col = idx - r * D;
+                float M = -INFINITY;
 #pragma unroll
-            for (int nt = 0; nt < NT_O; ++nt) {
-                *reinterpret_cast<float2*>(mo + g * D + nt * 8 + tq * 2) = make_float2(o[nt][0], o[nt][1]);
-                if (ROWS == 16)
-                    *reinterpret_cast<float2*>(mo + (g + 8) * D + nt * 8 + tq * 2) =
-                        make_float2(o[nt][2], o[nt][3]);
-            }
-            if (tq == 0) {
-                merge_ml[(warp * ROWS + g) * 2] = m0;
-                merge_ml[(warp * ROWS + g) * 2 + 1] = l0;
-                if (ROWS == 16) {
-                    merge_ml[(warp * ROWS + g + 8) * 2] = m1;
-                    merge_ml[(warp * ROWS + g + 8) * 2 + 1] = l1;
+                for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, merge_ml[(w * ROWS + r) * 2]);
+                float L = 0.f, acc = 0.f;
+                if (M != -INFINITY) {
+#pragma unroll
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        const float f = exp2f(merge_ml[(w * ROWS + r) * 2] - M);
+                        L += merge_ml[(w * ROWS + r) * 2 + 1] * f;
+                        acc += merge_o[(w * ROWS + r) * D + col] * f;
+                    }
+                }
+                const float outv = L > 0.f ? acc / L : 0.f;
+                const float lse = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+                if (final_out) {
+                    p.O[((int64_t)seg.q_row0 + r) * D + col] = __float2bfloat16(outv);
+                    if (p.lse && col == 0) p.lse[seg.q_row0 + r] = lse;
+                } else {
+                    p.part_o[((int64_t)slot * n_rows + r) * D + col] = outv;
+                    if (col == 0) p.part_lse[(int64_t)slot * n_rows + r] = lse;
                 }
             }
+            named_barrier_sync(1, kConsumerWarps * 32);
         }
-        named_barrier_sync(1, kConsumerWarps * 32);
-        const bool final_out = seg.stream_nseg == 1 && !p.force_partial && R == 1;
-        for (int idx = threadIdx.x; idx < n_rows * D; idx += kConsumerWarps * 32) {
-            const int r = idx / D, col = idx - r * D;
-            float M = -INFINITY;
-#pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, merge_ml[(w * ROWS + r) * 2]);
-            float L = 0.f, acc = 0.f;
-            if (M != -INFINITY) {
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float f = exp2f(merge_ml[(w * ROWS + r) * 2] - M);
-                    L += merge_ml[(w * ROWS + r) * 2 + 1] * f;
-                    acc += merge_o[(w * ROWS + r) * D + col] * f;
-                }
-            }
-            const float outv = L > 0.f ? acc / L : 0.f;
-            const float lse = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
-            if (final_out) {
-                p.O[((int64_t)seg.q_row0 + r) * D + col] = __float2bfloat16(outv);
-                if (p.lse && col == 0) p.lse[seg.q_row0 + r] = lse;
-            } else {
-                p.part_o[((int64_t)slot * n_rows + r) * D + col] = outv;
-                if (col == 0) p.part_lse[(int64_t)slot * n_rows + r] = lse;
-            }
-        }
-        named_barrier_sync(1, kConsumerWarps * 32);
-    }
     }
 }
 
