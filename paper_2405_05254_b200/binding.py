@@ -160,6 +160,31 @@ def yoco_xattn_decode(shape: Shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, s
     _run("yoco_xattn_decode", shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream)
 
 
+class PreparedCall:
+    """A decode or chunk call whose arguments are marshalled once: a serving loop that makes the same
+    layer call every step (same buffers, same lengths) pays the ctypes conversions a single time.
+    The tensors and arrays are kept alive by the object; run() only enqueues."""
+
+    def __init__(self, fn_name, shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream=None):
+        self._keep = (shape, Q, K, V, O, lse, workspace, stream) + _host_i32(cu_kv)[:1] + _host_i32(kv_len)[:1]
+        p_cu = None if self._keep[-2] is None else ctypes.c_void_p(self._keep[-2].ctypes.data)
+        p_len = None if self._keep[-1] is None else ctypes.c_void_p(self._keep[-1].ctypes.data)
+        self._name = fn_name
+        self._fn = getattr(lib(), fn_name)
+        self._args = (ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), p_cu, p_len, _ptr(O), _ptr(lse), _ptr(workspace),
+                      ctypes.c_size_t(workspace.numel() * workspace.element_size()), _stream_ptr(stream))
+
+    def run(self) -> None:
+        rc = self._fn(*self._args)
+        if rc != OK:
+            raise YocoError(rc, self._name)
+
+
+def prepare_decode(shape: Shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream=None) -> PreparedCall:
+    """yoco_xattn_decode with its arguments marshalled once; call .run() to enqueue it."""
+    return PreparedCall("yoco_xattn_decode", shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream)
+
+
 def yoco_xattn_chunk(shape: Shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream=None) -> None:
     """Enqueue the multi-token (tcgen05) attention on the stream."""
     _run("yoco_xattn_chunk", shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream)

@@ -329,3 +329,20 @@ def test_pieces_give_the_same_bits_whoever_runs_them():
         assert np.array_equal(lse, ref_lse)
     torch.cuda.synchronize()
     assert bd.yoco_xattn_status(W2) == 0
+
+
+def test_prepared_call_gives_the_same_bits_as_the_plain_call():
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    w = si.workload("ragged_small")
+    r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, w.T, w.kv_len, w.make_k(), w.make_v())
+    _, _, O1 = r.run(w.make_q(0))
+    want = O1.view(torch.int16).clone()
+    O, L, W = r._buffers(bd.MODE_DECODE)
+    Q = to_dev_bf16(w.make_q(0).reshape(-1))
+    call = bd.prepare_decode(r.shape, Q, r.K, r.V, r.cu, r.kv_len, O, L, W)
+    for _ in range(3):
+        O.zero_()
+        call.run()
+        assert bd.yoco_xattn_status(W) == 0
+        assert torch.equal(O.view(torch.int16), want)
