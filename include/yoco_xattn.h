@@ -96,9 +96,7 @@ typedef struct yoco_xattn_plan_info {
     int32_t m_tiles;         /* row tiles per stream = ceil(G*T / tile_m)                 */
     int32_t num_groups;      /* CTA groups; each streams one contiguous range of the flat
                                 (stream, key tile) space                                  */
-    int32_t num_ctas;        /* grid size: num_groups * m_tiles work items, one per CTA;
-                                chunk mode with tile_m = 256 may give a CTA several items
-                                (item b, b + num_ctas, ...) so that no SM stays idle       */
+    int32_t num_ctas;        /* grid size = num_groups * m_tiles                          */
     int32_t num_streams;     /* B * Hkv                                                   */
     int32_t num_segments;    /* total work segments = number of partial slots             */
     int32_t max_splits;      /* most segments any one stream was cut into                 */
@@ -113,9 +111,7 @@ typedef struct yoco_xattn_plan_info {
  * The flat space of (stream, key tile) pairs, streams ordered (b, c), is cut into
  * num_groups contiguous ranges of equal tile count (+-1); a range that crosses a
  * stream boundary becomes several segments.  num_groups = min(total_tiles,
- * sm_count * groups_per_sm(mode)); chunk mode: sm_count / m_tiles, or with 256-row tiles
- * W * sm_count / m_tiles for the W in 1..4 items per CTA that leaves the fewest SMs idle.
- * sm_count > 0 must be given (pure host call).
+ * sm_count * groups_per_sm(mode)).  sm_count > 0 must be given (pure host call).
  * Decode plans whose groups are long (>= 40 tiles) and made of long runs (at most two segments
  * per group on average) cut every group's range once more, into
  * sub_items pieces of decreasing size (yoco_xattn_sub_bound): the SMs of a GPU do not all

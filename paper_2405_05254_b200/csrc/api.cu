@@ -318,11 +318,10 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             p.T = shape->T;
             p.rows_per_stream = plan.rows_per_stream;
             p.m_tiles = plan.info.m_tiles;
-            p.n_items = plan.info.num_groups * plan.info.m_tiles;
             p.d = shape->d;
             p.window = shape->window;
             if (plan.info.tile_m == kChunkPairTileM)
-                YOCO_CUDA_TRY(launch_chunk_pair(p, tmQ, tmK, tmV, plan.info.num_ctas, stream));
+                YOCO_CUDA_TRY(launch_chunk_pair(p, tmQ, tmK, tmV, plan.info.num_groups, stream));
             else
                 YOCO_CUDA_TRY(launch_chunk(p, tmQ, tmK, tmV, plan.info.num_groups, stream));
         }

@@ -61,39 +61,9 @@ __host__ __device__ constexpr bool poly_pair(int j) {
     return ((j + 1) * kPolyPairs) / 16 != (j * kPolyPairs) / 16;
 }
 
-// The work items of one CTA, in order: item = (group, row-tile pair); a CTA takes items blockIdx.x,
-// blockIdx.x + gridDim.x, ... and every role walks the segments of those items one after the other.
-struct ItemWalk {
-    const int32_t* group_begin;
-    int item, n_items, stride, m_tiles;
-    int si, seg_hi, m_tile;
-    __device__ __forceinline__ void load() {
-        while (item < n_items) {
-            const int g = item / m_tiles;
-            m_tile = item - g * m_tiles;
-            si = group_begin[g];
-            seg_hi = group_begin[g + 1];
-            if (si < seg_hi) return;
-            item += stride;
-        }
-    }
-    __device__ __forceinline__ ItemWalk(const ChunkParams& p)
-        : group_begin(p.group_begin), item((int)blockIdx.x), n_items(p.n_items), stride((int)gridDim.x),
-          m_tiles(p.m_tiles), si(0), seg_hi(0), m_tile(0) {
-        load();
-    }
-    __device__ __forceinline__ bool valid() const { return item < n_items; }
-    __device__ __forceinline__ void next_segment() {
-        if (++si >= seg_hi) {
-            item += stride;
-            load();
-        }
-    }
-};
-
 // position in the CTA's flat sequence of (segment, key tile) pairs
 struct TileCursor {
-    int k0, k_end, h;
+    int si, k0, k_end, h;
     uint32_t tp;                 // parity of the key tile number since the start of the CTA
     uint32_t kb, kph, vb, vph;   // ring stage and phase parity of the K and V tiles
     bool first_tile;             // first key tile of its segment
@@ -125,6 +95,8 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int group = blockIdx.x / p.m_tiles, m_tile = blockIdx.x - group * p.m_tiles;
+    const int seg_lo = p.group_begin[group], seg_hi = p.group_begin[group + 1];
     const Abort ab{abort_flag, p.status};
     const bool aligned_ok = (smem_u32(smem) & 1023u) == 0;
 
@@ -168,10 +140,9 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tma_prefetch_desc(&tmV);
             uint32_t it = 0;
             bool ok = true;
-            uint32_t sidx = 0;           // segments started by this CTA
-            for (ItemWalk wk(p); wk.valid() && ok; wk.next_segment(), ++sidx) {
-                const DevSegment seg = p.segments[wk.si];
-                const int m_tile = wk.m_tile;
+            for (int si = seg_lo; si < seg_hi && ok; ++si) {
+                const DevSegment seg = p.segments[si];
+                const uint32_t sidx = si - seg_lo;
                 if (!(ok = wait_or_abort(q_empty, (sidx & 1u) ^ 1u, ab))) break;
                 mbar_expect_tx(q_full, 2 * C::TILE_BYTES);
                 for (int r = 0; r < 2; ++r)
@@ -206,17 +177,17 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             constexpr uint32_t idesc_qk = make_idesc(BH, false);
             constexpr uint32_t idesc_pv = make_idesc(D, true);
             const uint32_t sbase = smem_u32(smem);
-            ItemWalk wk(p);
             TileCursor c;
+            c.si = seg_lo;
             c.h = 0;
             c.tp = 0;
             c.kb = c.kph = c.vb = c.vph = 0;
             c.first_tile = false;
             auto cur_load = [&]() {
-                c.valid = wk.valid();
+                c.valid = c.si < seg_hi;
                 if (c.valid) {
-                    c.k0 = p.segments[wk.si].k_begin;
-                    c.k_end = p.segments[wk.si].k_end;
+                    c.k0 = p.segments[c.si].k_begin;
+                    c.k_end = p.segments[c.si].k_end;
                     c.first_tile = true;
                 }
             };
@@ -238,7 +209,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 c.first_tile = false;
                 c.k0 += BN;
                 if (c.k0 >= c.k_end) {
-                    wk.next_segment();
+                    ++c.si;
                     cur_load();
                 }
             };
@@ -316,13 +287,13 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const uint32_t tmem_s = tmem_base + r * BN + lane_addr;
         const uint32_t tmem_o = tmem_base + 2 * BN + r * BN + lane_addr;
+        const int r_local = (m_tile * 2 + r) * BM + row;   // row inside the stream's G*T rows
+        const bool row_valid = r_local < p.rows_per_stream;
         uint32_t it = 0;
         bool ok = aligned_ok;
 
-        for (ItemWalk wk(p); wk.valid(); wk.next_segment()) {
-            const DevSegment seg = p.segments[wk.si];
-            const int r_local = (wk.m_tile * 2 + r) * BM + row;   // row inside the stream's G*T rows
-            const bool row_valid = r_local < p.rows_per_stream;
+        for (int si = seg_lo; si < seg_hi; ++si) {
+            const DevSegment seg = p.segments[si];
             const int n_full = seg.n_kv - p.T + 1;     // keys visible to every row
             const int vis = min(seg.n_kv, max(0, n_full + (r_local % p.T)));
             // sliding window: the row at position i keeps i - C < j; lo_max is the highest such bound
@@ -511,8 +482,8 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
 template <int D>
 cudaError_t launch_one(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                       const CUtensorMap& tmV, int num_ctas, cudaStream_t stream) {
-    chunk_pair_kernel<D><<<num_ctas, kThreads, PCfg<D>::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, p);
+                       const CUtensorMap& tmV, int num_groups, cudaStream_t stream) {
+    chunk_pair_kernel<D><<<num_groups * p.m_tiles, kThreads, PCfg<D>::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, p);
     return cudaGetLastError();
 }
 
@@ -536,10 +507,10 @@ cudaError_t chunk_pair_kernel_setup() {
 }
 
 cudaError_t launch_chunk_pair(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                              const CUtensorMap& tmV, int num_ctas, cudaStream_t stream) {
-    if (num_ctas <= 0) return cudaSuccess;
-    return p.d == 128 ? launch_one<128>(p, tmQ, tmK, tmV, num_ctas, stream)
-                      : launch_one<64>(p, tmQ, tmK, tmV, num_ctas, stream);
+                              const CUtensorMap& tmV, int num_groups, cudaStream_t stream) {
+    if (num_groups <= 0) return cudaSuccess;
+    return p.d == 128 ? launch_one<128>(p, tmQ, tmK, tmV, num_groups, stream)
+                      : launch_one<64>(p, tmQ, tmK, tmV, num_groups, stream);
 }
 
 }  // namespace yoco

@@ -111,7 +111,6 @@ struct ChunkParams {
     int32_t T;
     int32_t rows_per_stream;    // G * T
     int32_t m_tiles;            // ceil(rows_per_stream / 128)
-    int32_t n_items;            // num_groups * m_tiles work items (the two-tile kernel may give a CTA several)
     int32_t d;
     int32_t window;             // sliding window C, 0 = none
 };
@@ -121,11 +120,10 @@ struct ChunkParams {
 cudaError_t launch_chunk(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                          const CUtensorMap& tmV, int num_groups, cudaStream_t stream);
 cudaError_t chunk_kernel_setup();
-// For streams with more than 128 rows: a work item is (group, pair of 128-row tiles), m_tiles =
-// ceil(rows_per_stream / 256), tmQ box is still {64, 128}.  Grid = num_ctas; CTA b runs items b,
-// b + num_ctas, ... of the p.n_items one after the other.
+// Same interface for streams with more than 128 rows: one CTA owns two 128-row tiles (m_tiles =
+// ceil(rows_per_stream / 256)), tmQ box is still {64, 128}.
 cudaError_t launch_chunk_pair(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                              const CUtensorMap& tmV, int num_ctas, cudaStream_t stream);
+                              const CUtensorMap& tmV, int num_groups, cudaStream_t stream);
 cudaError_t chunk_pair_kernel_setup();
 
 // ---- writing the cache: K^ = RMSNorm(X) W_K, V^ = RMSNorm(X) W_V appended head-major ------------

@@ -65,33 +65,11 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     }
 
     // number of CTA groups
-    // Chunk mode, two-tile kernel: a work item is (group, row-tile pair) and a CTA may run several,
-    // so the group count is chosen for the fewest idle SMs: with W items per CTA there are
-    // W * sm_count / m_tiles groups, and the time goes as ceil(items / sm_count) / groups.  More items
-    // per CTA mean more partial results to merge, so W grows only for a gain of at least 1 %.
     int64_t target;
-    int64_t items_per_cta = 1;
-    if (mode == YOCO_MODE_DECODE) {
+    if (mode == YOCO_MODE_DECODE)
         target = (int64_t)sm_count * kDecodeGroupsPerSm;
-    } else {
+    else
         target = std::max<int64_t>(1, sm_count / m_tiles);
-        if (tile_m == kChunkPairTileM) {
-            auto groups_of = [&](int64_t W) {
-                return std::max<int64_t>(1, std::min<int64_t>(W * sm_count / m_tiles, std::max<int64_t>(total_tiles, 1)));
-            };
-            auto cost = [&](int64_t W) {      // relative time: items a CTA runs / groups a stream is cut into
-                const int64_t g = groups_of(W);
-                return (double)((g * m_tiles + sm_count - 1) / sm_count) / (double)g;
-            };
-            double best = cost(1);
-            for (int64_t W = 2; W <= 4; ++W)
-                if (cost(W) < 0.99 * best) {
-                    best = cost(W);
-                    items_per_cta = W;
-                }
-            target = groups_of(items_per_cta);
-        }
-    }
     const int64_t num_groups = std::max<int64_t>(1, std::min<int64_t>(target, total_tiles));
 
     plan = Plan{};
@@ -212,13 +190,7 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     info.tile_m = tile_m;
     info.m_tiles = m_tiles;
     info.num_groups = (int32_t)num_groups;
-    {
-        // every CTA runs ceil(items / sm_count) items at most (one, except in the two-tile chunk kernel)
-        const int64_t items = num_groups * m_tiles;
-        const int64_t per_cta = mode == YOCO_MODE_CHUNK && tile_m == kChunkPairTileM
-                                    ? std::max<int64_t>(1, (items + sm_count - 1) / sm_count) : 1;
-        info.num_ctas = (int32_t)((items + per_cta - 1) / per_cta);
-    }
+    info.num_ctas = (int32_t)(num_groups * m_tiles);
     info.num_streams = num_streams;
     info.num_segments = (int32_t)plan.segments.size();
     info.sub_items = R;

@@ -97,20 +97,3 @@ def test_two_runs_are_bit_identical():
     a = O1.clone()
     _, _, O2 = r.run(Q, "chunk")
     assert torch.equal(a.view(torch.int16), O2.view(torch.int16))
-
-
-@pytest.mark.parametrize("Hq,Hkv,T,lens", [
-    (8, 2, 512, [4000, 2500]),      # 8 row-tile pairs per stream: 37 groups, every CTA runs two items
-    (4, 1, 300, [8000]),            # 5 pairs (the last one ragged): 59 groups on 148 CTAs
-    (16, 4, 300, [1500, 2700]),     # 5 pairs, groups that straddle heads and the two sequences
-])
-def test_ctas_that_run_several_items(Hq, Hkv, T, lens):
-    """Streams with many 256-row tile pairs: the plan gives a CTA of the two-tile kernel more than one
-    (group, pair) item, so it changes Q tiles, row offsets and causal limits between segments."""
-    import torch
-    from paper_2405_05254_b200 import binding as bd
-    w = si.Workload("items", B=len(lens), Hq=Hq, Hkv=Hkv, d=128, T=T, layers=1, seed=36, kv_len=lens)
-    sm = torch.cuda.get_device_properties(0).multi_processor_count
-    info, _ = bd.yoco_xattn_plan(bd.make_shape(w.B, Hq, Hkv, 128, T), w.kv_len, sm, bd.MODE_CHUNK)
-    assert info.tile_m == 256 and info.num_ctas < info.num_groups * info.m_tiles <= 4 * info.num_ctas
-    run_chunk(w)

@@ -46,15 +46,6 @@ def restated_plan(B, Hkv, lens, sm_count, mode, G, T):
     nts = [-(-int(n) // tile_n) for n in lens]
     total = Hkv * sum(nts)
     target = sm_count * 2 if mode == bd.MODE_DECODE else max(1, sm_count // m_tiles)
-    if mode == bd.MODE_CHUNK and tile_m == 256:
-        # a CTA of the two-tile kernel may run W items: W * sm / m_tiles groups, time ~ ceil(items / sm) / groups
-        groups_of = lambda W: max(1, min(W * sm_count // m_tiles, max(total, 1)))       # noqa: E731
-        cost = lambda W: -(-groups_of(W) * m_tiles // sm_count) / groups_of(W)          # noqa: E731
-        best, pick = cost(1), 1
-        for W in (2, 3, 4):
-            if cost(W) < 0.99 * best:
-                best, pick = cost(W), W
-        target = groups_of(pick)
     groups = max(1, min(target, total))
     bounds = [p * total // groups for p in range(groups + 1)]
     segs = []
@@ -118,7 +109,6 @@ CASES = [
     dict(B=3, Hq=24, Hkv=8, d=128, T=2, lens=[1, 0, 65]),
     dict(B=2, Hq=32, Hkv=8, d=128, T=512, lens=[262656, 262656]),
     dict(B=2, Hq=32, Hkv=8, d=128, T=160, lens=[1160, 937]),
-    dict(B=1, Hq=32, Hkv=8, d=128, T=2000, lens=[50000]),       # 32 row-tile pairs: two items per CTA
 ]
 
 
@@ -133,9 +123,7 @@ def test_plan_partitions_every_stream_exactly(case, sm_count):
         groups, m_tiles, want, want_slots, R, coarse = restated_plan(case["B"], case["Hkv"], case["lens"], sm_count,
                                                                      mode, G, case["T"])
         assert info.num_groups == groups and info.m_tiles == m_tiles
-        items = groups * m_tiles
-        per_cta = max(1, -(-items // sm_count)) if (mode == bd.MODE_CHUNK and info.tile_m == 256) else 1
-        assert info.num_ctas == -(-items // per_cta) and (per_cta == 1 or info.num_ctas <= sm_count)
+        assert info.num_ctas == groups * m_tiles
         assert info.sub_items == R and info.num_slots == coarse * R
         got = [(s.group, s.b, s.c, s.k_begin, s.k_end) for s in segs]
         assert got == want                                     # integer for integer
