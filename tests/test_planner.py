@@ -290,3 +290,32 @@ def test_new_entry_points_validate_arguments_before_touching_cuda():
     assert L.yoco_xattn_decode_partial(ctypes.byref(shape2), p(16), p(16), p(16), None, None, p(16), p(16), p(256),
                                        1 << 20, None) == bd.ERR_UNSUPPORTED                # T = 2
     assert L.yoco_xattn_combine_gathered(4, 0, 128, None, None, None, None, None) == bd.ERR_INVALID_ARG
+
+
+def test_public_header_is_plain_c_and_cxx(tmp_path):
+    """The boundary is a C ABI: the header must compile on its own as C99 and as C++11, warnings
+    as errors, and a C program must be able to link the planner (a pure host call) from the library."""
+    import shutil
+    import subprocess
+    inc = os.path.join(ROOT, "include")
+    src = tmp_path / "use.c"
+    src.write_text('#include "yoco_xattn.h"\n#include <stdio.h>\n#include <string.h>\n'
+                   'int main(void) {\n'
+                   '    yoco_xattn_shape s;\n    yoco_xattn_plan_info info;\n    int32_t len = 1048576;\n'
+                   '    memset(&s, 0, sizeof s);\n'
+                   '    s.B = 1; s.Hq = 32; s.Hkv = 8; s.d = 128; s.T = 1; s.max_kv_len = len;\n'
+                   '    int32_t rc = yoco_xattn_plan(&s, &len, 148, YOCO_MODE_DECODE, &info, 0, 0);\n'
+                   '    printf("%d %d %d %d\\n", (int)rc, (int)info.num_groups, (int)info.sub_items, (int)info.num_slots);\n'
+                   '    return rc;\n}\n')
+    for cc, std in (("gcc", "-std=c99"), ("g++", "-std=c++11")):
+        if shutil.which(cc) is None:
+            pytest.skip(f"{cc} not installed")
+        lang = ["-x", "c++"] if cc == "g++" else []
+        subprocess.run([cc, std, "-Wall", "-Wextra", "-Werror", "-pedantic", "-fsyntax-only", "-I", inc] + lang + [str(src)],
+                       check=True)
+    exe = tmp_path / "use"
+    libdir, libname = os.path.split(bd.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-I", inc, str(src), "-o", str(exe), os.path.join(libdir, libname),
+                    f"-Wl,-rpath,{libdir}"], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
+    assert out == ["0", "296", "4", "1184"]
