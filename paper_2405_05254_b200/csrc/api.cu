@@ -256,10 +256,12 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
     float* part_o = reinterpret_cast<float*>(ws + plan.ws_part_o);
     int32_t* status = reinterpret_cast<int32_t*>(ws);
 
+    bool timed = false;   // an event pair was put around the attention kernel of this call
     if (plan.info.num_segments > 0) {
         bool prof = false;
         cudaEvent_t ev = prof_event(false, &prof);
         if (prof) YOCO_CUDA_TRY(cudaEventRecord(ev, stream));
+        timed = prof;
         if (mode == YOCO_MODE_DECODE) {
             CUtensorMap tmK, tmV;
             if (fp8) {
@@ -351,7 +353,7 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
         c.merge_unsplit = part_out ? 1 : 0;
         // directly behind the attention kernel (no event in between): its launch may overlap
         // that kernel's tail
-        const bool chained = plan.info.num_segments > 0 && g_prof.events.empty();
+        const bool chained = plan.info.num_segments > 0 && !timed;
         YOCO_CUDA_TRY(launch_combine(c, stream, inline_tables ? &ready->combine_tab : nullptr, chained));
     }
     return YOCO_OK;
