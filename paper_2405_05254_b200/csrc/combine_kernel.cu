@@ -65,6 +65,21 @@ __device__ __forceinline__ void combine_body(const CombineParams& p) {
         }
     }
 
+    // The partial rows this warp will need do not depend on the weights: ask for the first U of them
+    // now, so that they travel while the log-sum-exps are read and reduced (one memory round trip
+    // instead of two or more; U covers all of a warp's pieces in the launch shapes used).
+    constexpr int U = WPR == 1 ? 4 : (WARPS == kCombineWarpsMany ? 2 : 10);
+    const int e0 = lane * 4;
+    float4 pre[U][2];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int s = sub + u * WPR;
+#pragma unroll
+        for (int blk = 0; blk < 2; ++blk)
+            if (s < nseg && e0 + blk * 128 < p.d)
+                pre[u][blk] = *reinterpret_cast<const float4*>(p.part_o + o_base + s * o_stride + e0 + blk * 128);
+    }
+
     float m = -INFINITY;
     for (int s = lane; s < nseg; s += 32) m = fmaxf(m, p.part_lse[lse_base + s * lse_stride]);
 #pragma unroll
@@ -93,9 +108,27 @@ __device__ __forceinline__ void combine_body(const CombineParams& p) {
 
     // each lane owns 4 consecutive channels of each 128-channel block (d <= 256: two blocks)
     float4 acc[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
-    const int e0 = lane * 4;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int s = sub + u * WPR;
+        if (s < nseg) {
+            const float l = p.part_lse[lse_base + s * lse_stride];
+            const float w = l == -INFINITY ? 0.f : __expf(l - m) * inv;
+#pragma unroll
+            for (int blk = 0; blk < 2; ++blk) {
+                if (e0 + blk * 128 < p.d) {
+                    const float4 v = pre[u][blk];
+                    // an empty piece may hold anything: select, never multiply by zero
+                    acc[blk].x += w != 0.f ? w * v.x : 0.f;
+                    acc[blk].y += w != 0.f ? w * v.y : 0.f;
+                    acc[blk].z += w != 0.f ? w * v.z : 0.f;
+                    acc[blk].w += w != 0.f ? w * v.w : 0.f;
+                }
+            }
+        }
+    }
 #pragma unroll 4
-    for (int s = sub; s < nseg; s += WPR) {
+    for (int s = sub + U * WPR; s < nseg; s += WPR) {
         const float l = p.part_lse[lse_base + s * lse_stride];
         const float w = l == -INFINITY ? 0.f : __expf(l - m) * inv;
         const float* src = p.part_o + o_base + s * o_stride;
