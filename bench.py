@@ -322,7 +322,7 @@ def measure_kv_append(dev, peaks, hbm_peak):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         for k in range(n):
             flush.fill_(k)                       # weights (16.8 MB) would otherwise stay in L2
-            flush.view(torch.int32).sum()        # ... and a read pass, so that L2 is left clean: the write-back
+            flush.view(torch.float32).sum()      # ... and a read pass, so that L2 is left clean: the write-back
                                                  # of ~126 MB of dirty flush lines would otherwise land in the call
             e0.record()
             bd.yoco_kv_append(shape, X, Wgk, Wgv, K, V, None, lens)
