@@ -3,7 +3,7 @@ import numpy as np
 
 import synth_inputs as si
 
-MAX_ABS_TOL = 1e-2     # bf16 in, fp32 accumulate (the tolerance the benchmark spec fixes)
+MAX_ABS_TOL = 1e-2     # bf16 in, fp32 accumulate: max-abs 1e-2 and relative L2 5e-3 against the fp64 oracle
 REL_L2_TOL = 5e-3
 LSE_ABS_TOL = 2e-3
 GUARD = 4096           # sentinel elements on both sides of every output buffer
