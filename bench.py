@@ -118,13 +118,21 @@ def oracle_sample_rate(w, Q_layers, K, V, seconds_hint=None):
     key of that head): returns (KV GB/s, seconds, description, threads)."""
     import oracle
     G = w.Hq // w.Hkv
-    rows = np.array([(b, h, t) for b in range(w.B) for h in range(G) for t in range(w.T)], dtype=np.int32)
+    heads = sample_kv_heads(w)
+    rows = np.array([(b, h, t) for b in range(w.B) for h in range(heads * G) for t in range(w.T)], dtype=np.int32)
     t0 = time.perf_counter()
     oracle.xattn_rows(Q_layers[0], K, V, w.cu, w.kv_len, rows, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T)
     dt = time.perf_counter() - t0
-    sample_bytes = w.kv_bytes / w.Hkv
-    return sample_bytes / dt / 1e9, dt, (f"one layer call restricted to KV head 0 ({G} query heads x all "
-                                         f"{w.total_tokens} keys = 1/{w.Hkv} of a layer call)"), oracle.num_threads()
+    sample_bytes = w.kv_bytes * heads / w.Hkv
+    return sample_bytes / dt / 1e9, dt, (f"one layer call restricted to KV heads 0..{heads - 1} ({heads * G} query heads x "
+                                         f"all {w.total_tokens} keys = {heads}/{w.Hkv} of a layer call)"), oracle.num_threads()
+
+
+def sample_kv_heads(w, madds=2e10):
+    """KV heads in the oracle's timed sample: about `madds` multiply-adds (2e10: 10-30 s of CPU work spread over
+    the host's cores), never more than the workload has."""
+    per_head = (w.Hq // w.Hkv) * w.T * w.total_tokens * w.d * 2
+    return int(max(1, min(w.Hkv, round(madds / max(per_head, 1)))))
 
 
 def run_reference(args):
@@ -137,9 +145,11 @@ def run_reference(args):
     K, V = w.make_k(), w.make_v()
     Qs = [w.make_q(l) for l in range(w.layers)]
     G = w.Hq // w.Hkv
-    rows = np.array([(b, h, t) for b in range(w.B) for h in range(G) for t in range(w.T)], dtype=np.int32)
+    # every step is one sample; steps + warm-up of them must end within a few minutes
+    heads = sample_kv_heads(w, madds=2e11 / max(args.steps + args.warmup, 1))
+    rows = np.array([(b, h, t) for b in range(w.B) for h in range(heads * G) for t in range(w.T)], dtype=np.int32)
     kw = dict(B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T)
-    sample_bytes = w.kv_bytes / w.Hkv
+    sample_bytes = w.kv_bytes * heads / w.Hkv
 
     def step(k):
         oracle.xattn_rows(Qs[k % w.layers], K, V, w.cu, w.kv_len, rows, **kw)
@@ -152,12 +162,12 @@ def run_reference(args):
     dt = time.perf_counter() - t0
     per_sample = dt / args.steps
     gbs = sample_bytes / per_sample / 1e9
-    us_tl = per_sample * w.Hkv / w.B * 1e6
-    sample = (f"each step = one layer call restricted to KV head 0 ({G} query heads x all "
-              f"{w.total_tokens} keys, 1/{w.Hkv} of a layer call); ms_per_step extrapolated x{w.Hkv} x{w.layers} layers")
+    us_tl = per_sample * w.Hkv / heads / w.B * 1e6
+    sample = (f"each step = one layer call restricted to KV heads 0..{heads - 1} ({heads * G} query heads x all "
+              f"{w.total_tokens} keys, {heads}/{w.Hkv} of a layer call); ms_per_step extrapolated x{w.Hkv}/{heads} x{w.layers} layers")
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_sample * w.Hkv * w.layers * 1e3,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_sample * w.Hkv / heads * w.layers * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "us_per_token_layer": us_tl,
         "config": workload_config(w, 1),
@@ -611,7 +621,7 @@ def run_ours(args):
             gbs, dt, sample, cores = oracle_sample_rate(w, Qh, Kh, Vh)
             line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
                                     "sample": sample, "seconds": dt,
-                                    "us_per_token_layer": dt * w.Hkv / w.B * 1e6}
+                                    "us_per_token_layer": dt * w.Hkv / sample_kv_heads(w) / w.B * 1e6}
         print(json.dumps(line), flush=True)
     if world > 1:
         torch.distributed.destroy_process_group()
