@@ -306,15 +306,23 @@ kv_append_small_kernel(const __grid_constant__ CUtensorMap tmWk, const __grid_co
     float sq = 0.f;                                         // this thread's share of a row's sum of squares
     const int xr = threadIdx.x >> 3, xc = (threadIdx.x & 7) * 16;   // X staging: row, first of 16 elements
 
+    // this thread's 16 elements of X[:, chunk]; the next chunk's are requested one iteration ahead, so
+    // that only the first load's latency is exposed
+    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+    const uint4* xsrc = reinterpret_cast<const uint4*>(p.X + (int64_t)(xr < p.M ? xr : 0) * p.d_model + k_base + xc);
+    uint4 v0 = zero4, v1 = zero4;
+    if (xr < p.M && n_chunks > 0) {
+        v0 = xsrc[0];
+        v1 = xsrc[1];
+    }
     for (int c = 0; c < n_chunks; ++c) {
         // X[:, chunk] -> shared memory (rows beyond M are zero), squares on the way
+        uint4 nv0 = zero4, nv1 = zero4;
+        if (xr < p.M && c + 1 < n_chunks) {
+            nv0 = xsrc[(c + 1) * (SK_KBOX / 8)];
+            nv1 = xsrc[(c + 1) * (SK_KBOX / 8) + 1];
+        }
         {
-            uint4 v0 = make_uint4(0u, 0u, 0u, 0u), v1 = v0;
-            if (xr < p.M) {
-                const uint4* src = reinterpret_cast<const uint4*>(p.X + (int64_t)xr * p.d_model + k_base + c * SK_KBOX + xc);
-                v0 = src[0];
-                v1 = src[1];
-            }
             const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -357,6 +365,8 @@ kv_append_small_kernel(const __grid_constant__ CUtensorMap tmWk, const __grid_co
             mbar_expect_tx(&full[stage], HALF_BYTES);
             tma_load_2d(smem + stage * HALF_BYTES, tmW, col0, k_base + (c + SK_STAGES) * SK_KBOX, &full[stage]);
         }
+        v0 = nv0;
+        v1 = nv1;
     }
 
     // partial results of this CTA -> its shared memory
