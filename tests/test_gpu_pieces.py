@@ -101,3 +101,38 @@ def test_partial_entry_point_in_pieces():
     o_ref, lse_ref = oracle.xattn(Q, K, V, w.cu, w.kv_len, B=1, Hq=32, Hkv=8, d=128, T=1)
     assert_close(po.cpu().numpy().astype(np.float64).reshape(1, 32, 1, 128), o_ref, "partial in pieces")
     assert_lse_close(pl.cpu().numpy().reshape(1, 32, 1), lse_ref, "partial in pieces")
+
+
+def test_two_streams_running_pieces_at_once_keep_their_bits():
+    """Two long-cache decode problems, each with its own workspace, enqueued on two streams so that their
+    grids share the SMs (neither has all its CTAs resident at once): every CTA still runs piece 0 of its
+    group whenever it starts, the rest is handed out, and both results stay bit-identical to a solo run."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    probs = []
+    for seed, N in ((41, 300000), (42, 180000)):
+        w = si.Workload("two", B=1, Hq=32, Hkv=8, d=128, T=1, layers=1, seed=seed, kv_len=[N])
+        shape = bd.make_shape(1, 32, 8, 128, 1, max_kv_len=N)
+        ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_DECODE), dtype=torch.uint8, device="cuda")
+        probs.append(dict(shape=shape, K=to_dev_bf16(w.make_k()), V=to_dev_bf16(w.make_v()),
+                          Q=to_dev_bf16(w.make_q(0).reshape(-1)), lens=w.kv_len, ws=ws,
+                          O=torch.empty(32 * 128, dtype=torch.bfloat16, device="cuda")))
+
+    def call(x, stream=None):
+        bd.yoco_xattn_decode(x["shape"], x["Q"], x["K"], x["V"], None, x["lens"], x["O"], None, x["ws"], stream)
+
+    for x in probs:
+        call(x)
+    torch.cuda.synchronize()
+    solo = [x["O"].view(torch.int16).clone() for x in probs]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for _ in range(3):
+        for x, s, n in zip(probs, streams, (6, 10)):
+            x["O"].zero_()
+            with torch.cuda.stream(s):
+                for _ in range(n):
+                    call(x, s)
+        torch.cuda.synchronize()
+        for x, ref in zip(probs, solo):
+            assert bd.yoco_xattn_status(x["ws"]) == 0
+            assert torch.equal(x["O"].view(torch.int16), ref)
