@@ -143,7 +143,11 @@ int32_t yoco_xattn_workspace_size(const yoco_xattn_shape* shape, const int32_t* 
  * whole cache.  Runs the split kernel, then the merge when a stream was split.
  *   Q, K, V, O, lse (may be NULL), workspace: device.  cu_kv_host: host [B+1] token
  *   offsets, or NULL = prefix sums of kv_len (tight packing).  kv_len_host: host [B]
- *   or NULL.  workspace: >= yoco_xattn_workspace_size(), 256-byte aligned.        */
+ *   or NULL.  workspace: >= yoco_xattn_workspace_size(), 256-byte aligned; it holds the
+ *   status word, the work counter of the run-time piece assignment, the work tables and the
+ *   partial results of THIS call: successive calls on one stream may share it (the 13 layer
+ *   calls of a step do), calls that can overlap on the GPU need one each.  Its contents need
+ *   no initialisation and mean nothing after the call except to yoco_xattn_status.   */
 int32_t yoco_xattn_decode(const yoco_xattn_shape* shape, const void* Q, const void* K,
                           const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
                           void* O, float* lse, void* workspace, size_t workspace_bytes,
