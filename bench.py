@@ -188,6 +188,44 @@ def workload_config(w, n_gpus):
             "parallelism": f"replicas x{n_gpus} (one cache per GPU, no collective)"}
 
 
+def measure_few_rows(dev, w, K, V, peak_gbs, peaks):
+    """The multi-token entry point with a few new rows per head over the headline cache (verification of
+    drafted tokens: T = 8, 16, 32, i.e. 32-128 rows per KV head, the one-tile tcgen05 kernel): up to T of
+    about 55 the call streams K/V once and is bound by HBM, like decode."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    out = {}
+    for T in (8, 16, 32):
+        shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, T, max_kv_len=int(w.kv_len.max()))
+        ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_CHUNK), dtype=torch.uint8, device=dev)
+        Q = torch.empty(w.B * w.Hq * T * w.d, dtype=torch.bfloat16, device=dev).normal_()
+        O = torch.empty_like(Q)
+        for _ in range(3):
+            bd.yoco_xattn_chunk(shape, Q, K, V, w.cu, w.kv_len, O, None, ws)
+        assert bd.yoco_xattn_status(ws) == 0
+        n = 10
+        bd.yoco_xattn_profile_enable(n)
+        for _ in range(n):
+            bd.yoco_xattn_chunk(shape, Q, K, V, w.cu, w.kv_len, O, None, ws)
+        k_us = float(bd.yoco_xattn_profile_collect(n).mean()) * 1e3
+        bd.yoco_xattn_profile_enable(0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            bd.yoco_xattn_chunk(shape, Q, K, V, w.cu, w.kv_len, O, None, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        call_us = e0.elapsed_time(e1) * 1e3 / n
+        flop = sum(w.Hq * (T * (int(nk) - T) + T * (T + 1) / 2) * 4 * w.d for nk in w.kv_len)
+        out[f"T={T}"] = {"rows_per_kv_head": (w.Hq // w.Hkv) * T, "kernel_us": k_us, "call_us": call_us,
+                         "bound": "hbm", "achieved": w.kv_bytes / k_us / 1e3, "unit": "GB/s", "peak": peak_gbs,
+                         "frac": w.kv_bytes / k_us / 1e3 / peak_gbs, "tflops": flop / k_us / 1e6,
+                         "frac_of_bf16_burst": flop / k_us / 1e6 / float(peaks.get("bf16_tflops", 1590.0))}
+    out["workload"] = f"{w.name}: B={w.B} Hq={w.Hq} Hkv={w.Hkv} d={w.d} kv_len={int(w.kv_len.max())}, T new rows per sequence"
+    out["algorithmic_bytes_per_launch"] = w.kv_bytes
+    return out
+
+
 def measure_chunk(dev, peaks, name="chunk"):
     """The multi-token path on its own workload (512 new rows after 262,144 cached keys, B = 2):
     achieved TFLOP/s of the tcgen05 kernel against the measured bf16 peaks."""
@@ -612,6 +650,8 @@ def run_ours(args):
             line["fp8_cache"] = measure_fp8_cache(dev, w, Qd[0], peak)
         if world == 1 and w.B == 1 and w.T == 1 and not args.no_shard:
             line["key_range_shard"] = measure_key_range_shard(dev, w, K, V, Qd[0])
+        if world == 1 and not args.no_chunk and w.T == 1:
+            line["chunk_few_rows"] = measure_few_rows(dev, w, K, V, peak, peaks)
         if world == 1 and not args.no_chunk:
             del K, V
             torch.cuda.empty_cache()
