@@ -60,7 +60,7 @@ extern "C" {
 #define YOCO_ERR_TIMEOUT              (-5)  /* a bounded device-side wait expired               */
 #define YOCO_ERR_STATIC_SCRATCH_EXCEEDED (-6) /* yoco_xattn_decode_static: problem too large    */
 
-#define YOCO_MODE_DECODE 0   /* split-KV kernel, G*T <= 32 query rows per KV head        */
+#define YOCO_MODE_DECODE 0   /* split-KV kernel, G*T <= 16 query rows per KV head        */
 #define YOCO_MODE_CHUNK  1   /* tensor-core (tcgen05) kernel, any T >= 1                 */
 
 typedef struct yoco_xattn_shape {
@@ -138,7 +138,7 @@ int64_t yoco_xattn_sub_bound(int64_t n_tiles, int32_t sub_items, int32_t r);
 int32_t yoco_xattn_workspace_size(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
                                   int32_t sm_count, int32_t mode, size_t* bytes);
 
-/* Split-KV decode (flash-decoding style): a few query rows per KV head (G*T <= 32;
+/* Split-KV decode (flash-decoding style): a few query rows per KV head (G*T <= 16;
  * typically T = 1, the next-token call of a cross-decoder layer) against the
  * whole cache.  Runs the split kernel, then the merge when a stream was split.
  *   Q, K, V, O, lse (may be NULL), workspace: device.  cu_kv_host: host [B+1] token

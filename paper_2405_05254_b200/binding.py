@@ -156,7 +156,7 @@ def _run(fn_name, shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream):
 
 
 def yoco_xattn_decode(shape: Shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream=None) -> None:
-    """Enqueue split-KV decode attention (G*T <= 32 rows per KV head) on the stream."""
+    """Enqueue split-KV decode attention (G*T <= 16 rows per KV head) on the stream."""
     _run("yoco_xattn_decode", shape, Q, K, V, cu_kv, kv_len, O, lse, workspace, stream)
 
 

@@ -513,8 +513,6 @@ int32_t yoco_xattn_decode_fp8(const yoco_xattn_shape* shape, const void* Q, cons
                               size_t workspace_bytes, void* stream) {
     if (!shape || !k_scale_host || !v_scale_host) return YOCO_ERR_INVALID_ARG;
     if (shape->d != 128 || shape->Hkv > kFp8MaxHeads) return YOCO_ERR_UNSUPPORTED;
-    if ((int64_t)(shape->Hq / (shape->Hkv > 0 ? shape->Hkv : 1)) * shape->T > kDecodeTileM)
-        return YOCO_ERR_UNSUPPORTED;   // the 8-bit kernel holds one 16-row tile
     for (int c = 0; c < shape->Hkv; ++c)
         if (!(k_scale_host[c] > 0.f) || !(v_scale_host[c] > 0.f) || !std::isfinite(k_scale_host[c]) ||
             !std::isfinite(v_scale_host[c]))

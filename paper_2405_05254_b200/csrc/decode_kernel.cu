@@ -5,8 +5,7 @@
 // ring of mbarrier-guarded stages; four consumer warps each take 16 keys of every tile and
 // keep their own online-softmax state, so there is no CTA-wide synchronisation inside the
 // key loop.  All G = Hq/Hkv query heads of the group (and the T rows of each) form the
-// <= 16 rows of one mma.sync tile (or, for 17-32 rows, of two tiles that two pairs of warps share
-// out), so one K/V read from HBM serves the whole group.
+// <= 16 rows of one mma.sync tile, so one K/V read from HBM serves the whole group.
 // The arithmetic intensity is 4*G flop per K/V byte: far below the ridge, the kernel is
 // bound by HBM bandwidth; the small matrix products go through mma.sync (bf16 in, fp32
 // accumulate) only to keep the issue slots free for the memory pipeline.
@@ -35,11 +34,8 @@ struct Cfg {
     static constexpr int HALVES = D / 64;
     static constexpr int TENSOR_BYTES = HALVES * HALF_BYTES;
     static constexpr int STAGE_BYTES = 2 * TENSOR_BYTES;
-    // ROWS = 8 or 16: one MMA row tile, each warp takes 16 keys of every tile.  ROWS = 32: two row
-    // tiles; warps 0-1 own rows 0-15, warps 2-3 rows 16-31, each with 32 keys of every tile.
-    static constexpr int MROWS = ROWS > 16 ? 16 : ROWS;            // rows of the MMA tile a warp holds
-    static constexpr int MERGE_O_BYTES = kConsumerWarps * MROWS * D * 4;
-    static constexpr int MERGE_ML_BYTES = kConsumerWarps * MROWS * 2 * 4;
+    static constexpr int MERGE_O_BYTES = kConsumerWarps * ROWS * D * 4;
+    static constexpr int MERGE_ML_BYTES = kConsumerWarps * ROWS * 2 * 4;
     // two CTAs per SM: (228 KB - 2 x 1 KB reserved) / 2 = 113 KB each
     static constexpr int BUDGET = 113 * 1024;
     static constexpr int STAGES_FIT = (BUDGET - MERGE_O_BYTES - MERGE_ML_BYTES - 128) / STAGE_BYTES;
@@ -61,9 +57,6 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
     constexpr int STAGES = C::STAGES;
     constexpr int KSTEPS = D / 16;
     constexpr int NT_O = D / 8;
-    constexpr bool WIDE = ROWS > 16;          // two row tiles, two warps each
-    constexpr int MROWS = C::MROWS;
-    constexpr int NSL = WIDE ? 2 : 1;         // 16-key slices of a tile per warp
 
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* stage_mem = smem;
@@ -166,7 +159,6 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
     // ----------------------------------- consumers ---------------------------------------
     const int g = lane >> 2, tq = lane & 3;
     const int n_rows = p.rows_per_stream;
-    const int row_off = WIDE ? (warp >> 1) * 16 : 0;      // first row of this warp's MMA tile
     uint32_t it = 0;
     bool ok = true;
 
@@ -210,9 +202,9 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
             // Q as the A operand of m16n8k16: rows = (head in group, t), zero beyond n_rows
             uint32_t qa[KSTEPS][4];
             {
-                const __nv_bfloat16* q0 = p.Q + ((int64_t)seg.q_row0 + row_off + g) * D + tq * 2;
+                const __nv_bfloat16* q0 = p.Q + ((int64_t)seg.q_row0 + g) * D + tq * 2;
                 const __nv_bfloat16* q1 = q0 + 8 * D;
-                const bool v0 = row_off + g < n_rows, v1 = MROWS == 16 && (row_off + g + 8) < n_rows;
+                const bool v0 = g < n_rows, v1 = ROWS == 16 && (g + 8) < n_rows;
 #pragma unroll
                 for (int ks = 0; ks < KSTEPS; ++ks) {
                     qa[ks][0] = v0 ? ld_global_u32(q0 + ks * 16) : 0u;
@@ -223,8 +215,8 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
             }
             // causal limits: row t sees keys j < n_kv - T + 1 + t
             const int n_full = seg.n_kv - p.T + 1;
-            const int vis0 = min(seg.n_kv, max(0, n_full + ((row_off + g) % p.T)));
-            const int vis1 = min(seg.n_kv, max(0, n_full + ((row_off + g + 8) % p.T)));
+            const int vis0 = min(seg.n_kv, max(0, n_full + (g % p.T)));
+            const int vis1 = min(seg.n_kv, max(0, n_full + ((g + 8) % p.T)));
 
             float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
             float o[NT_O][4];
@@ -239,129 +231,124 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
                     ok = false;
                     continue;
                 }
-                // a warp takes one 16-key slice of the tile, or two when there are two row tiles
-#pragma unroll
-                for (int sl = 0; sl < NSL; ++sl) {
-                    const int slice = WIDE ? (warp & 1) * 2 + sl : warp;
-                    const int kw = k0 + slice * 16;          // first key of the slice
-                    if (kw < k_hi) {
-                        const uint32_t kbase = smem_u32(stage_mem + stage * C::STAGE_BYTES);
-                        const uint32_t vbase = kbase + C::TENSOR_BYTES;
+                const int kw = k0 + warp * 16;          // first key of this warp's slice
+                if (kw < k_hi) {
+                    const uint32_t kbase = smem_u32(stage_mem + stage * C::STAGE_BYTES);
+                    const uint32_t vbase = kbase + C::TENSOR_BYTES;
 
-                        // ---- S = Q K^T for 16 keys (two n-tiles of 8 keys) ----
-                        float s[2][4];
+                    // ---- S = Q K^T for 16 keys (two n-tiles of 8 keys) ----
+                    float s[2][4];
 #pragma unroll
-                        for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-                        {
-                            const int key_l = slice * 16 + (lane >> 4) * 8 + (lane & 7);
-                            const int sel = (lane >> 3) & 1;
-                            const uint32_t rowaddr = kbase + key_l * 128;
+                    for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+                    {
+                        const int key_l = warp * 16 + (lane >> 4) * 8 + (lane & 7);
+                        const int sel = (lane >> 3) & 1;
+                        const uint32_t rowaddr = kbase + key_l * 128;
 #pragma unroll
-                            for (int ks = 0; ks < KSTEPS; ++ks) {
-                                const int c = 2 * ks + sel;
-                                const uint32_t addr =
-                                    rowaddr + (c >> 3) * HALF_BYTES + ((((c & 7) ^ key_l) & 7) << 4);
-                                uint32_t b0, b1, b2, b3;
-                                ldmatrix_x4(addr, b0, b1, b2, b3);
-                                mma_bf16_16816(s[0], qa[ks], b0, b1);
-                                mma_bf16_16816(s[1], qa[ks], b2, b3);
-                            }
+                        for (int ks = 0; ks < KSTEPS; ++ks) {
+                            const int c = 2 * ks + sel;
+                            const uint32_t addr =
+                                rowaddr + (c >> 3) * HALF_BYTES + ((((c & 7) ^ key_l) & 7) << 4);
+                            uint32_t b0, b1, b2, b3;
+                            ldmatrix_x4(addr, b0, b1, b2, b3);
+                            mma_bf16_16816(s[0], qa[ks], b0, b1);
+                            mma_bf16_16816(s[1], qa[ks], b2, b3);
                         }
-                        // ---- scale, mask, online softmax ----
-                        // sliding window: the row at position i = n_kv - T + t keeps i - C < j, i.e.
-                        // j >= i - C + 1 = n_full + t - C; the highest such bound of any row is n_kv - C
-                        const bool need_mask = kw + 16 > n_full || (p.window > 0 && kw < seg.n_kv - p.window);
-                        // window start of the two rows this lane holds (no window: below every key)
-                        int lo0 = -1, lo1 = -1;
-                        if (need_mask && p.window > 0) {
-                            lo0 = n_full + ((row_off + g) % p.T) - p.window;
-                            lo1 = n_full + ((row_off + g + 8) % p.T) - p.window;
-                        }
-#pragma unroll
-                        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                float v = s[nt][e] * p.scale_log2;
-                                if (need_mask) {
-                                    const int j = kw + nt * 8 + tq * 2 + (e & 1);
-                                    v = (j < ((e & 2) ? vis1 : vis0) && j >= ((e & 2) ? lo1 : lo0)) ? v : -INFINITY;
-                                }
-                                s[nt][e] = v;
-                            }
-                        float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-                        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-                        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-                        const float mn0 = fmaxf(m0, mx0);
-                        const float ms0 = mn0 == -INFINITY ? 0.f : mn0;
-                        const float alpha0 = exp2f(m0 - ms0);
-                        m0 = mn0;
-                        float alpha1 = 1.f, ms1 = 0.f;
-                        if (MROWS == 16) {
-                            float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
-                            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-                            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-                            const float mn1 = fmaxf(m1, mx1);
-                            ms1 = mn1 == -INFINITY ? 0.f : mn1;
-                            alpha1 = exp2f(m1 - ms1);
-                            m1 = mn1;
-                        }
-                        uint32_t pa[4];
-                        {
-                            const float p00 = exp2f(s[0][0] - ms0), p01 = exp2f(s[0][1] - ms0);
-                            const float p10 = exp2f(s[1][0] - ms0), p11 = exp2f(s[1][1] - ms0);
-                            l0 = l0 * alpha0 + ((p00 + p01) + (p10 + p11));
-                            pa[0] = pack_bf16x2(p00, p01);
-                            pa[2] = pack_bf16x2(p10, p11);
-                            if (MROWS == 16) {
-                                const float q00 = exp2f(s[0][2] - ms1), q01 = exp2f(s[0][3] - ms1);
-                                const float q10 = exp2f(s[1][2] - ms1), q11 = exp2f(s[1][3] - ms1);
-                                l1 = l1 * alpha1 + ((q00 + q01) + (q10 + q11));
-                                pa[1] = pack_bf16x2(q00, q01);
-                                pa[3] = pack_bf16x2(q10, q11);
-                            } else {
-                                pa[1] = pa[3] = 0u;
-                            }
-                        }
-                        if (__any_sync(0xffffffffu, alpha0 != 1.f || alpha1 != 1.f)) {
-#pragma unroll
-                            for (int nt = 0; nt < NT_O; ++nt) {
-                                o[nt][0] *= alpha0; o[nt][1] *= alpha0;
-                                o[nt][2] *= alpha1; o[nt][3] *= alpha1;
-                            }
-                        }
-                        // ---- rows past the end of the sequence may hold anything: zero them so that
-                        //      0 * garbage cannot produce NaN in O += P V ----
-                        if (kw + 16 > seg.n_kv) {
-                            const int first_bad = max(seg.n_kv - kw, 0);          // 0..15
-                            uint8_t* vrow = stage_mem + stage * C::STAGE_BYTES + C::TENSOR_BYTES;
-                            for (int r = first_bad; r < 16; ++r) {
-                                const int key_l = slice * 16 + r;
-                                for (int b = lane * 16; b < C::HALVES * 128; b += 512) {
-                                    const int h = b >> 7, off = b & 127;
-                                    *reinterpret_cast<uint4*>(vrow + h * HALF_BYTES + key_l * 128 + off) =
-                                        make_uint4(0u, 0u, 0u, 0u);
-                                }
-                            }
-                            __syncwarp();
-                        }
-                        // ---- O += P V ----
-                        {
-                            const int key_l = slice * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
-                            const int sel = lane >> 4;
-                            const uint32_t rowaddr = vbase + key_l * 128;
-#pragma unroll
-                            for (int nt = 0; nt < NT_O; nt += 2) {
-                                const int c = nt + sel;
-                                const uint32_t addr =
-                                    rowaddr + (c >> 3) * HALF_BYTES + ((((c & 7) ^ key_l) & 7) << 4);
-                                uint32_t b0, b1, b2, b3;
-                                ldmatrix_x4_trans(addr, b0, b1, b2, b3);
-                                mma_bf16_16816(o[nt], pa, b0, b1);
-                                mma_bf16_16816(o[nt + 1], pa, b2, b3);
-                            }
-                        }
-                        if (kw + 16 > seg.n_kv) fence_proxy_async_smem();   // generic writes before TMA reuse
                     }
+                    // ---- scale, mask, online softmax ----
+                    // sliding window: the row at position i = n_kv - T + t keeps i - C < j, i.e.
+                    // j >= i - C + 1 = n_full + t - C; the highest such bound of any row is n_kv - C
+                    const bool need_mask = kw + 16 > n_full || (p.window > 0 && kw < seg.n_kv - p.window);
+                    // window start of the two rows this lane holds (no window: below every key)
+                    int lo0 = -1, lo1 = -1;
+                    if (need_mask && p.window > 0) {
+                        lo0 = n_full + (g % p.T) - p.window;
+                        lo1 = n_full + ((g + 8) % p.T) - p.window;
+                    }
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            float v = s[nt][e] * p.scale_log2;
+                            if (need_mask) {
+                                const int j = kw + nt * 8 + tq * 2 + (e & 1);
+                                v = (j < ((e & 2) ? vis1 : vis0) && j >= ((e & 2) ? lo1 : lo0)) ? v : -INFINITY;
+                            }
+                            s[nt][e] = v;
+                        }
+                    float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+                    const float mn0 = fmaxf(m0, mx0);
+                    const float ms0 = mn0 == -INFINITY ? 0.f : mn0;
+                    const float alpha0 = exp2f(m0 - ms0);
+                    m0 = mn0;
+                    float alpha1 = 1.f, ms1 = 0.f;
+                    if (ROWS == 16) {
+                        float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+                        const float mn1 = fmaxf(m1, mx1);
+                        ms1 = mn1 == -INFINITY ? 0.f : mn1;
+                        alpha1 = exp2f(m1 - ms1);
+                        m1 = mn1;
+                    }
+                    uint32_t pa[4];
+                    {
+                        const float p00 = exp2f(s[0][0] - ms0), p01 = exp2f(s[0][1] - ms0);
+                        const float p10 = exp2f(s[1][0] - ms0), p11 = exp2f(s[1][1] - ms0);
+                        l0 = l0 * alpha0 + ((p00 + p01) + (p10 + p11));
+                        pa[0] = pack_bf16x2(p00, p01);
+                        pa[2] = pack_bf16x2(p10, p11);
+                        if (ROWS == 16) {
+                            const float q00 = exp2f(s[0][2] - ms1), q01 = exp2f(s[0][3] - ms1);
+                            const float q10 = exp2f(s[1][2] - ms1), q11 = exp2f(s[1][3] - ms1);
+                            l1 = l1 * alpha1 + ((q00 + q01) + (q10 + q11));
+                            pa[1] = pack_bf16x2(q00, q01);
+                            pa[3] = pack_bf16x2(q10, q11);
+                        } else {
+                            pa[1] = pa[3] = 0u;
+                        }
+                    }
+                    if (__any_sync(0xffffffffu, alpha0 != 1.f || alpha1 != 1.f)) {
+#pragma unroll
+                        for (int nt = 0; nt < NT_O; ++nt) {
+                            o[nt][0] *= alpha0; o[nt][1] *= alpha0;
+                            o[nt][2] *= alpha1; o[nt][3] *= alpha1;
+                        }
+                    }
+                    // ---- rows past the end of the sequence may hold anything: zero them so that
+                    //      0 * garbage cannot produce NaN in O += P V ----
+                    if (kw + 16 > seg.n_kv) {
+                        const int first_bad = max(seg.n_kv - kw, 0);          // 0..15
+                        uint8_t* vrow = stage_mem + stage * C::STAGE_BYTES + C::TENSOR_BYTES;
+                        for (int r = first_bad; r < 16; ++r) {
+                            const int key_l = warp * 16 + r;
+                            for (int b = lane * 16; b < C::HALVES * 128; b += 512) {
+                                const int h = b >> 7, off = b & 127;
+                                *reinterpret_cast<uint4*>(vrow + h * HALF_BYTES + key_l * 128 + off) =
+                                    make_uint4(0u, 0u, 0u, 0u);
+                            }
+                        }
+                        __syncwarp();
+                    }
+                    // ---- O += P V ----
+                    {
+                        const int key_l = warp * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+                        const int sel = lane >> 4;
+                        const uint32_t rowaddr = vbase + key_l * 128;
+#pragma unroll
+                        for (int nt = 0; nt < NT_O; nt += 2) {
+                            const int c = nt + sel;
+                            const uint32_t addr =
+                                rowaddr + (c >> 3) * HALF_BYTES + ((((c & 7) ^ key_l) & 7) << 4);
+                            uint32_t b0, b1, b2, b3;
+                            ldmatrix_x4_trans(addr, b0, b1, b2, b3);
+                            mma_bf16_16816(o[nt], pa, b0, b1);
+                            mma_bf16_16816(o[nt + 1], pa, b2, b3);
+                        }
+                    }
+                    if (kw + 16 > seg.n_kv) fence_proxy_async_smem();   // generic writes before TMA reuse
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty_bar[stage]);
@@ -370,25 +357,25 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
             // ---- merge the four warps' states, write the final rows or this segment's partial ----
             l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
             l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-            if (MROWS == 16) {
+            if (ROWS == 16) {
                 l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
                 l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
             }
             {
-                float* mo = merge_o + (warp * MROWS) * D;
+                float* mo = merge_o + (warp * ROWS) * D;
 #pragma unroll
                 for (int nt = 0; nt < NT_O; ++nt) {
                     *reinterpret_cast<float2*>(mo + g * D + nt * 8 + tq * 2) = make_float2(o[nt][0], o[nt][1]);
-                    if (MROWS == 16)
+                    if (ROWS == 16)
                         *reinterpret_cast<float2*>(mo + (g + 8) * D + nt * 8 + tq * 2) =
                             make_float2(o[nt][2], o[nt][3]);
                 }
                 if (tq == 0) {
-                    merge_ml[(warp * MROWS + g) * 2] = m0;
-                    merge_ml[(warp * MROWS + g) * 2 + 1] = l0;
-                    if (MROWS == 16) {
-                        merge_ml[(warp * MROWS + g + 8) * 2] = m1;
-                        merge_ml[(warp * MROWS + g + 8) * 2 + 1] = l1;
+                    merge_ml[(warp * ROWS + g) * 2] = m0;
+                    merge_ml[(warp * ROWS + g) * 2 + 1] = l0;
+                    if (ROWS == 16) {
+                        merge_ml[(warp * ROWS + g + 8) * 2] = m1;
+                        merge_ml[(warp * ROWS + g + 8) * 2 + 1] = l1;
                     }
                 }
             }
@@ -396,20 +383,16 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
             const bool final_out = seg.stream_nseg == 1 && !p.force_partial && R == 1;
             for (int idx = threadIdx.x; idx < n_rows * D; idx += kConsumerWarps * 32) {
                 const int r = idx / D, col = idx - r * D;
-                // the warps that hold this row: all four, or the two of its row tile
-                const int w0 = WIDE ? (r >> 4) * 2 : 0;
-                const int rl = WIDE ? (r & 15) : r;
-                constexpr int NW = WIDE ? 2 : kConsumerWarps;
                 float M = -INFINITY;
 #pragma unroll
-                for (int w = 0; w < NW; ++w) M = fmaxf(M, merge_ml[((w0 + w) * MROWS + rl) * 2]);
+                for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, merge_ml[(w * ROWS + r) * 2]);
                 float L = 0.f, acc = 0.f;
                 if (M != -INFINITY) {
 #pragma unroll
-                    for (int w = 0; w < NW; ++w) {
-                        const float f = exp2f(merge_ml[((w0 + w) * MROWS + rl) * 2] - M);
-                        L += merge_ml[((w0 + w) * MROWS + rl) * 2 + 1] * f;
-                        acc += merge_o[((w0 + w) * MROWS + rl) * D + col] * f;
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        const float f = exp2f(merge_ml[(w * ROWS + r) * 2] - M);
+                        L += merge_ml[(w * ROWS + r) * 2 + 1] * f;
+                        acc += merge_o[(w * ROWS + r) * D + col] * f;
                     }
                 }
                 const float outv = L > 0.f ? acc / L : 0.f;
@@ -472,24 +455,19 @@ cudaError_t decode_kernel_setup() {
     cudaError_t e;
     if ((e = setup_one<128, 8>()) != cudaSuccess) return e;
     if ((e = setup_one<128, 16>()) != cudaSuccess) return e;
-    if ((e = setup_one<128, 32>()) != cudaSuccess) return e;
     if ((e = setup_one<64, 8>()) != cudaSuccess) return e;
-    if ((e = setup_one<64, 16>()) != cudaSuccess) return e;
-    return setup_one<64, 32>();
+    return setup_one<64, 16>();
 }
 
 cudaError_t launch_decode(const DecodeParams& p, const CUtensorMap& tmK, const CUtensorMap& tmV,
                           int num_groups, cudaStream_t stream, const DecodeInlineTables* tab) {
     if (num_groups <= 0) return cudaSuccess;
-    const int rows = p.rows_per_stream > 16 ? 32 : p.rows_per_stream > 8 ? 16 : 8;
-    if (p.d == 128) {
-        if (rows == 32) return launch_one<128, 32>(p, tmK, tmV, num_groups, stream, tab);
-        return rows == 16 ? launch_one<128, 16>(p, tmK, tmV, num_groups, stream, tab)
-                          : launch_one<128, 8>(p, tmK, tmV, num_groups, stream, tab);
-    }
-    if (rows == 32) return launch_one<64, 32>(p, tmK, tmV, num_groups, stream, tab);
-    return rows == 16 ? launch_one<64, 16>(p, tmK, tmV, num_groups, stream, tab)
-                      : launch_one<64, 8>(p, tmK, tmV, num_groups, stream, tab);
+    const bool wide = p.rows_per_stream > 8;
+    if (p.d == 128)
+        return wide ? launch_one<128, 16>(p, tmK, tmV, num_groups, stream, tab)
+                    : launch_one<128, 8>(p, tmK, tmV, num_groups, stream, tab);
+    return wide ? launch_one<64, 16>(p, tmK, tmV, num_groups, stream, tab)
+                : launch_one<64, 8>(p, tmK, tmV, num_groups, stream, tab);
 }
 
 }  // namespace yoco

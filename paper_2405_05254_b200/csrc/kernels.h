@@ -68,7 +68,7 @@ struct DecodeParams {
     int32_t* status;
     float scale_log2;           // scale * log2(e)
     int32_t T;
-    int32_t rows_per_stream;    // G * T (<= 32)
+    int32_t rows_per_stream;    // G * T (<= 16)
     int32_t d;
     int32_t window;             // sliding window C, 0 = none
     int32_t force_partial;      // write every segment to its partial slot, even of an unsplit stream

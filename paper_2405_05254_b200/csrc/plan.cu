@@ -14,7 +14,7 @@ int32_t validate_shape(const yoco_xattn_shape& s, int32_t mode) {
     if (s.Hq % s.Hkv != 0) return YOCO_ERR_UNSUPPORTED;
     if (s.kv_head_stride % s.d != 0) return YOCO_ERR_UNSUPPORTED;
     const int64_t rows = (int64_t)(s.Hq / s.Hkv) * s.T;
-    if (mode == YOCO_MODE_DECODE && rows > kDecodeMaxRows) return YOCO_ERR_UNSUPPORTED;
+    if (mode == YOCO_MODE_DECODE && rows > kDecodeTileM) return YOCO_ERR_UNSUPPORTED;
     if ((int64_t)s.B * s.Hq * s.T >= (1ll << 31)) return YOCO_ERR_UNSUPPORTED;
     return YOCO_OK;
 }
@@ -28,7 +28,7 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     const int G = s.Hq / s.Hkv;
     const int rows_per_stream = G * s.T;
     const int tile_n = mode == YOCO_MODE_DECODE ? kDecodeTileN : kChunkTileN;
-    const int tile_m = mode == YOCO_MODE_DECODE ? (rows_per_stream > kDecodeTileM ? kDecodeMaxRows : kDecodeTileM)
+    const int tile_m = mode == YOCO_MODE_DECODE ? kDecodeTileM
                        : rows_per_stream > kChunkTileM ? kChunkPairTileM : kChunkTileM;
     const int m_tiles = (rows_per_stream + tile_m - 1) / tile_m;
     const int num_streams = s.B * s.Hkv;

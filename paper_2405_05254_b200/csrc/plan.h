@@ -16,7 +16,6 @@ namespace yoco {
 
 constexpr int kDecodeTileN = 64;      // keys per shared-memory stage of the decode kernel
 constexpr int kDecodeTileM = 16;      // query rows of one mma.sync tile
-constexpr int kDecodeMaxRows = 32;    // most rows per KV head the decode kernel takes (two tiles)
 constexpr int kDecodeGroupsPerSm = 2; // resident decode CTAs per SM
 constexpr int kChunkTileN = 128;      // keys per tcgen05 tile
 constexpr int kChunkTileM = 128;      // query rows per tcgen05 tile

@@ -15,7 +15,7 @@ def random_case(rng, mode):
     Hkv = int(rng.choice([1, 2, 3, 8]))
     if mode == "decode":
         G = int(rng.choice([1, 2, 3, 4, 8, 16]))
-        T = int(rng.integers(1, 32 // G + 1))
+        T = int(rng.integers(1, 16 // G + 1))
     else:
         G = int(rng.choice([1, 3, 4, 8]))
         T = int(rng.choice([1, 7, 32, 33, 100, 129, 260]))
@@ -30,7 +30,7 @@ def random_case(rng, mode):
 
 
 @pytest.mark.parametrize("mode", ["decode", "chunk"])
-@pytest.mark.parametrize("seed", range(16))
+@pytest.mark.parametrize("seed", range(12))
 def test_random_shapes(mode, seed):
     rng = np.random.default_rng(1000 * (mode == "chunk") + seed)
     c = random_case(rng, mode)
@@ -62,7 +62,7 @@ def random_long_case(rng):
     d = int(rng.choice([64, 128]))
     Hkv = int(rng.choice([1, 2, 4, 8]))
     G = int(rng.choice([1, 2, 4, 8, 16]))
-    T = int(rng.integers(1, 32 // G + 1))
+    T = int(rng.integers(1, 16 // G + 1))
     B = int(rng.integers(1, 4))
     total = int(rng.integers(800_000, 2_400_000)) // Hkv          # keys per head, all sequences together
     cuts = np.sort(rng.integers(1, total, size=B - 1)) if B > 1 else np.array([], dtype=np.int64)

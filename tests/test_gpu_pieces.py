@@ -136,22 +136,3 @@ def test_two_streams_running_pieces_at_once_keep_their_bits():
         for x, ref in zip(probs, solo):
             assert bd.yoco_xattn_status(x["ws"]) == 0
             assert torch.equal(x["O"].view(torch.int16), ref)
-
-
-def test_wide_rows_in_pieces_with_window_and_rescales():
-    """24 rows per KV head (G = 4, T = 6: the two-row-tile variant of the decode kernel) over long caches in
-    pieces, with a window; and peaked scores, so that the running maximum moves late in the stream."""
-    w = si.Workload("wide", B=2, Hq=8, Hkv=2, d=128, T=6, layers=1, seed=35, kv_len=[420001, 77])
-    C = 400000
-    info, _ = plan_of(w, window=C)
-    assert info.sub_items >= 2 and info.tile_m == 32
-    K, V, Q = w.make_k(), w.make_v(), w.make_q(0)
-    Kf = si.bf16_bits_to_f32(K).copy()
-    Kf[-3 * w.d:] *= 6.0                      # the last keys of the last head of sequence 1 stand out
-    Kf[(2 * 420001 - 5) * w.d:(2 * 420001) * w.d] *= 5.0      # and the last keys of sequence 0, head 1
-    K = si.f32_to_bf16_bits(Kf)
-    r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, w.T, w.kv_len, K, V, window=C)
-    o, lse, _ = r.run(Q)
-    o_ref, lse_ref = oracle.xattn(Q, K, V, w.cu, w.kv_len, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T, window=C)
-    assert_close(o, o_ref, "wide rows in pieces")
-    assert_lse_close(lse, lse_ref, "wide rows in pieces")

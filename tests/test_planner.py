@@ -41,7 +41,7 @@ def test_strerror_covers_the_codes():
 def restated_plan(B, Hkv, lens, sm_count, mode, G, T):
     """Test-side restatement of the rule: flat (stream, tile) space cut into equal ranges."""
     tile_n = 64 if mode == bd.MODE_DECODE else 128
-    tile_m = (32 if G * T > 16 else 16) if mode == bd.MODE_DECODE else (256 if G * T > 128 else 128)
+    tile_m = 16 if mode == bd.MODE_DECODE else (256 if G * T > 128 else 128)
     m_tiles = -(-G * T // tile_m)
     nts = [-(-int(n) // tile_n) for n in lens]
     total = Hkv * sum(nts)
@@ -116,7 +116,7 @@ CASES = [
 @pytest.mark.parametrize("sm_count", [148, 7])
 def test_plan_partitions_every_stream_exactly(case, sm_count):
     G = case["Hq"] // case["Hkv"]
-    modes = [bd.MODE_CHUNK] + ([bd.MODE_DECODE] if G * case["T"] <= 32 else [])
+    modes = [bd.MODE_CHUNK] + ([bd.MODE_DECODE] if G * case["T"] <= 16 else [])
     for mode in modes:
         shape = bd.make_shape(case["B"], case["Hq"], case["Hkv"], case["d"], case["T"])
         info, segs = bd.yoco_xattn_plan(shape, case["lens"], sm_count, mode)
@@ -182,7 +182,7 @@ def test_unsplit_streams_need_no_combine():
 @pytest.mark.parametrize("kw,code", [
     (dict(d=96), bd.ERR_UNSUPPORTED),
     (dict(Hq=30), bd.ERR_UNSUPPORTED),
-    (dict(T=9), bd.ERR_UNSUPPORTED),           # G*T = 36 rows > 32 in decode mode
+    (dict(T=5), bd.ERR_UNSUPPORTED),           # G*T = 20 rows > 16 in decode mode
     (dict(T=0), bd.ERR_INVALID_ARG),
     (dict(B=-1), bd.ERR_INVALID_ARG),
     (dict(kv_head_stride=100), bd.ERR_UNSUPPORTED),
@@ -232,7 +232,7 @@ def test_sliding_window_plan_skips_only_tiles_no_row_can_see(case):
     """With a window C the lowest key any row sees is that of row 0, (N - T) - C + 1; the plan
     starts at the tile that holds it and still partitions the rest exactly."""
     G, T, C = case["Hq"] // case["Hkv"], case["T"], case["C"]
-    modes = [bd.MODE_CHUNK] + ([bd.MODE_DECODE] if G * T <= 32 else [])
+    modes = [bd.MODE_CHUNK] + ([bd.MODE_DECODE] if G * T <= 16 else [])
     for mode in modes:
         shape = bd.make_shape(case["B"], case["Hq"], case["Hkv"], case["d"], T, window=C)
         info, segs = bd.yoco_xattn_plan(shape, case["lens"], 148, mode)
