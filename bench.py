@@ -45,14 +45,18 @@ def measured_peaks():
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of decode_kernel_inline<128, 8> per launch from the ncu capture
-# (mean of two launches, 128K-token case; the summary sits with the other profiler summaries).
+# (mean of two launches, 128K-token case), with the summary file that holds the capture.  Set to None when the
+# kernel has changed since the counters were taken.
 NCU_DECODE_DRAM_BYTES = 542587136
 NCU_DECODE_KV_BYTES = 536870912
+NCU_DECODE_PROFILE = "profiles/decode_kernel_128k_ncu_full.md"
 
 
 def ncu_traffic_per_launch(kv_bytes: int):
-    """Traffic of a full-size launch: every K/V byte is read exactly once, so DRAM bytes grow in
-    proportion to the keys streamed."""
+    """Traffic of a full-size launch, scaled from the profiler capture of a shorter case: every K/V byte is
+    read exactly once, so DRAM bytes grow in proportion to the keys streamed.  None without a capture."""
+    if NCU_DECODE_DRAM_BYTES is None:
+        return None
     return NCU_DECODE_DRAM_BYTES * (kv_bytes / NCU_DECODE_KV_BYTES)
 
 
@@ -457,7 +461,7 @@ def measure_fp8_cache(dev, w, Q, peak_gbs):
 
 def measure_other_configs(dev, peak_gbs):
     """Layer-call time of the decode path on the other decode configurations (tiny, 32K with a cold and a
-    warm L2, the ragged batch of 16), for the record; not part of the default run."""
+    warm L2, the ragged batch of 16): a few seconds, part of the default run."""
     import torch
     from paper_2405_05254_b200 import binding as bd
     out = {}
@@ -481,19 +485,31 @@ def measure_other_configs(dev, peak_gbs):
         e1.record()
         torch.cuda.synchronize()
         warm_us = e0.elapsed_time(e1) * 1e3 / n
-        cold = 0.0
-        for k in range(10):
+        def flush_l2(k):
             flush.fill_(k)
             flush.view(torch.float32).sum()      # read pass: leaves L2 clean (no write-back during the call)
+
+        cold = 0.0
+        for k in range(10):
+            flush_l2(k)
             e0.record()
             bd.yoco_xattn_decode(shape, Qs[k % w.layers], K, V, w.cu, w.kv_len, O, None, ws)
             e1.record()
             torch.cuda.synchronize()
             cold += e0.elapsed_time(e1) * 1e3 / 10
+        bd.yoco_xattn_profile_enable(10)
+        for k in range(10):
+            flush_l2(k)
+            bd.yoco_xattn_decode(shape, Qs[k % w.layers], K, V, w.cu, w.kv_len, O, None, ws)
+        kern_cold = float(bd.yoco_xattn_profile_collect(10).mean()) * 1e3
+        bd.yoco_xattn_profile_enable(0)
         out[name] = {"workload": f"B={w.B} Hq={w.Hq} Hkv={w.Hkv} d={w.d} T={w.T} tokens={w.total_tokens}",
                      "kv_bytes_per_call": w.kv_bytes, "back_to_back_call_us": warm_us, "cold_l2_call_us": cold,
+                     "cold_l2_kernel_us": kern_cold,
                      "back_to_back_gbs": w.kv_bytes / warm_us / 1e3, "cold_l2_gbs": w.kv_bytes / cold / 1e3,
-                     "us_per_token_layer": warm_us / w.B, "frac_of_measured_hbm_cold": w.kv_bytes / cold / 1e3 / peak_gbs}
+                     "cold_l2_kernel_gbs": w.kv_bytes / kern_cold / 1e3,
+                     "us_per_token_layer": warm_us / w.B, "frac_of_measured_hbm_cold": w.kv_bytes / cold / 1e3 / peak_gbs,
+                     "frac_of_measured_hbm_cold_kernel": w.kv_bytes / kern_cold / 1e3 / peak_gbs}
         del K, V
     return out
 
@@ -653,8 +669,12 @@ def run_ours(args):
                          "kernel_us": k_avg_ms * 1e3, "algorithmic_bytes_per_launch": w.kv_bytes,
                          "timed_over": f"a second pass of the same {args.steps} steps with an event pair around "
                                        "every attention kernel",
-                         "traffic": traffic},
+                         "traffic": traffic,
+                         "traffic_source": f"ncu capture of the 128K-token case scaled by keys streamed ({NCU_DECODE_PROFILE}); "
+                                           "not measured in this run"},
         }
+        if world == 1 and not args.no_other_configs:
+            line["other_configs"] = measure_other_configs(dev, peak)
         if world == 1 and w.d == 128 and not args.no_fp8:
             line["fp8_cache"] = measure_fp8_cache(dev, w, Qd[0], peak)
         if world == 1 and w.B == 1 and w.T == 1 and not args.no_shard:
@@ -669,8 +689,6 @@ def run_ours(args):
             line["kv_append"] = measure_kv_append(dev, peaks, peak)
         if world == 1 and not args.no_window:
             line["sliding_window"] = measure_window(dev, peak)
-        if world == 1 and args.all_configs:
-            line["other_configs"] = measure_other_configs(dev, peak)
         if world == 1 and not args.no_cpu_baseline:
             gbs, dt, sample, cores = oracle_sample_rate(w, Qh, Kh, Vh)
             line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
@@ -690,8 +708,8 @@ def main():
     ap.add_argument("--workload", default="1m", choices=["1m", "128k", "3b_32k", "ragged", "tiny"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-chunk", action="store_true", help="skip the extra measurement of the chunk path")
-    ap.add_argument("--all-configs", action="store_true",
-                    help="also time a layer call on the tiny, 32K and ragged configurations")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the layer-call times of the tiny, 32K and ragged configurations")
     ap.add_argument("--no-fp8", action="store_true", help="skip the decode over an 8-bit cache")
     ap.add_argument("--no-append", action="store_true", help="skip the cache-writing (K/V projection) measurement")
     ap.add_argument("--no-shard", action="store_true", help="skip the key-range-shard measurement")

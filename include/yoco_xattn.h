@@ -21,6 +21,8 @@
  *          head_stride_i = kv_head_stride if non-zero (a cache with spare
  *          capacity per head; must be a multiple of d), else N_i*d (tight).
  *          With equal lengths and tight packing this is [B, Hkv, N, d].
+ *          A sequence occupies Hkv * head_stride_i elements from its offset, so
+ *          cu_kv[i+1] - cu_kv[i] >= head_stride_i / d is required (else INVALID_ARG).
  *          Both buffers must start on a 16-byte boundary.
  *   kv_len[i] = N_i  counts ALL keys of sequence i including the T positions of
  *          the current call (the self-decoder has already appended them).
@@ -40,7 +42,17 @@
  * Errors: every function returns YOCO_OK or a negative code.  Argument and
  * shape checks happen before anything is enqueued.  A device-side bounded wait
  * that ran out (never expected) is recorded in a status word inside the
- * workspace and read back by yoco_xattn_status().
+ * workspace and read back by yoco_xattn_status(); the kernel that gave up first
+ * waits for the copies and products it had started, then returns normally, so the
+ * context stays usable.
+ *
+ * CUDA graphs: a call may be recorded into a graph.  The work tables of a problem
+ * with at most 448 work segments, 303 CTA groups and 256 (sequence, KV head) streams
+ * travel as kernel parameters and the recorded nodes refer to nothing but the
+ * caller's buffers.  A larger problem uploads its tables from host memory owned by
+ * the library's plan cache; the library then keeps that plan for the life of the
+ * process, so a replay never reads released memory.  In both cases the caller's
+ * buffers, kv_len and cu_kv as they were at recording time are what a replay uses.
  */
 #ifndef YOCO_XATTN_H_
 #define YOCO_XATTN_H_
@@ -107,7 +119,9 @@ typedef struct yoco_xattn_plan_info {
     int32_t num_slots;       /* partial-result slots the workspace holds                  */
 } yoco_xattn_plan_info;
 
-/* Split-count / tile heuristic (host only, integers only, deterministic).
+/* Split-count / tile heuristic (host only, integers only, deterministic).  No counterpart in the
+ * paper, which names no kernel for cross-attention (Section 4.4 attributes split-KV decoding only
+ * to its Transformer baseline); exported so that tests can check the plan integer for integer.
  * The flat space of (stream, key tile) pairs, streams ordered (b, c), is cut into
  * num_groups contiguous ranges of equal tile count (+-1); a range that crosses a
  * stream boundary becomes several segments.  num_groups = min(total_tiles,
@@ -127,20 +141,21 @@ int32_t yoco_xattn_plan(const yoco_xattn_shape* shape, const int32_t* kv_len_hos
                         int32_t sm_count, int32_t mode, yoco_xattn_plan_info* info,
                         yoco_xattn_segment* segments_out, int32_t capacity);
 
-/* First tile, counted inside a group of n_tiles key tiles, of piece r of sub_items
+/* (No counterpart in the paper.)  First tile, counted inside a group of n_tiles key tiles, of piece r of sub_items
  * (r = 0 .. sub_items; sub_items in {1, 2, 4}): piece r covers tiles [bound(r), bound(r+1))
  * with bound(r) = n_tiles * c(r) / 64 rounded down, c = 0, 52, 64 for two pieces and
  * 0, 44, 54, 61, 64 for four.  Returns -1 for other arguments.  Pure host. */
 int64_t yoco_xattn_sub_bound(int64_t n_tiles, int32_t sub_items, int32_t r);
 
-/* Workspace bytes for decode/chunk on this problem.  sm_count = 0 queries the
+/* (No counterpart in the paper.)  Workspace bytes for decode/chunk on this problem.  sm_count = 0 queries the
  * current CUDA device (then YOCO_ERR_CUDA is possible).  Pure host otherwise. */
 int32_t yoco_xattn_workspace_size(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
                                   int32_t sm_count, int32_t mode, size_t* bytes);
 
-/* Split-KV decode (flash-decoding style): a few query rows per KV head (G*T <= 16;
- * typically T = 1, the next-token call of a cross-decoder layer) against the
- * whole cache.  Runs the split kernel, then the merge when a stream was split.
+/* Attention(Q^l, K^, V^) of Section 2.2 (cross-decoder equations) for the next-token call of a
+ * cross-decoder layer, the call whose cost Section 2.3 reduces to one pass over the single shared
+ * cache: split-KV decode (flash-decoding style) of a few query rows per KV head (G*T <= 16;
+ * typically T = 1) against the whole cache.  Runs the split kernel, then the merge when a stream was split.
  *   Q, K, V, O, lse (may be NULL), workspace: device.  cu_kv_host: host [B+1] token
  *   offsets, or NULL = prefix sums of kv_len (tight packing).  kv_len_host: host [B]
  *   or NULL.  workspace: >= yoco_xattn_workspace_size(), 256-byte aligned; it holds the
@@ -164,9 +179,12 @@ int32_t yoco_xattn_decode(const yoco_xattn_shape* shape, const void* Q, const vo
  * loads the library carries those 4 MiB until the process ends.
  *
  * Limits and rules:
- *  - A problem whose decode workspace (yoco_xattn_workspace_size, decode mode) exceeds
- *    yoco_xattn_static_scratch_bytes() is refused with YOCO_ERR_STATIC_SCRATCH_EXCEEDED and
+ *  - A problem whose one-piece decode plan (every CTA group a single work piece, which is how this
+ *    entry always runs; at most what yoco_xattn_workspace_size reports for decode mode) needs more
+ *    than yoco_xattn_static_scratch_bytes() is refused with YOCO_ERR_STATIC_SCRATCH_EXCEEDED and
  *    nothing is enqueued.  4 MiB covers, e.g., B = 1 at 1M tokens and 16 ragged sequences.
+ *  - The status word of these calls lives in the built-in buffer: yoco_xattn_status(NULL, stream)
+ *    reads it (for the current device).
  *  - No cudaMalloc / cudaFree and no allocating library routine is called.
  *  - The first call on each device looks the buffer's device address up (and sets kernel
  *    attributes); make that first call with the device current and before any stream capture.
@@ -180,10 +198,12 @@ int32_t yoco_xattn_decode_static(const yoco_xattn_shape* shape, const void* Q, c
                                  const void* V, const int32_t* cu_kv_host,
                                  const int32_t* kv_len_host, void* O, float* lse, void* stream);
 
-/* Size in bytes of the built-in buffer used by yoco_xattn_decode_static. */
+/* (No counterpart in the paper.)  Size in bytes of the built-in buffer used by yoco_xattn_decode_static. */
 int32_t yoco_xattn_static_scratch_bytes(void);
 
-/* Multi-token chunk / full-sequence path: T new query rows per sequence, causal
+/* Attention(Q^l, K^, V^) of Section 2.2 for many positions at once ("causal masking is also used
+ * for cross-attention"): a prefill or scoring chunk, whose cost is the O(N) per position of
+ * Section 2.3's prefill table.  T new query rows per sequence, causal
  * inside the chunk, as a dense contraction on the tcgen05 tensor cores (S = Q K^T
  * and O = P V with accumulators in tensor memory).  Same arguments as decode; any
  * T >= 1.  */
@@ -192,7 +212,8 @@ int32_t yoco_xattn_chunk(const yoco_xattn_shape* shape, const void* Q, const voi
                          void* O, float* lse, void* workspace, size_t workspace_bytes,
                          void* stream);
 
-/* Stand-alone log-sum-exp merge of S partial attention results per row:
+/* (No counterpart in the paper: the exact recombination of softmax attention evaluated over
+ * disjoint key ranges.)  Stand-alone log-sum-exp merge of S partial attention results per row:
  *   lse = log sum_s exp(lse_s),   O = sum_s exp(lse_s - lse) * O_s
  * part_o [rows, S, d] fp32 (each O_s already normalised), part_lse [rows, S] fp32
  * natural log, -inf marks an empty piece (weight 0; all empty -> O = 0, lse = -inf).
@@ -214,7 +235,7 @@ int32_t yoco_xattn_decode_fp8(const yoco_xattn_shape* shape, const void* Q, cons
                               const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
                               void* workspace, size_t workspace_bytes, void* stream);
 
-/* The same merge for pieces laid out piece-major: part_o [S, rows, d], part_lse [S, rows] -- what
+/* (No counterpart in the paper.)  The same merge for pieces laid out piece-major: part_o [S, rows, d], part_lse [S, rows] -- what
  * an all-gather over S ranks leaves when every rank contributes its [rows, d] partial result and
  * its [rows] log-sum-exp.  Otherwise as yoco_xattn_combine. */
 int32_t yoco_xattn_combine_gathered(int64_t rows, int32_t S, int32_t d, const float* part_o,
@@ -252,13 +273,14 @@ typedef struct yoco_kv_append_shape {
     int64_t kv_head_stride;  /* as in yoco_xattn_shape                                    */
 } yoco_kv_append_shape;
 
-/* Folds the RMSNorm gain into a projection weight once per model (weights do not change between
+/* (Section 2.1's RMSNorm as used by Section 2.2's first equation; the folding itself has no
+ * counterpart in the paper.)  Folds the RMSNorm gain into a projection weight once per model (weights do not change between
  * calls):  Wg[k, n] = g[k] * W[k, n], one rounding to bf16.  g [d_model], W and Wg [d_model, n_out]
  * row-major bf16, all device; Wg may not alias W. */
 int32_t yoco_kv_fold_gain(int64_t d_model, int64_t n_out, const void* g, const void* W, void* Wg,
                           void* stream);
 
-/* Computes the new cache rows and stores them.  X [B*T, d_model] bf16 (sequence-major, the T
+/* Section 2.2, first cross-decoder equation.  Computes the new cache rows and stores them.  X [B*T, d_model] bf16 (sequence-major, the T
  * tokens of a sequence consecutive); Wgk, Wgv [d_model, Hkv*d] bf16 = gain-folded W_K, W_V (see
  * yoco_kv_fold_gain); K, V: the packed caches (device, written in place, 16-byte aligned);
  * cu_kv_host [B+1] or NULL (tight packing), kv_len_host [B]: host, N_i >= T including the new
@@ -277,13 +299,42 @@ int32_t yoco_kv_append_fp8(const yoco_kv_append_shape* shape, const void* X, con
                            void* K8, void* V8, const float* k_scale_host, const float* v_scale_host,
                            const int32_t* cu_kv_host, const int32_t* kv_len_host, void* stream);
 
-/* Synchronises `stream`; returns YOCO_OK or YOCO_ERR_TIMEOUT if an append kernel on the current
- * device gave up a wait since the last call of this function (which clears the record). */
+/* (No counterpart in the paper.)  Synchronises `stream`; returns YOCO_OK or YOCO_ERR_TIMEOUT if an
+ * append kernel on the current device gave up a wait since the last call of this function (which
+ * clears the record).  The _detail form also reports which wait and which CTA (see below). */
 int32_t yoco_kv_append_status(void* stream);
+int32_t yoco_kv_append_status_detail(void* stream, int32_t* wait_class, int32_t* cta);
 
-/* Synchronises `stream`, reads the status word that the last decode/chunk call
- * using `workspace` left, returns it (YOCO_OK or YOCO_ERR_TIMEOUT). */
+/* (No counterpart in the paper.)  Synchronises `stream`, reads the status word that the last
+ * decode/chunk call using `workspace` left, returns YOCO_OK or YOCO_ERR_TIMEOUT.  workspace = NULL
+ * reads the word of the built-in buffer of yoco_xattn_decode_static on the current device. */
 int32_t yoco_xattn_status(const void* workspace, void* stream);
+
+/* What gave up.  The status word is 0, or  wait_class | (cta + 1) << 8  of the first wait that ran
+ * out: the kind of wait (YOCO_WAIT_*) and the linear index of the CTA.  yoco_xattn_status_detail
+ * reads the word like yoco_xattn_status and decodes it (either output may be NULL; wait_class 0
+ * and cta -1 when nothing happened); yoco_xattn_decode_status_word decodes a word the caller holds
+ * (pure host).  Both return YOCO_OK or YOCO_ERR_TIMEOUT. */
+#define YOCO_WAIT_ITEM_QUEUE 1  /* decode: hand-over of the next work item inside a CTA            */
+#define YOCO_WAIT_RING_FULL  2  /* a consumer waiting for a tile copy to land                      */
+#define YOCO_WAIT_RING_EMPTY 3  /* the producer waiting for a stage to be released                 */
+#define YOCO_WAIT_TENSOR     4  /* tensor-core hand-over: scores ready, P written, product done    */
+#define YOCO_WAIT_DRAIN      5  /* on the way out: something already started did not finish        */
+#define YOCO_WAIT_MISALIGNED 6  /* shared memory not 1 KB aligned; the kernel did nothing          */
+int32_t yoco_xattn_status_detail(const void* workspace, void* stream, int32_t* wait_class, int32_t* cta);
+int32_t yoco_xattn_decode_status_word(int32_t word, int32_t* wait_class, int32_t* cta);
+
+/* Self-test of the bounded waits (no counterpart in the paper).  Runs the decode kernel on the given
+ * problem (arguments as for yoco_xattn_decode, one work piece per CTA group) with a producer that
+ * starts no copy at all and a wait limit of limit_ms milliseconds (1..1000): the first wait for a
+ * tile runs out with nothing in flight, the CTAs record it and return, and O is left undefined.
+ * Afterwards yoco_xattn_status(workspace) must report YOCO_ERR_TIMEOUT with YOCO_WAIT_RING_FULL, and
+ * the next ordinary call on the same device and workspace must work.  Nothing faults, traps or
+ * waits without a limit. */
+int32_t yoco_xattn_selftest_wait_expiry(const yoco_xattn_shape* shape, const void* Q, const void* K,
+                                        const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
+                                        void* O, void* workspace, size_t workspace_bytes, int32_t limit_ms,
+                                        void* stream);
 
 /* Measurement aid (no counterpart in the paper).  After yoco_xattn_profile_enable(n), each of
  * the next n decode/chunk calls records a CUDA event pair on its stream around the attention
@@ -293,9 +344,10 @@ int32_t yoco_xattn_status(const void* workspace, void* stream);
 int32_t yoco_xattn_profile_enable(int32_t max_records);
 int32_t yoco_xattn_profile_collect(float* kernel_ms, int32_t capacity, int32_t* count);
 
+/* (No counterpart in the paper.)  Text of an error code. */
 const char* yoco_xattn_strerror(int32_t code);
 
-/* cudaError_t (as int) of the most recent failing CUDA call on this thread, 0 if none. */
+/* (No counterpart in the paper.)  cudaError_t (as int) of the most recent failing CUDA call on this thread, 0 if none. */
 int32_t yoco_xattn_last_cuda_error(void);
 
 #ifdef __cplusplus

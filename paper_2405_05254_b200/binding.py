@@ -86,6 +86,13 @@ def lib() -> ctypes.CDLL:
         for name in ("yoco_kv_fold_gain", "yoco_kv_append", "yoco_kv_append_status"):
             getattr(L, name).restype = i32
         L.yoco_xattn_status.argtypes = [vp, vp]
+        L.yoco_xattn_status_detail.argtypes = [vp, vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.yoco_xattn_decode_status_word.argtypes = [i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.yoco_kv_append_status_detail.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.yoco_xattn_selftest_wait_expiry.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, sz, i32, vp]
+        for name in ("yoco_xattn_status_detail", "yoco_xattn_decode_status_word", "yoco_kv_append_status_detail",
+                     "yoco_xattn_selftest_wait_expiry"):
+            getattr(L, name).restype = i32
         L.yoco_xattn_profile_enable.argtypes = [i32]
         L.yoco_xattn_profile_collect.argtypes = [vp, i32, vp]
         L.yoco_xattn_strerror.argtypes = [i32]
@@ -278,8 +285,44 @@ def yoco_kv_append_status(stream=None) -> int:
 
 
 def yoco_xattn_status(workspace, stream=None) -> int:
-    """Synchronise the stream and return the device status word of the last call (0 = ok)."""
+    """Synchronise the stream and return the status of the last call that used ``workspace`` (0 = ok);
+    ``workspace=None`` reads the built-in buffer of yoco_xattn_decode_static on the current device."""
     return int(lib().yoco_xattn_status(_ptr(workspace), _stream_ptr(stream)))
+
+
+WAIT_ITEM_QUEUE, WAIT_RING_FULL, WAIT_RING_EMPTY, WAIT_TENSOR, WAIT_DRAIN, WAIT_MISALIGNED = 1, 2, 3, 4, 5, 6
+
+
+def yoco_xattn_status_detail(workspace, stream=None):
+    """(status, wait_class, cta): which kind of bounded wait ran out first, and in which CTA."""
+    wc, cta = ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = lib().yoco_xattn_status_detail(_ptr(workspace), _stream_ptr(stream), ctypes.byref(wc), ctypes.byref(cta))
+    return int(rc), int(wc.value), int(cta.value)
+
+
+def yoco_xattn_decode_status_word(word: int):
+    """Pure host: (status, wait_class, cta) of a status word."""
+    wc, cta = ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = lib().yoco_xattn_decode_status_word(int(word), ctypes.byref(wc), ctypes.byref(cta))
+    return int(rc), int(wc.value), int(cta.value)
+
+
+def yoco_kv_append_status_detail(stream=None):
+    wc, cta = ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = lib().yoco_kv_append_status_detail(_stream_ptr(stream), ctypes.byref(wc), ctypes.byref(cta))
+    return int(rc), int(wc.value), int(cta.value)
+
+
+def yoco_xattn_selftest_wait_expiry(shape: Shape, Q, K, V, cu_kv, kv_len, O, workspace, limit_ms: int, stream=None) -> None:
+    """Run the decode kernel with a producer that starts no copy and a wait limit of ``limit_ms``: the
+    first tile wait runs out, the kernel records it and returns.  O is left undefined."""
+    keep_cu, p_cu = _host_i32(cu_kv)
+    keep_len, p_len = _host_i32(kv_len)
+    rc = lib().yoco_xattn_selftest_wait_expiry(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), p_cu, p_len, _ptr(O),
+                                               _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                               int(limit_ms), _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_selftest_wait_expiry")
 
 
 def yoco_xattn_profile_enable(max_records: int) -> None:

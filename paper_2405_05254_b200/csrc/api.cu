@@ -82,6 +82,9 @@ struct PlanEntry {
 };
 std::list<PlanEntry> g_plans;   // most recently used first
 constexpr size_t kPlanCacheEntries = 16;
+// Plans whose table upload was recorded into a CUDA graph: the recorded copy reads the plan's host
+// image at every replay, so these are never dropped.
+std::vector<std::shared_ptr<const ReadyPlan>> g_captured_plans;
 
 // Looks the plan up (most recently used first) or makes it.  The shared pointer keeps the entry
 // alive for the caller even if another thread evicts it from the cache meanwhile.
@@ -151,8 +154,42 @@ int32_t get_encoder(EncodeTiledFn* fn) {
     return YOCO_OK;
 }
 
+// A serving loop calls with the same cache pointers and extents step after step: the last few
+// encoded maps are kept per host thread, keyed by everything that goes into the encoding.
+struct MapKey {
+    const void* base;
+    int64_t rows;
+    int32_t d, box_rows, u8;
+    bool operator==(const MapKey& o) const {
+        return base == o.base && rows == o.rows && d == o.d && box_rows == o.box_rows && u8 == o.u8;
+    }
+};
+struct MapCache {
+    static constexpr int kEntries = 8;
+    MapKey key[kEntries];
+    CUtensorMap map[kEntries];
+    int used = 0, next = 0;
+    bool find(const MapKey& k, CUtensorMap* out) const {
+        for (int i = 0; i < used; ++i)
+            if (key[i] == k) {
+                *out = map[i];
+                return true;
+            }
+        return false;
+    }
+    void put(const MapKey& k, const CUtensorMap& m) {
+        key[next] = k;
+        map[next] = m;
+        next = (next + 1) % kEntries;
+        if (used < kEntries) ++used;
+    }
+};
+thread_local MapCache g_maps;
+
 // 2-D bf16 map over a row-major [rows, d] matrix, box {64 channels, box_rows}, 128-byte swizzle.
 int32_t make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int32_t d, int32_t box_rows) {
+    const MapKey mk{base, rows, d, box_rows, 0};
+    if (g_maps.find(mk, map)) return YOCO_OK;
     EncodeTiledFn enc;
     int32_t rc = get_encoder(&enc);
     if (rc != YOCO_OK) return rc;
@@ -164,11 +201,14 @@ int32_t make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int32_t d,
                      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+    g_maps.put(mk, *map);
     return YOCO_OK;
 }
 
 // 2-D byte map over a row-major [rows, 128] matrix of FP8 values, box {128, box_rows}, 128-byte swizzle.
 int32_t make_map_2d_u8(CUtensorMap* map, const void* base, int64_t rows, int32_t box_rows) {
+    const MapKey mk{base, rows, 128, box_rows, 1};
+    if (g_maps.find(mk, map)) return YOCO_OK;
     EncodeTiledFn enc;
     int32_t rc = get_encoder(&enc);
     if (rc != YOCO_OK) return rc;
@@ -180,6 +220,7 @@ int32_t make_map_2d_u8(CUtensorMap* map, const void* base, int64_t rows, int32_t
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+    g_maps.put(mk, *map);
     return YOCO_OK;
 }
 
@@ -210,10 +251,15 @@ cudaEvent_t prof_event(bool after, bool* active) {
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
+// self-test of the give-up path of the decode kernel (yoco_xattn_selftest_wait_expiry)
+struct SelfTest {
+    int64_t wait_limit_ns;
+};
+
 int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const void* K, const void* V,
             const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
             void* workspace, size_t workspace_bytes, void* stream_v, float* part_out = nullptr,
-            const Fp8Scales* fp8 = nullptr, int32_t max_sub = kMaxSubItems) {
+            const Fp8Scales* fp8 = nullptr, int32_t max_sub = kMaxSubItems, const SelfTest* selftest = nullptr) {
     // part_out != null: the result is a partial one (fp32 rows + their LSE in `lse`, no bf16 O)
     if (!shape) return YOCO_ERR_INVALID_ARG;
     int32_t rc = validate_shape(*shape, mode);
@@ -224,6 +270,7 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) ||
         !aligned(workspace, 256) || (lse && !aligned(lse, 4)))
         return YOCO_ERR_INVALID_ARG;
+    if ((rc = validate_layout(*shape, cu_kv_host, kv_len_host)) != YOCO_OK) return rc;
 
     DeviceState* dev = nullptr;
     if ((rc = device_state(&dev)) != YOCO_OK) return rc;
@@ -246,8 +293,18 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
         // the tables travel as kernel parameters: only the status word has to be cleared
         YOCO_CUDA_TRY(cudaMemsetAsync(ws, 0, kWorkspaceHeaderBytes, stream));
     } else {
-        // header (status word = 0) + work tables in one copy.  The source is pageable memory,
-        // which the runtime stages before the call returns, so the cache entry may go away.
+        // header (status word = 0) + work tables in one copy.  The source is pageable memory, which
+        // the runtime stages before the call returns, so the cache entry may go away afterwards --
+        // unless the stream is being recorded into a graph: the recorded copy reads the same host
+        // memory again at every replay, so such a plan is kept for the life of the process.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        YOCO_CUDA_TRY(cudaStreamIsCapturing(stream, &cap));
+        if (cap != cudaStreamCaptureStatusNone) {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            bool kept = false;
+            for (const auto& q : g_captured_plans) kept = kept || q == ready;
+            if (!kept) g_captured_plans.push_back(ready);
+        }
         YOCO_CUDA_TRY(cudaMemcpyAsync(ws, ready->blob.data(), ready->blob.size() * 4, cudaMemcpyHostToDevice,
                                       stream));
     }
@@ -288,6 +345,10 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             p.force_partial = part_out ? 1 : 0;
             p.sub_items = plan.sub_items;
             p.work_counter = reinterpret_cast<int32_t*>(ws + kWorkCounterOffset);
+            if (selftest) {
+                p.wait_limit_ns = selftest->wait_limit_ns;
+                p.selftest_skip_loads = 1;
+            }
             if (fp8) {
                 DecodeFp8Params p8{};
                 p8.base = p;
@@ -547,10 +608,6 @@ int32_t kv_append_impl(const yoco_kv_append_shape* shape, const void* X, const v
     if (!X || !Wgk || !Wgv || !K || !V || !kv_len_host) return YOCO_ERR_INVALID_ARG;
     if (!aligned(X, 16) || !aligned(Wgk, 16) || !aligned(Wgv, 16) || !aligned(K, 16) || !aligned(V, 16))
         return YOCO_ERR_INVALID_ARG;
-    DeviceState* dev = nullptr;
-    int32_t rc = device_state(&dev);
-    if (rc != YOCO_OK) return rc;
-
     KvAppendTables tab;
     std::memset(&tab, 0, sizeof tab);
     int64_t tok = 0;
@@ -561,6 +618,8 @@ int32_t kv_append_impl(const yoco_kv_append_shape* shape, const void* X, const v
         if (head_rows < n) return YOCO_ERR_INVALID_ARG;
         if (cu_kv_host) {
             if (cu_kv_host[i] < 0 || cu_kv_host[i + 1] < cu_kv_host[i]) return YOCO_ERR_INVALID_ARG;
+            // the rows written for sequence i may not reach into the next sequence's heads
+            if ((int64_t)cu_kv_host[i + 1] - cu_kv_host[i] < head_rows) return YOCO_ERR_INVALID_ARG;
             tok = cu_kv_host[i];
         }
         const int64_t row0 = tok * s.Hkv + (n - s.T);
@@ -569,6 +628,9 @@ int32_t kv_append_impl(const yoco_kv_append_shape* shape, const void* X, const v
         tab.head_rows[i] = (int32_t)head_rows;
         if (!cu_kv_host) tok += head_rows;
     }
+    DeviceState* dev = nullptr;
+    int32_t rc = device_state(&dev);
+    if (rc != YOCO_OK) return rc;
     KvAppendParams p{};
     p.X = static_cast<const __nv_bfloat16*>(X);
     p.K = static_cast<__nv_bfloat16*>(K);
@@ -618,13 +680,55 @@ int32_t yoco_kv_append_status(void* stream) {
     return word == kStatusOk ? YOCO_OK : YOCO_ERR_TIMEOUT;
 }
 
-int32_t yoco_xattn_status(const void* workspace, void* stream) {
-    if (!workspace) return YOCO_ERR_INVALID_ARG;
+int32_t yoco_kv_append_status_detail(void* stream, int32_t* wait_class, int32_t* cta) {
     int32_t word = 0;
+    YOCO_CUDA_TRY(read_and_clear_kv_append_status(&word, reinterpret_cast<cudaStream_t>(stream)));
+    return yoco_xattn_decode_status_word(word, wait_class, cta);
+}
+
+namespace {
+// reads the status word of `workspace`, or of the built-in buffer of the current device when null
+int32_t read_status_word(const void* workspace, void* stream, int32_t* word) {
+    void* builtin = nullptr;
+    if (!workspace) {
+        int32_t rc = static_scratch_address(&builtin);
+        if (rc != YOCO_OK) return rc;
+        workspace = builtin;
+    }
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    YOCO_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost, s));
+    YOCO_CUDA_TRY(cudaMemcpyAsync(word, workspace, sizeof *word, cudaMemcpyDeviceToHost, s));
     YOCO_CUDA_TRY(cudaStreamSynchronize(s));
+    return YOCO_OK;
+}
+}  // namespace
+
+int32_t yoco_xattn_status(const void* workspace, void* stream) {
+    int32_t word = 0;
+    int32_t rc = read_status_word(workspace, stream, &word);
+    if (rc != YOCO_OK) return rc;
     return word == kStatusOk ? YOCO_OK : YOCO_ERR_TIMEOUT;
+}
+
+int32_t yoco_xattn_status_detail(const void* workspace, void* stream, int32_t* wait_class, int32_t* cta) {
+    int32_t word = 0;
+    int32_t rc = read_status_word(workspace, stream, &word);
+    if (rc != YOCO_OK) return rc;
+    return yoco_xattn_decode_status_word(word, wait_class, cta);
+}
+
+int32_t yoco_xattn_decode_status_word(int32_t word, int32_t* wait_class, int32_t* cta) {
+    if (wait_class) *wait_class = word & 0xFF;
+    if (cta) *cta = (int32_t)((uint32_t)word >> 8) - 1;
+    return word == kStatusOk ? YOCO_OK : YOCO_ERR_TIMEOUT;
+}
+
+int32_t yoco_xattn_selftest_wait_expiry(const yoco_xattn_shape* shape, const void* Q, const void* K, const void* V,
+                                        const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O,
+                                        void* workspace, size_t workspace_bytes, int32_t limit_ms, void* stream) {
+    if (limit_ms <= 0 || limit_ms > 1000) return YOCO_ERR_INVALID_ARG;
+    const SelfTest st{(int64_t)limit_ms * 1000000ll};
+    return run(shape, YOCO_MODE_DECODE, Q, K, V, cu_kv_host, kv_len_host, O, nullptr, workspace, workspace_bytes,
+               stream, nullptr, nullptr, 1, &st);
 }
 
 int32_t yoco_xattn_profile_enable(int32_t max_records) {

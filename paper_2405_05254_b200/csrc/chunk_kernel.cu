@@ -36,7 +36,7 @@ struct CCfg {
     static constexpr int OFF_V = OFF_K + 2 * TILE_BYTES;
     static constexpr int OFF_P = OFF_V + 2 * TILE_BYTES;
     static constexpr int OFF_BAR = OFF_P + 2 * P_BYTES;
-    static constexpr int NUM_BARS = 18;
+    static constexpr int NUM_BARS = 19;
     static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16;
 };
 
@@ -61,20 +61,22 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     uint64_t* s_empty = bars + 12;  // [2]
     uint64_t* p_full = bars + 14;   // [2]
     uint64_t* p_empty = bars + 16;  // [2]
+    uint64_t* drain_bar = bars + 18; // everything the issuer started has finished
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int group = blockIdx.x / p.m_tiles, m_tile = blockIdx.x - group * p.m_tiles;
     const int seg_lo = p.group_begin[group], seg_hi = p.group_begin[group + 1];
-    const Abort ab{abort_flag, p.status};
+    const Abort ab{abort_flag, p.status, kWaitLimitNs};
     const bool aligned_ok = (smem_u32(smem) & 1023u) == 0;
 
     if (threadIdx.x == 0) {
         *abort_flag = aligned_ok ? 0 : 1;
-        if (!aligned_ok) atomicExch(p.status, kStatusTimeout + 1);
+        if (!aligned_ok) atomicCAS(p.status, 0, status_word(kWaitMisaligned, linear_cta()));
         mbar_init(q_full, 1);
         mbar_init(q_empty, 1);
+        mbar_init(drain_bar, 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&k_full[b], 1);
             mbar_init(&k_empty[b], 1);
@@ -103,27 +105,38 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             tma_prefetch_desc(&tmK);
             tma_prefetch_desc(&tmV);
             uint32_t it = 0;
+            uint32_t q_armed = 0, k_armed = 0, v_armed = 0;   // copies started, for the drain on the way out
             bool ok = true;
             for (int si = seg_lo; si < seg_hi && ok; ++si) {
                 const DevSegment seg = p.segments[si];
                 const uint32_t sidx = si - seg_lo;
-                if (!(ok = wait_or_abort(q_empty, (sidx & 1u) ^ 1u, ab))) break;
+                if (!(ok = wait_or_abort(q_empty, (sidx & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
+                ++q_armed;
                 mbar_expect_tx(q_full, C::TILE_BYTES);
                 for (int h = 0; h < HALVES; ++h)
                     tma_load_2d(smem + C::OFF_Q + h * HALF_BYTES, &tmQ, h * 64, seg.q_row0 + m_tile * BM, q_full);
                 for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
                     const uint32_t b = it & 1u, n = it >> 1;
                     const int row = seg.kv_row0 + (k0 - seg.k_begin);
-                    if (!(ok = wait_or_abort(&k_empty[b], (n & 1u) ^ 1u, ab))) break;
+                    if (!(ok = wait_or_abort(&k_empty[b], (n & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
+                    ++k_armed;
                     mbar_expect_tx(&k_full[b], C::TILE_BYTES);
                     for (int h = 0; h < HALVES; ++h)
                         tma_load_2d(smem + C::OFF_K + b * C::TILE_BYTES + h * HALF_BYTES, &tmK, h * 64, row, &k_full[b]);
-                    if (!(ok = wait_or_abort(&v_empty[b], (n & 1u) ^ 1u, ab))) break;
+                    if (!(ok = wait_or_abort(&v_empty[b], (n & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
+                    ++v_armed;
                     mbar_expect_tx(&v_full[b], C::TILE_BYTES);
                     for (int h = 0; h < HALVES; ++h)
                         tma_load_2d(smem + C::OFF_V + b * C::TILE_BYTES + h * HALF_BYTES, &tmV, h * 64, row, &v_full[b]);
                 }
             }
+            // Every copy this thread started must have landed before the CTA may end (at once when all
+            // went well: the tiles were consumed long ago).
+            bool drained = q_armed == 0 || drain_wait(q_full, (q_armed - 1) & 1u, ab);
+            for (uint32_t k = k_armed > 2 ? k_armed - 2 : 0; drained && k < k_armed; ++k)
+                drained = drain_wait(&k_full[k & 1u], (k >> 1) & 1u, ab);
+            for (uint32_t k = v_armed > 2 ? v_armed - 2 : 0; drained && k < v_armed; ++k)
+                drained = drain_wait(&v_full[k & 1u], (k >> 1) & 1u, ab);
         }
     } else if (warp == 1) {
         // ======================================= MMA issuer ==================================
@@ -143,8 +156,8 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             uint32_t prev_it = 0;
             auto issue_pv = [&](uint32_t i, bool first_of_segment) -> bool {
                 const uint32_t b = i & 1u, n = i >> 1;
-                if (!warp_wait(&p_full[b], n & 1u, ab)) return false;
-                if (!warp_wait(&v_full[b], n & 1u, ab)) return false;
+                if (!warp_wait(&p_full[b], n & 1u, ab, kWaitTensor)) return false;
+                if (!warp_wait(&v_full[b], n & 1u, ab, kWaitRingFull)) return false;
                 tc_fence_after();
                 const uint64_t p_desc = make_desc(sbase + C::OFF_P + b * C::P_BYTES, 16, 1024);
                 const uint64_t v_desc = make_desc(sbase + C::OFF_V + b * C::TILE_BYTES, BN * 128, 1024);
@@ -169,11 +182,11 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     if (!(ok = issue_pv(prev_it, prev_first))) break;
                     have_prev = false;
                 }
-                if (!(ok = warp_wait(q_full, sidx & 1u, ab))) break;
+                if (!(ok = warp_wait(q_full, sidx & 1u, ab, kWaitRingFull))) break;
                 for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
                     const uint32_t b = it & 1u, n = it >> 1;
-                    if (!(ok = warp_wait(&k_full[b], n & 1u, ab))) break;
-                    if (!(ok = warp_wait(&s_empty[b], (n & 1u) ^ 1u, ab))) break;
+                    if (!(ok = warp_wait(&k_full[b], n & 1u, ab, kWaitRingFull))) break;
+                    if (!(ok = warp_wait(&s_empty[b], (n & 1u) ^ 1u, ab, kWaitTensor))) break;
                     tc_fence_after();
                     const uint64_t k_desc = make_desc(sbase + C::OFF_K + b * C::TILE_BYTES, 16, 1024);
                     if (elect_one()) {
@@ -195,6 +208,14 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 }
             }
             if (ok && have_prev) issue_pv(prev_it, prev_first);
+            // Nothing this warp issued may still be running (or still owe an arrive on one of this CTA's
+            // barriers) when tensor memory is released and the CTA ends: one more commit, which
+            // completes after every earlier product and commit of the issuing lane, and a wait for it.
+            if (elect_one()) {
+                umma_commit(drain_bar);
+                drain_wait(drain_bar, 0u, ab);
+            }
+            __syncwarp();
         }
     } else {
         // ======================================= softmax warps ===============================
@@ -220,7 +241,7 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
                 if (!ok) continue;
                 const uint32_t b = it & 1u, n = it >> 1;
-                if (!(ok = warp_wait(&s_full[b], n & 1u, ab))) continue;
+                if (!(ok = warp_wait(&s_full[b], n & 1u, ab, kWaitTensor))) continue;
                 tc_fence_after();
                 float s[BN];
 #pragma unroll
@@ -252,7 +273,7 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 if (__any_sync(0xffffffffu, grow) && it > seg_first_it) {
                     // O holds the sums of the earlier tiles of this segment: wait for the last PV
                     const uint32_t pi = it - 1;
-                    if (!(ok = warp_wait(&p_empty[pi & 1u], (pi >> 1) & 1u, ab))) continue;
+                    if (!(ok = warp_wait(&p_empty[pi & 1u], (pi >> 1) & 1u, ab, kWaitTensor))) continue;
                     tc_fence_after();
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
@@ -269,7 +290,7 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
 
                 // P buffer b is free once PV of tile it-2 has completed
-                if (!(ok = warp_wait(&p_empty[b], (n & 1u) ^ 1u, ab))) continue;
+                if (!(ok = warp_wait(&p_empty[b], (n & 1u) ^ 1u, ab, kWaitTensor))) continue;
                 uint8_t* prow = smem + C::OFF_P + b * C::P_BYTES + row * 128;
                 float ls4[4] = {0.f, 0.f, 0.f, 0.f};
                 const float neg_m = -m_use;
@@ -294,7 +315,7 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 // keys past the end of the sequence: their V rows may hold anything; zero them so
                 // that 0 * garbage cannot make NaN
                 if (k0 + BN > seg.n_kv) {
-                    if (!(ok = warp_wait(&v_full[b], n & 1u, ab))) continue;
+                    if (!(ok = warp_wait(&v_full[b], n & 1u, ab, kWaitRingFull))) continue;
                     if (k0 + row >= seg.n_kv) {
                         uint8_t* vrow = smem + C::OFF_V + b * C::TILE_BYTES + row * 128;
 #pragma unroll
@@ -312,7 +333,7 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             // ---- end of segment: O is complete once the last PV has finished ----
             if (ok && it > seg_first_it) {
                 const uint32_t pi = it - 1;
-                ok = warp_wait(&p_empty[pi & 1u], (pi >> 1) & 1u, ab);
+                ok = warp_wait(&p_empty[pi & 1u], (pi >> 1) & 1u, ab, kWaitTensor);
             }
             if (ok) {
                 tc_fence_after();

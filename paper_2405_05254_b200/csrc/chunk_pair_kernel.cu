@@ -49,7 +49,7 @@ struct PCfg {
     static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
     static constexpr int OFF_V = OFF_K + K_STAGES * TILE_BYTES;
     static constexpr int OFF_BAR = OFF_V + V_STAGES * TILE_BYTES;
-    static constexpr int NUM_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 12;
+    static constexpr int NUM_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 12 + 3;
     static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16;
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
 };
@@ -91,20 +91,22 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     uint64_t* s_full = v_empty + VS;         // [2][2]  S_r^h holds the scores of the current half step
     uint64_t* p_full = s_full + 4;           // [2][2]  P_r^h has been written over S_r^h
     uint64_t* pv_done = p_full + 4;          // [2][2]  O_r includes the current half step; P_r^h is dead
+    uint64_t* drain_bar = pv_done + 4;       // [3]     everything issuer warp 1 + i started has finished
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int group = blockIdx.x / p.m_tiles, m_tile = blockIdx.x - group * p.m_tiles;
     const int seg_lo = p.group_begin[group], seg_hi = p.group_begin[group + 1];
-    const Abort ab{abort_flag, p.status};
+    const Abort ab{abort_flag, p.status, kWaitLimitNs};
     const bool aligned_ok = (smem_u32(smem) & 1023u) == 0;
 
     if (threadIdx.x == 0) {
         *abort_flag = aligned_ok ? 0 : 1;
-        if (!aligned_ok) atomicExch(p.status, kStatusTimeout + 1);
+        if (!aligned_ok) atomicCAS(p.status, 0, status_word(kWaitMisaligned, linear_cta()));
         mbar_init(q_full, 1);
         mbar_init(q_empty, 2);
+        for (int b = 0; b < 3; ++b) mbar_init(&drain_bar[b], 1);
         for (int b = 0; b < KS; ++b) {
             mbar_init(&k_full[b], 1);
             mbar_init(&k_empty[b], 2);            // released by both issuers
@@ -139,11 +141,13 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tma_prefetch_desc(&tmK);
             tma_prefetch_desc(&tmV);
             uint32_t it = 0;
+            uint32_t q_armed = 0, k_armed = 0, v_armed = 0;   // copies started, for the drain on the way out
             bool ok = true;
             for (int si = seg_lo; si < seg_hi && ok; ++si) {
                 const DevSegment seg = p.segments[si];
                 const uint32_t sidx = si - seg_lo;
-                if (!(ok = wait_or_abort(q_empty, (sidx & 1u) ^ 1u, ab))) break;
+                if (!(ok = wait_or_abort(q_empty, (sidx & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
+                ++q_armed;
                 mbar_expect_tx(q_full, 2 * C::TILE_BYTES);
                 for (int r = 0; r < 2; ++r)
                     for (int h = 0; h < HALVES; ++h)
@@ -152,19 +156,28 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
                     const int row = seg.kv_row0 + (k0 - seg.k_begin);
                     const uint32_t kb = it % KS, kn = it / KS;
-                    if (!(ok = wait_or_abort(&k_empty[kb], (kn & 1u) ^ 1u, ab))) break;
+                    if (!(ok = wait_or_abort(&k_empty[kb], (kn & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
+                    ++k_armed;
                     mbar_expect_tx(&k_full[kb], C::TILE_BYTES);
                     for (int h = 0; h < HALVES; ++h)
                         tma_load_2d(smem + C::OFF_K + kb * C::TILE_BYTES + h * HALF_BYTES, &tmK, h * 64, row,
                                     &k_full[kb]);
                     const uint32_t vb = it % VS, vn = it / VS;
-                    if (!(ok = wait_or_abort(&v_empty[vb], (vn & 1u) ^ 1u, ab))) break;
+                    if (!(ok = wait_or_abort(&v_empty[vb], (vn & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
+                    ++v_armed;
                     mbar_expect_tx(&v_full[vb], C::TILE_BYTES);
                     for (int h = 0; h < HALVES; ++h)
                         tma_load_2d(smem + C::OFF_V + vb * C::TILE_BYTES + h * HALF_BYTES, &tmV, h * 64, row,
                                     &v_full[vb]);
                 }
             }
+            // Every copy this thread started must have landed before the CTA may end (at once when all
+            // went well: the tiles were consumed long ago).
+            bool drained = q_armed == 0 || drain_wait(q_full, (q_armed - 1) & 1u, ab);
+            for (uint32_t k = k_armed > (uint32_t)KS ? k_armed - KS : 0; drained && k < k_armed; ++k)
+                drained = drain_wait(&k_full[k % KS], (k / KS) & 1u, ab);
+            for (uint32_t k = v_armed > (uint32_t)VS ? v_armed - VS : 0; drained && k < v_armed; ++k)
+                drained = drain_wait(&v_full[k % VS], (k / VS) & 1u, ab);
         } else if (warp >= 1 && aligned_ok) {
             // =================================== MMA issuers =================================
             // Issuing a tensor-core instruction costs a single warp tens of cycles (a chain of
@@ -224,13 +237,13 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 while (ok && c.valid) {
                     if (c.h == 0) {
                         if (c.first_tile) {
-                            ok = warp_wait(q_full, seg_par, ab);
+                            ok = warp_wait(q_full, seg_par, ab, kWaitRingFull);
                             seg_par ^= 1u;
                         }
-                        ok = ok && warp_wait(&k_full[c.kb], c.kph, ab);
+                        ok = ok && warp_wait(&k_full[c.kb], c.kph, ab, kWaitRingFull);
                     }
                     // the buffer S_r^h still holds the P of the previous key tile until its product ran
-                    if (ok && tiles_seen > 0) ok = warp_wait(&pv_done[r * 2 + c.h], c.tp ^ 1u, ab);
+                    if (ok && tiles_seen > 0) ok = warp_wait(&pv_done[r * 2 + c.h], c.tp ^ 1u, ab, kWaitTensor);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t k_lo = desc_lo(sbase + C::OFF_K + c.kb * C::TILE_BYTES + c.h * BH * 128, 16);
@@ -254,12 +267,12 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 }
             } else {
                 while (ok && c.valid) {
-                    if (c.h == 0) ok = warp_wait(&v_full[c.vb], c.vph, ab);
+                    if (c.h == 0) ok = warp_wait(&v_full[c.vb], c.vph, ab, kWaitRingFull);
                     const uint32_t v_lo = desc_lo(sbase + C::OFF_V + c.vb * C::TILE_BYTES + c.h * BH * 128, BN * 128);
                     const uint32_t first = (c.first_tile && c.h == 0) ? 0u : 1u;
 #pragma unroll
                     for (int r = 0; r < 2; ++r) {
-                        ok = ok && warp_wait(&p_full[r * 2 + c.h], c.tp, ab);
+                        ok = ok && warp_wait(&p_full[r * 2 + c.h], c.tp, ab, kWaitTensor);
                         if (!ok) break;
                         tc_fence_after();
                         const uint32_t a_tmem = tmem_base + r * BN + c.h * BH;
@@ -277,6 +290,14 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     cur_next();
                 }
             }
+            // Nothing this warp issued may still be running (or still owe an arrive on one of this CTA's
+            // barriers) when tensor memory is released and the CTA ends: one more commit, which
+            // completes after every earlier product and commit of the issuing lane, and a wait for it.
+            if (elect_one()) {
+                umma_commit(&drain_bar[warp - 1]);
+                drain_wait(&drain_bar[warp - 1], 0u, ab);
+            }
+            __syncwarp();
         }
     } else {
         // ======================================= softmax warpgroups ==========================
@@ -308,7 +329,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     if (!ok) continue;
                     const uint32_t u = 2 * it + h;             // half step number
                     const int kh = k0 + h * BH;                // first key of the half step
-                    if (!(ok = warp_wait(&s_full[r * 2 + h], it & 1u, ab))) continue;
+                    if (!(ok = warp_wait(&s_full[r * 2 + h], it & 1u, ab, kWaitTensor))) continue;
                     tc_fence_after();
                     float s[BH];
 #pragma unroll
@@ -338,7 +359,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         // O_r holds the sums of the earlier half steps of this segment: wait for
                         // the product of the previous one (the other buffer; it belongs to this key
                         // tile when h = 1, to the previous one when h = 0)
-                        if (!(ok = warp_wait(&pv_done[r * 2 + (h ^ 1)], (it ^ (h ^ 1)) & 1u, ab))) continue;
+                        if (!(ok = warp_wait(&pv_done[r * 2 + (h ^ 1)], (it ^ (h ^ 1)) & 1u, ab, kWaitTensor))) continue;
                         tc_fence_after();
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c) {
@@ -407,7 +428,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     // the first half step, each before it releases its own first product on this tile.
                     if (h == 0 && k0 + BN > seg.n_kv) {
                         const uint32_t vb = it % VS, vn = it / VS;
-                        if (!(ok = warp_wait(&v_full[vb], vn & 1u, ab))) continue;
+                        if (!(ok = warp_wait(&v_full[vb], vn & 1u, ab, kWaitRingFull))) continue;
                         if (k0 + row >= seg.n_kv) {
                             uint8_t* vrow = smem + C::OFF_V + vb * C::TILE_BYTES + row * 128;
 #pragma unroll
@@ -426,7 +447,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
             // ---- end of segment: O_r is complete once the last PV has finished ----
             // (the products of one row tile complete in order, so the last one covers all)
-            if (ok && it > seg_first_it) ok = warp_wait(&pv_done[r * 2 + 1], (it - 1) & 1u, ab);
+            if (ok && it > seg_first_it) ok = warp_wait(&pv_done[r * 2 + 1], (it - 1) & 1u, ab, kWaitTensor);
             if (ok) {
                 tc_fence_after();
                 const bool has = l > 0.f;

@@ -79,16 +79,20 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
     float* merge_ml = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES + C::MERGE_O_BYTES);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES + C::MERGE_O_BYTES + C::MERGE_ML_BYTES);
     uint64_t* empty_bar = full_bar + STAGES;
+    volatile int* give_up = reinterpret_cast<volatile int*>(empty_bar + STAGES);   // some thread ran out of patience
+    static_assert(2 * STAGES * 8 + 4 <= 128, "barrier block");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int seg_lo = group_begin[blockIdx.x], seg_hi = group_begin[blockIdx.x + 1];
     asm volatile("griddepcontrol.launch_dependents;");
 
     if ((smem_u32(smem) & 1023u) != 0) {   // the swizzle arithmetic below needs 1 KB alignment
-        if (threadIdx.x == 0) atomicExch(p.status, kStatusTimeout + 1);
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, status_word(kWaitMisaligned, linear_cta()));
         return;
     }
+    const Abort ab{give_up, p.status, p.wait_limit_ns > 0 ? p.wait_limit_ns : kWaitLimitNs};
     if (threadIdx.x == 0) {
+        *give_up = 0;
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);                 // released by the one warp that read the tile
@@ -108,8 +112,7 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
                 const DevSegment seg = segments[si];
                 for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += TILE_N, ++it) {
                     const uint32_t stage = it % STAGES, round = it / STAGES;
-                    if (!mbar_wait(&empty_bar[stage], (round & 1u) ^ 1u)) {
-                        atomicExch(p.status, kStatusTimeout);
+                    if (!wait_or_abort(&empty_bar[stage], (round & 1u) ^ 1u, ab, kWaitRingEmpty)) {
                         ok = false;
                         break;
                     }
@@ -120,6 +123,11 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
                     tma_load_2d(kdst + TENSOR_BYTES, &tmV, 0, row, &full_bar[stage]);
                 }
             }
+            // every copy this thread armed must have landed before it leaves (the CTA ends with its last
+            // thread, and its shared memory then belongs to another CTA); at once when all went well
+            const uint32_t in_flight = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+            for (uint32_t k = it - in_flight; k < it; ++k)
+                if (!drain_wait(&full_bar[k % STAGES], (k / STAGES) & 1u, ab)) break;
         }
         return;
     }
@@ -172,9 +180,8 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
         for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += TILE_N, ++it) {
             if (!ok || (int)(it % kConsumerWarps) != warp) continue;       // not this warp's tile
             const uint32_t stage = it % STAGES, round = it / STAGES;
-            if (!mbar_wait(&full_bar[stage], round & 1u)) {
-                atomicExch(p.status, kStatusTimeout);
-                ok = false;
+            if (!wait_or_abort(&full_bar[stage], round & 1u, ab, kWaitRingFull)) {
+                ok = false;         // this warp touches no tile any more; it still walks to the barriers below
                 continue;
             }
             const uint32_t kbase = smem_u32(stage_mem + stage * STAGE_BYTES);

@@ -79,9 +79,10 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
     asm volatile("griddepcontrol.launch_dependents;");
 
     if ((smem_u32(smem) & 1023u) != 0) {   // the swizzle arithmetic below needs 1 KB alignment
-        if (threadIdx.x == 0) atomicExch(p.status, kStatusTimeout + 1);
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, status_word(kWaitMisaligned, linear_cta()));
         return;
     }
+    const Abort ab{give_up, p.status, p.wait_limit_ns > 0 ? p.wait_limit_ns : kWaitLimitNs};
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full_bar[s], 1);
@@ -106,10 +107,7 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
             int item = blockIdx.x;
             for (uint32_t n = 0; ok; ++n) {
                 // hand the item (or the end mark) to the consumers
-                if (!mbar_wait(&item_empty[n & 1u], ((n >> 1) & 1u) ^ 1u)) {
-                    atomicExch(p.status, kStatusTimeout);
-                    break;
-                }
+                if (!wait_or_abort(&item_empty[n & 1u], ((n >> 1) & 1u) ^ 1u, ab, kWaitItemQueue)) break;
                 item_q[n & 1u] = item;
                 mbar_arrive(&item_full[n & 1u]);
                 if (item >= n_items) break;
@@ -133,8 +131,10 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
                     const int k_hi = min(seg.k_begin + s_hi * TILE_N, seg.k_end);
                     for (int k0 = k_lo; k0 < k_hi; k0 += TILE_N, ++it) {
                         const uint32_t stage = it % STAGES, round = it / STAGES;
-                        if (!mbar_wait(&empty_bar[stage], (round & 1u) ^ 1u)) {
-                            atomicExch(p.status, kStatusTimeout);
+                        // self-test of the give-up path: nothing is armed, so no stage is needed either
+                        // and the wait that runs out is the consumers' first wait for a tile
+                        if (p.selftest_skip_loads) continue;
+                        if (!wait_or_abort(&empty_bar[stage], (round & 1u) ^ 1u, ab, kWaitRingEmpty)) {
                             ok = false;
                             break;
                         }
@@ -152,6 +152,15 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
                 // all loads of this item are on their way: claim the next one
                 item = R > 1 ? n_groups + atomicAdd(p.work_counter, 1) : n_items;
             }
+            // Before this thread leaves, every copy it armed must have landed: the CTA ends when its
+            // last thread does, and a copy that lands later would write into (and arrive on barriers
+            // in) shared memory that already belongs to another CTA.  When all went well the
+            // consumers are still reading these tiles and the waits return at once.
+            if (!p.selftest_skip_loads) {
+                const uint32_t in_flight = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+                for (uint32_t k = it - in_flight; k < it; ++k)
+                    if (!drain_wait(&full_bar[k % STAGES], (k / STAGES) & 1u, ab)) break;
+            }
         }
         return;
     }
@@ -165,13 +174,10 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
     for (uint32_t n_item = 0;; ++n_item) {
         // the next item from the producer; the four warps must take the same decision, so a warp
         // that gives up waiting says so before the barrier and all of them leave together
-        if (!mbar_wait(&item_full[n_item & 1u], (n_item >> 1) & 1u)) {
-            atomicExch(p.status, kStatusTimeout);
-            *give_up = 1;
-        }
+        const bool got_item = wait_or_abort(&item_full[n_item & 1u], (n_item >> 1) & 1u, ab, kWaitItemQueue);
         const int item = item_q[n_item & 1u];
-        named_barrier_sync(1, kConsumerWarps * 32);
-        if (*give_up) break;
+        // one answer for all four warps (a barrier that ORs): nobody reads the flag on its own
+        if (named_barrier_or(1, kConsumerWarps * 32, !got_item || !ok)) break;
         if (lane == 0) mbar_arrive(&item_empty[n_item & 1u]);
         if (item >= n_items) break;
         const int grp = item % n_groups, piece = item / n_groups;
@@ -226,9 +232,8 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
             for (int k0 = k_lo; k0 < k_hi; k0 += TILE_N, ++it) {
                 if (!ok) continue;
                 const uint32_t stage = it % STAGES, round = it / STAGES;
-                if (!mbar_wait(&full_bar[stage], round & 1u)) {
-                    atomicExch(p.status, kStatusTimeout);
-                    ok = false;
+                if (!wait_or_abort(&full_bar[stage], round & 1u, ab, kWaitRingFull)) {
+                    ok = false;     // this warp touches no tile any more; it still walks to the barriers below
                     continue;
                 }
                 const int kw = k0 + warp * 16;          // first key of this warp's slice

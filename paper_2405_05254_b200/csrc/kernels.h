@@ -10,9 +10,23 @@
 
 namespace yoco {
 
-// device status word values (first int32 of the workspace)
 constexpr int32_t kStatusOk = 0;
-constexpr int32_t kStatusTimeout = 1;
+// Status word (first int32 of a workspace, or the append kernel's own word): 0 = ok, otherwise
+//   bits 0-7   which kind of wait ran out (WaitClass)
+//   bits 8-31  1 + linear index of the CTA that gave up first
+// The first failure wins (compare-and-swap against 0), so the word names where the trouble began.
+enum WaitClass : int32_t {
+    kWaitItemQueue = 1,   // decode: next work item from the producer / queue entry read by the consumers
+    kWaitRingFull = 2,    // a consumer waiting for a K/V (or Q, X, W) tile to land
+    kWaitRingEmpty = 3,   // the producer waiting for a stage to be released
+    kWaitTensor = 4,      // a tensor-core hand-over: scores ready, P written, product finished
+    kWaitDrain = 5,       // leaving: a copy or product that had been started did not finish in time
+    kWaitMisaligned = 6,  // dynamic shared memory not 1 KB aligned (no wait involved; nothing ran)
+};
+__host__ __device__ constexpr int32_t status_word(int32_t wait_class, int32_t cta) {
+    return wait_class | ((cta + 1) << 8);
+}
+
 
 // Work tables small enough to travel as kernel parameters (the decode call then needs no
 // host-to-device copy): every benchmark shape fits; larger problems read them from the workspace.
@@ -74,6 +88,9 @@ struct DecodeParams {
     int32_t force_partial;      // write every segment to its partial slot, even of an unsplit stream
     int32_t sub_items;          // pieces per group (plan.h: sub_bound); slot = segment slot * sub_items + piece
     int32_t* work_counter;      // zeroed before the launch; hands out the pieces beyond each CTA's first
+    int64_t wait_limit_ns;      // 0 = the default limit of a bounded wait
+    int32_t selftest_skip_loads;// self-test of the give-up path: the producer arms no copy, so the first
+                                // consumer wait runs out (with nothing in flight) and the kernel returns
 };
 // tmK / tmV: 2-D tensor maps over the [rows, d] view of K and V, box {64, kDecodeTileN},
 // 128-byte swizzle.

@@ -35,7 +35,7 @@ constexpr int TILE_BYTES = 2 * HALF_BYTES;       // an X tile [128 tokens, 128 k
 constexpr int STAGES = 3;
 constexpr int STAGE_BYTES = 2 * TILE_BYTES;
 constexpr int OFF_BAR = STAGES * STAGE_BYTES;
-constexpr int SMEM_BYTES = OFF_BAR + (2 * STAGES + 1) * 8 + 16;
+constexpr int SMEM_BYTES = OFF_BAR + (2 * STAGES + 2) * 8 + 16;
 constexpr uint32_t TMEM_COLS = 128;
 
 // FP8 = false: rows stored as bf16.  FP8 = true: rows divided by the head's scale and stored as FP8
@@ -49,24 +49,26 @@ kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + OFF_BAR);   // [STAGES] tile pair has landed
     uint64_t* empty = full + STAGES;                                // [STAGES] MMA and row sums are done with it
     uint64_t* acc_full = empty + STAGES;                            // accumulator complete
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+    uint64_t* drain_bar = acc_full + 1;                             // everything the issuer started has finished
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * BN;          // first output column (K^ columns, then V^ columns)
     const int m0 = blockIdx.y * BM;          // first token
     const int KT = p.d_model / BK;
-    const Abort ab{abort_flag, &g_kv_append_status};
+    const Abort ab{abort_flag, &g_kv_append_status, kWaitLimitNs};
     const bool aligned_ok = (smem_u32(smem) & 1023u) == 0;
 
     if (threadIdx.x == 0) {
         *abort_flag = aligned_ok ? 0 : 1;
-        if (!aligned_ok) atomicExch(&g_kv_append_status, kStatusTimeout + 1);
+        if (!aligned_ok) atomicCAS(&g_kv_append_status, 0, status_word(kWaitMisaligned, linear_cta()));
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1 + 4);     // one tcgen05.commit + four row-sum warps
         }
         mbar_init(acc_full, 1);
+        mbar_init(drain_bar, 1);
         mbar_fence_init();
     }
     if (warp == 1) {
@@ -86,9 +88,10 @@ kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             const int nw = n0 - (is_v ? p.n_half : 0);
             tma_prefetch_desc(&tmX);
             tma_prefetch_desc(tmW);
-            for (int kt = 0; kt < KT; ++kt) {
+            int armed = 0;                                   // copies started, for the drain on the way out
+            for (int kt = 0; kt < KT; ++kt, ++armed) {
                 const uint32_t s = kt % STAGES, ph = (kt / STAGES) & 1u;
-                if (!wait_or_abort(&empty[s], ph ^ 1u, ab)) break;
+                if (!wait_or_abort(&empty[s], ph ^ 1u, ab, kWaitRingEmpty)) break;
                 uint8_t* a = smem + s * STAGE_BYTES;
                 uint8_t* b = a + TILE_BYTES;
                 mbar_expect_tx(&full[s], STAGE_BYTES);
@@ -97,6 +100,9 @@ kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                     tma_load_2d(b + h * HALF_BYTES, tmW, nw + h * 64, kt * BK, &full[s]);
                 }
             }
+            // every copy this thread started must have landed before the CTA may end
+            for (int k = armed > STAGES ? armed - STAGES : 0; k < armed; ++k)
+                if (!drain_wait(&full[k % STAGES], (uint32_t)(k / STAGES) & 1u, ab)) break;
         }
     } else if (warp == 1) {
         // ======================================= MMA issuer ==================================
@@ -106,7 +112,7 @@ kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             bool ok = true;
             for (int kt = 0; kt < KT && ok; ++kt) {
                 const uint32_t s = kt % STAGES, ph = (kt / STAGES) & 1u;
-                if (!(ok = warp_wait(&full[s], ph, ab))) break;
+                if (!(ok = warp_wait(&full[s], ph, ab, kWaitRingFull))) break;
                 tc_fence_after();
                 const uint32_t a_lo = desc_lo(sbase + s * STAGE_BYTES, 16);
                 const uint32_t b_lo = desc_lo(sbase + s * STAGE_BYTES + TILE_BYTES, BK * 128);
@@ -123,6 +129,12 @@ kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                 }
                 __syncwarp();
             }
+            // nothing this warp issued may still be running when tensor memory is released and the CTA ends
+            if (elect_one()) {
+                umma_commit(drain_bar);
+                drain_wait(drain_bar, 0u, ab);
+            }
+            __syncwarp();
         }
     } else {
         // ============================ row statistics, then epilogue ==========================
@@ -134,7 +146,7 @@ kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         for (int kt = 0; kt < KT; ++kt) {
             if (!ok) continue;
             const uint32_t s = kt % STAGES, ph = (kt / STAGES) & 1u;
-            if (!(ok = warp_wait(&full[s], ph, ab))) continue;
+            if (!(ok = warp_wait(&full[s], ph, ab, kWaitRingFull))) continue;
             const uint8_t* a = smem + s * STAGE_BYTES + row * 128;
             float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -156,7 +168,7 @@ kv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[s]);
         }
-        if (ok) ok = warp_wait(acc_full, 0u, ab);
+        if (ok) ok = warp_wait(acc_full, 0u, ab, kWaitTensor);
         if (ok) {
             tc_fence_after();
             const float r = 1.f / sqrtf(ss / (float)p.d_model + p.eps);
@@ -285,16 +297,20 @@ kv_append_small_kernel(const __grid_constant__ CUtensorMap tmWk, const __grid_co
     const int n_chunks = k_slice / SK_KBOX;
     const CUtensorMap* tmW = is_v ? &tmWv : &tmWk;
     bool ok = (smem_u32(smem) & 1023u) == 0;
-    if (!ok && threadIdx.x == 0) atomicExch(&g_kv_append_status, kStatusTimeout + 1);
+    if (!ok && threadIdx.x == 0) atomicCAS(&g_kv_append_status, 0, status_word(kWaitMisaligned, linear_cta()));
+    volatile int* give_up = reinterpret_cast<volatile int*>(full + SK_STAGES);   // behind the barriers
+    const Abort ab{give_up, &g_kv_append_status, kWaitLimitNs};
+    int armed = 0;                                          // thread 0: copies started
 
     if (threadIdx.x == 0) {
+        *give_up = 0;
         for (int s = 0; s < SK_STAGES; ++s) mbar_init(&full[s], 1);
         mbar_fence_init();
     }
     __syncthreads();
     if (threadIdx.x == 0 && ok) {
         tma_prefetch_desc(tmW);
-        for (int c = 0; c < n_chunks && c < SK_STAGES; ++c) {
+        for (int c = 0; c < n_chunks && c < SK_STAGES; ++c, ++armed) {
             mbar_expect_tx(&full[c], HALF_BYTES);
             tma_load_2d(smem + c * HALF_BYTES, tmW, col0, k_base + c * SK_KBOX, &full[c]);
         }
@@ -336,10 +352,7 @@ kv_append_small_kernel(const __grid_constant__ CUtensorMap tmWk, const __grid_co
         }
         __syncthreads();
         const int stage = c % SK_STAGES;
-        if (ok && !mbar_wait(&full[stage], (uint32_t)(c / SK_STAGES) & 1u)) {
-            atomicExch(&g_kv_append_status, kStatusTimeout);
-            ok = false;
-        }
+        if (ok && !wait_or_abort(&full[stage], (uint32_t)(c / SK_STAGES) & 1u, ab, kWaitRingFull)) ok = false;
         if (ok) {
             const uint32_t wbase = smem_u32(smem + stage * HALF_BYTES);
             const int k_l = ((lane >> 3) & 1) * 8 + (lane & 7);      // ldmatrix row inside a 16-k step
@@ -364,6 +377,7 @@ kv_append_small_kernel(const __grid_constant__ CUtensorMap tmWk, const __grid_co
             fence_proxy_async_smem();
             mbar_expect_tx(&full[stage], HALF_BYTES);
             tma_load_2d(smem + stage * HALF_BYTES, tmW, col0, k_base + (c + SK_STAGES) * SK_KBOX, &full[stage]);
+            ++armed;
         }
         v0 = nv0;
         v1 = nv1;
@@ -438,6 +452,10 @@ kv_append_small_kernel(const __grid_constant__ CUtensorMap tmWk, const __grid_co
             }
         }
     }
+    // every copy thread 0 started must have landed before the CTA may end (at once unless a wait gave up)
+    if (threadIdx.x == 0)
+        for (int k = armed > SK_STAGES ? armed - SK_STAGES : 0; k < armed; ++k)
+            if (!drain_wait(&full[k % SK_STAGES], (uint32_t)(k / SK_STAGES) & 1u, ab)) break;
     cluster_sync_all();                                     // nobody leaves while its memory is being read
 }
 

@@ -19,11 +19,27 @@ int32_t validate_shape(const yoco_xattn_shape& s, int32_t mode) {
     return YOCO_OK;
 }
 
+int32_t validate_layout(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const int32_t* kv_len_host) {
+    for (int i = 0; i < s.B; ++i) {
+        const int64_t n = kv_len_host ? kv_len_host[i] : s.max_kv_len;
+        if (n < 0) return YOCO_ERR_INVALID_ARG;
+        const int64_t head_rows = s.kv_head_stride ? s.kv_head_stride / s.d : n;
+        if (head_rows < n) return YOCO_ERR_INVALID_ARG;
+        if (cu_kv_host) {
+            if (cu_kv_host[i] < 0 || cu_kv_host[i + 1] < cu_kv_host[i]) return YOCO_ERR_INVALID_ARG;
+            // sequence i occupies Hkv * head_rows rows from token offset cu[i]: the next one may not start inside it
+            if (n > 0 && (int64_t)cu_kv_host[i + 1] - cu_kv_host[i] < head_rows) return YOCO_ERR_INVALID_ARG;
+        }
+    }
+    return YOCO_OK;
+}
+
 int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const int32_t* kv_len_host,
                   int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items) {
     int32_t rc = validate_shape(s, mode);
     if (rc != YOCO_OK) return rc;
     if (sm_count <= 0) return YOCO_ERR_INVALID_ARG;
+    if ((rc = validate_layout(s, cu_kv_host, kv_len_host)) != YOCO_OK) return rc;
 
     const int G = s.Hq / s.Hkv;
     const int rows_per_stream = G * s.T;
@@ -39,13 +55,8 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     int64_t extent = 0;
     for (int i = 0; i < s.B; ++i) {
         len[i] = kv_len_host ? kv_len_host[i] : s.max_kv_len;
-        if (len[i] < 0) return YOCO_ERR_INVALID_ARG;
-        if (cu_kv_host) {
-            if (cu_kv_host[i] < 0 || cu_kv_host[i + 1] < cu_kv_host[i]) return YOCO_ERR_INVALID_ARG;
-            tok_off[i] = cu_kv_host[i];
-        }
+        if (cu_kv_host) tok_off[i] = cu_kv_host[i];
         const int64_t head_rows = s.kv_head_stride ? s.kv_head_stride / s.d : len[i];
-        if (head_rows < len[i]) return YOCO_ERR_INVALID_ARG;
         if (!cu_kv_host) tok_off[i + 1] = tok_off[i] + head_rows;
         if (len[i] > 0)
             extent = std::max(extent, tok_off[i] * s.Hkv + (int64_t)(s.Hkv - 1) * head_rows + len[i]);

@@ -90,5 +90,7 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
                   int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items = kMaxSubItems);
 
 int32_t validate_shape(const yoco_xattn_shape& s, int32_t mode);
+// Lengths, head stride and token offsets must describe sequences that do not overlap (pure host).
+int32_t validate_layout(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const int32_t* kv_len_host);
 
 }  // namespace yoco

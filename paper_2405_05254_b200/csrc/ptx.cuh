@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 
+#include "kernels.h"
+
 namespace yoco {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -37,21 +39,68 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after about two seconds, so a lost signal ends the kernel with an
-// error status instead of hanging the GPU.
+// ---- bounded waits ---------------------------------------------------------------------------
+// No wait in this library is open-ended: a signal that never comes ends the kernel with a status
+// word instead of hanging the GPU.  The limit is wall-clock time read from %globaltimer, taken as a
+// SIGNED difference (a backward step of that counter then reads as "no time has passed", never as
+// an instant expiry), backed by a cap on the number of polls in case the timer does not advance.
 __device__ __forceinline__ uint64_t global_timer_ns() {
     uint64_t t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+constexpr int64_t kWaitLimitNs = 2000000000ll;    // a lost signal: give up after about two seconds
+constexpr int64_t kDrainLimitNs = 200000000ll;    // copies already in flight when a CTA wants to leave
+constexpr uint32_t kWaitMaxPolls = 1u << 28;      // each poll takes >= ~10 ns: a few seconds at least
+
+struct Abort {
+    volatile int* flag;      // shared memory: some thread of this CTA has given up
+    int32_t* status;         // global status word
+    int64_t limit_ns;        // how long a wait may last
+};
+__device__ __forceinline__ int32_t linear_cta() {
+    return (int32_t)(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z));
+}
+__device__ __forceinline__ void report_give_up(const Abort& ab, int32_t wait_class) {
+    atomicCAS(ab.status, 0, status_word(wait_class, linear_cta()));
+    *ab.flag = 1;
+}
+// Waits for the phase with the given parity; false when the limit ran out (then the status word
+// and the CTA's flag are set) or when another thread of the CTA has already given up.
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, const Abort& ab, int32_t wait_class) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 0 && global_timer_ns() - t0 > kWaitLimitNs) return false;
+        if ((i & 63u) == 0) {
+            if (*ab.flag) return false;
+            if ((int64_t)(global_timer_ns() - t0) > ab.limit_ns || i >= kWaitMaxPolls) {
+                report_give_up(ab, wait_class);
+                return false;
+            }
+        }
     }
+}
+// Used on the way out: waits (for a short, fixed time) for something this thread started itself -- a
+// bulk copy it armed, a tensor-core product it issued -- whatever the state of the CTA's flag.  A
+// CTA must not exit while a copy can still land in its shared memory or arrive on its barriers: the
+// memory belongs to the next CTA by then.
+__device__ __forceinline__ bool drain_wait(uint64_t* bar, uint32_t parity, const Abort& ab) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 0 && ((int64_t)(global_timer_ns() - t0) > kDrainLimitNs || i >= kWaitMaxPolls)) {
+            report_give_up(ab, kWaitDrain);
+            return false;
+        }
+    }
+}
+// All lanes of a warp wait on the same barrier; the result is made warp-uniform so that the
+// lanes never diverge around the __syncwarp / elected arrives that follow.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, const Abort& ab, int32_t wait_class) {
+    const bool r = wait_or_abort(bar, parity, ab, wait_class);
+    return __all_sync(0xffffffffu, r);
 }
 
 // ---- TMA ------------------------------------------------------------------------------
@@ -101,6 +150,20 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// Barrier over `threads` threads that also ORs a predicate: every participant gets the same answer.
+__device__ __forceinline__ bool named_barrier_or(int id, int threads, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "r"(id), "r"(threads)
+        : "memory");
+    return r != 0;
 }
 
 }  // namespace yoco

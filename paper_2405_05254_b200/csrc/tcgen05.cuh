@@ -1,5 +1,4 @@
-// Inline-PTX wrappers for the fifth-generation tensor cores (tcgen05) and tensor memory (TMEM),
-// plus the bounded-wait helpers shared by the tensor-core kernels.
+// Inline-PTX wrappers for the fifth-generation tensor cores (tcgen05) and tensor memory (TMEM).
 #pragma once
 
 #include "kernels.h"
@@ -181,33 +180,5 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
            ((uint32_t)(128 >> 4) << 24);
 }
-
-struct Abort {
-    volatile int* flag;
-    int32_t* status;
-};
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, const Abort& ab) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
-    for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 63u) == 0) {
-            if (*ab.flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
-                atomicExch(ab.status, kStatusTimeout);
-                *ab.flag = 1;
-                return false;
-            }
-        }
-    }
-}
-
-// All lanes of a warp wait on the same barrier; the result is made warp-uniform so that the
-// lanes never diverge around the __syncwarp / elected arrives that follow.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, const Abort& ab) {
-    const bool r = wait_or_abort(bar, parity, ab);
-    return __all_sync(0xffffffffu, r);
-}
-
 
 }  // namespace yoco

@@ -1,10 +1,12 @@
 """Parity at the full benchmark sizes, in the launch configuration bench.py times.
 
-The 1M-token and ragged decode configs are checked against the full oracle (one or two layers
-completely, the other layers on sampled heads); the 512 x 262K chunk config on sampled query
-rows over the full key range (t = 0, T-1, the 128-row tile edges), each computed one by one by
-the oracle; and the split/merge indexing at 1M tokens bit-exactly with one-hot scores planted on
-every segment boundary of the plan.
+The 1M-token (all 13 layers) and ragged decode configs are checked against the full oracle; the
+512 x 262K chunk config on at least 64 sampled (sequence, position) query rows, all heads each, over
+the full key range (t = 0, T-1, the 128-row tile edges), each computed one by one by the oracle; the
+split/merge indexing at 1M tokens bit-exactly with one-hot scores planted on every segment boundary
+of the plan; and the side measurements of bench.py at their sizes: the 8-bit cache at 1M keys, a few
+new rows per head (the one-tile tensor-core kernel) over a long cache, and one shard of an 8-way
+key-range split read through a head-stride view of the resident cache.
 """
 import math
 
@@ -19,6 +21,7 @@ pytestmark = pytest.mark.gpu
 
 
 def test_one_million_token_decode_thirteen_layers():
+    """Every one of the 13 layer calls over the 1M-token cache, every head, against the full oracle."""
     w = si.workload("1m")
     K, V = w.make_k(), w.make_v()
     r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, w.T, w.kv_len, K, V)
@@ -26,17 +29,9 @@ def test_one_million_token_decode_thirteen_layers():
     for layer in range(w.layers):
         Q = w.make_q(layer)
         o, lse, _ = r.run(Q)
-        if layer in (0, w.layers - 1):
-            o_ref, lse_ref = oracle.xattn(Q, K, V, w.cu, w.kv_len, **kw)
-            assert_close(o, o_ref, f"1m layer {layer}")
-            assert_lse_close(lse, lse_ref, f"1m layer {layer}")
-        else:   # two query heads of different KV heads, chosen by layer
-            heads = [(3 * layer) % w.Hq, (3 * layer + 17) % w.Hq]
-            rows = np.array([(0, h, 0) for h in heads], dtype=np.int32)
-            o_ref, lse_ref = oracle.xattn_rows(Q, K, V, w.cu, w.kv_len, rows, **kw)
-            got = np.stack([o[0, h, 0] for h in heads])
-            assert_close(got, o_ref, f"1m layer {layer} heads {heads}")
-            assert_lse_close(np.array([lse[0, h, 0] for h in heads]), lse_ref, f"1m layer {layer}")
+        o_ref, lse_ref = oracle.xattn(Q, K, V, w.cu, w.kv_len, **kw)
+        assert_close(o, o_ref, f"1m layer {layer}")
+        assert_lse_close(lse, lse_ref, f"1m layer {layer}")
 
 
 def test_ragged_batch_full_size():
@@ -56,7 +51,13 @@ def test_chunk_config_sampled_rows_over_the_full_key_range():
     K, V, Q = w.make_k(), w.make_v(), w.make_q(0)
     r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, w.T, w.kv_len, K, V)
     o, lse, _ = r.run(Q, "chunk")
-    ts = [0, 1, 127, 128, 255, 256, 383, 384, 510, 511, 77, 300]
+    # 36 positions per sequence = 72 (b, t) rows, every head of each: the first and last row, both sides of
+    # every 128-row tile edge of the (head in group, t) row order, and seeded draws in between
+    edges = [0, 1, 127, 128, 255, 256, 383, 384, 510, 511]
+    rng = np.random.default_rng(505)
+    inner = [t for t in range(2, 510) if t not in edges]
+    ts = sorted(set(edges) | set(int(t) for t in rng.choice(inner, size=26, replace=False)))
+    assert len(ts) == 36
     rows = np.array([(b, h, t) for b in range(w.B) for t in ts for h in range(w.Hq)], dtype=np.int32)
     o_ref, lse_ref = oracle.xattn_rows(Q, K, V, w.cu, w.kv_len, rows, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T)
     got = np.stack([o[b, h, t] for b, h, t in rows])
@@ -98,3 +99,86 @@ def test_split_merge_indexing_is_bit_exact_at_one_million_tokens():
             np.testing.assert_array_equal(o[0, h, 0], Vf[h // G, picks[h // G]].astype(np.float64),
                                           err_msg=f"round {k} head {h} key {picks[h // G]}")
         assert np.allclose(lse, 16 * 8 * d / math.sqrt(d), rtol=1e-6)
+
+
+def test_fp8_cache_decode_at_one_million_tokens():
+    """The 8-bit-cache decode at the size bench.py times it, on a really quantised cache (the 1M K/V
+    draws rounded to E4M3 with per-head amax / 448 scales), every head, against the oracle reading the
+    same bytes."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    from helpers import bf16_dev_to_f64, to_dev_bf16
+    w = si.workload("1m")
+    K8, V8, ks, vs = w.make_kv_fp8()
+    Q = w.make_q(0)
+    shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(w.kv_len.max()))
+    n = w.B * w.Hq * w.T
+    ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_DECODE), dtype=torch.uint8, device="cuda")
+    O = torch.empty(n * w.d, dtype=torch.bfloat16, device="cuda")
+    L = torch.empty(n, dtype=torch.float32, device="cuda")
+    bd.yoco_xattn_decode_fp8(shape, to_dev_bf16(Q.reshape(-1)), torch.from_numpy(K8).cuda(), torch.from_numpy(V8).cuda(),
+                             ks, vs, w.cu, w.kv_len, O, L, ws)
+    assert bd.yoco_xattn_status(ws) == 0
+    o_ref, lse_ref = oracle.xattn_fp8(Q, K8, V8, ks, vs, w.cu, w.kv_len, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T)
+    assert_close(bf16_dev_to_f64(O).reshape(o_ref.shape), o_ref, "fp8 cache, 1M keys")
+    assert_lse_close(L.cpu().numpy().reshape(lse_ref.shape), lse_ref, "fp8 cache, 1M keys")
+
+
+@pytest.mark.parametrize("T", [8, 32])
+def test_few_new_rows_over_a_long_cache(T):
+    """T = 8 and 32 new positions per sequence (32 and 128 rows per KV head: the one-tile tensor-core
+    kernel, split over the key range and merged) after 131,072 cached keys; every head of sampled
+    positions, first and last included, against the oracle row by row."""
+    base = si.workload("128k")
+    w = si.Workload("few_rows", B=1, Hq=base.Hq, Hkv=base.Hkv, d=base.d, T=T, layers=1, seed=base.seed,
+                    kv_len=[131072 + T])
+    K, V, Q = w.make_k(), w.make_v(), w.make_q(0)
+    r = GpuRunner(w.B, w.Hq, w.Hkv, w.d, w.T, w.kv_len, K, V)
+    o, lse, _ = r.run(Q, "chunk")
+    ts = sorted({0, 1, T // 2, T - 2, T - 1} | {3, 5} & set(range(T)))
+    rows = np.array([(0, h, t) for t in ts for h in range(w.Hq)], dtype=np.int32)
+    o_ref, lse_ref = oracle.xattn_rows(Q, K, V, w.cu, w.kv_len, rows, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T)
+    got = np.stack([o[b, h, t] for b, h, t in rows])
+    assert_close(got, o_ref, f"T={T} over 131072 keys")
+    assert_lse_close(np.array([lse[b, h, t] for b, h, t in rows]), lse_ref, f"T={T} over 131072 keys")
+    assert np.isfinite(o).all() and np.isfinite(lse).all()
+
+
+def test_one_shard_of_an_eight_way_key_split_read_through_a_head_stride_view():
+    """What bench.py's key-range-shard measurement runs: the 1M cache stays where it is and a shard is
+    the view (pointer offset to its first key, head stride of the whole cache, 131,072 keys per head).
+    The partial result of the first, a middle and the last shard against the oracle over the same view,
+    and the merge of all eight against the oracle over the whole cache."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd, shard
+    from helpers import bf16_dev_to_f64, to_dev_bf16
+    w = si.workload("1m")
+    K, V, Q = w.make_k(), w.make_v(), w.make_q(0)
+    N, shards = int(w.kv_len[0]), 8
+    off, cnt = shard.key_range_shards([N], shards)
+    Kd, Vd, Qd = to_dev_bf16(K), to_dev_bf16(V), to_dev_bf16(Q.reshape(-1))
+    rows = w.B * w.Hq
+    all_o = torch.zeros((shards, rows, w.d), dtype=torch.float32, device="cuda")
+    all_l = torch.zeros((shards, rows), dtype=torch.float32, device="cuda")
+    cu = np.array([0, N], dtype=np.int32)
+    for r in range(shards):
+        n_local = int(cnt[r, 0])
+        assert n_local == 131072
+        lens = np.array([n_local], dtype=np.int32)
+        shape = bd.make_shape(1, w.Hq, w.Hkv, w.d, 1, kv_head_stride=N * w.d, max_kv_len=n_local)
+        ws = torch.empty(bd.yoco_xattn_workspace_size(shape, lens, bd.MODE_DECODE), dtype=torch.uint8, device="cuda")
+        o = int(off[r, 0]) * w.d
+        bd.yoco_xattn_decode_partial(shape, Qd, Kd[o:], Vd[o:], cu, lens, all_o[r], all_l[r], ws)
+        assert bd.yoco_xattn_status(ws) == 0
+        if r in (0, 3, 7):
+            po, pl = oracle.xattn(Q, K[o:], V[o:], cu, lens, B=1, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=1, kv_head_stride=N * w.d)
+            got = all_o[r].cpu().numpy().astype(np.float64).reshape(po.shape)
+            assert_close(got, po, f"shard {r}")
+            assert_lse_close(all_l[r].cpu().numpy().reshape(pl.shape), pl, f"shard {r}")
+    O = torch.empty(rows * w.d, dtype=torch.bfloat16, device="cuda")
+    L = torch.empty(rows, dtype=torch.float32, device="cuda")
+    bd.yoco_xattn_combine_gathered(all_o, all_l, O, L)
+    torch.cuda.synchronize()
+    o_ref, lse_ref = oracle.xattn(Q, K, V, w.cu, w.kv_len, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T)
+    assert_close(bf16_dev_to_f64(O).reshape(o_ref.shape), o_ref, "eight shards merged")
+    assert_lse_close(L.cpu().numpy().reshape(lse_ref.shape), lse_ref, "eight shards merged")

@@ -65,6 +65,47 @@ def test_identical_keys_give_prefix_means_under_causal_mask():
             assert LSE[0, h, t] == pytest.approx(s + math.log(n_vis), rel=1e-13)
 
 
+def test_selected_rows_of_a_ragged_batch_give_prefix_means_of_their_own_sequence():
+    """The row-sampling entry (what the full-size chunk checks and the timed CPU baseline call) on a
+    ragged batch of three sequences with a head stride, rows taken from every sequence in scrambled
+    order.  Keys are identical inside a (sequence, KV head), so every answer is a closed form: the mean
+    of that sequence's, that head's values over keys [0, N_i - T + t], and LSE = score + log(count).
+    A slip in the (b, h, t) indexing, in the per-sequence offset or in the GQA head would pick another
+    sequence's or head's values, which differ."""
+    rng = np.random.default_rng(11)
+    B, Hq, Hkv, d, T = 3, 6, 2, 4, 4
+    lens = np.array([9, 4, 14], dtype=np.int32)
+    cap = 16                                                   # rows per head: spare capacity behind every head
+    cu = np.array([0, cap, 2 * cap, 3 * cap], dtype=np.int32)
+    Q = rnd(rng, B, Hq, T, d)
+    K = rnd(rng, B * Hkv * cap * d)                            # slack rows hold noise
+    V = rnd(rng, B * Hkv * cap * d)
+    Kv, Vv = K.reshape(B, Hkv, cap, d), V.reshape(B, Hkv, cap, d)
+    krows = rnd(rng, B, Hkv, d)
+    for b in range(B):
+        for c in range(Hkv):
+            Kv[b, c, :lens[b]] = krows[b, c]
+    rows = [(b, h, t) for b in range(B) for h in range(Hq) for t in range(T)]
+    rng.shuffle(rows)
+    rows = np.array(rows, dtype=np.int32)
+    O, LSE = oracle.xattn_rows(Q, K, V, cu, lens, rows, B=B, Hq=Hq, Hkv=Hkv, d=d, T=T, kv_head_stride=cap * d)
+    Vf, Qf, Kf = b2f(Vv).astype(np.float64), b2f(Q).astype(np.float64), b2f(krows).astype(np.float64)
+    seen = set()
+    for k, (b, h, t) in enumerate(rows):
+        c = h // (Hq // Hkv)
+        n_vis = int(lens[b]) - T + t + 1
+        seen.add(b)
+        np.testing.assert_allclose(O[k], Vf[b, c, :n_vis].mean(axis=0), rtol=1e-14, atol=1e-15)
+        s_ = float(Qf[b, h, t] @ Kf[b, c]) / math.sqrt(d)
+        assert LSE[k] == pytest.approx(s_ + math.log(n_vis), rel=1e-13)
+    assert seen == {0, 1, 2}
+    # and it is the same routine as the full evaluation, row for row
+    Of, Lf = oracle.xattn(Q, K, V, cu, lens, B=B, Hq=Hq, Hkv=Hkv, d=d, T=T, kv_head_stride=cap * d)
+    for k, (b, h, t) in enumerate(rows):
+        np.testing.assert_array_equal(O[k], Of[b, h, t])
+        assert LSE[k] == Lf[b, h, t]
+
+
 def test_zero_query_gives_plain_mean_and_log_n():
     rng = np.random.default_rng(2)
     N, d = 37, 16

@@ -292,6 +292,67 @@ def test_new_entry_points_validate_arguments_before_touching_cuda():
     assert L.yoco_xattn_combine_gathered(4, 0, 128, None, None, None, None, None) == bd.ERR_INVALID_ARG
 
 
+def test_overlapping_offsets_and_a_stride_too_short_are_rejected_on_the_host():
+    """Sequence i occupies Hkv * head_rows rows from token offset cu[i]; offsets that let the next
+    sequence start inside it would make attention read a neighbour's keys and the cache write land in
+    a neighbour's heads.  Both entry points must say so before any CUDA call."""
+    L = bd.lib()
+    p = ctypes.c_void_p
+    lens = np.array([100, 50], dtype=np.int32)
+    pl = p(lens.ctypes.data)
+
+    def decode(shape, cu):
+        cu = np.asarray(cu, dtype=np.int32)
+        return L.yoco_xattn_decode(ctypes.byref(shape), p(4096), p(4096), p(4096), p(cu.ctypes.data), pl, p(4096),
+                                   None, p(4096), 1 << 20, None)
+
+    tight = bd.make_shape(2, 8, 8, 128, 1, max_kv_len=100)
+    assert decode(tight, [0, 99, 150]) == bd.ERR_INVALID_ARG          # second sequence starts inside the first
+    assert decode(tight, [0, 100, 149]) == bd.ERR_INVALID_ARG         # the last one does not fit its own range
+    assert decode(tight, [0, 120, 100]) == bd.ERR_INVALID_ARG         # not monotone
+    strided = bd.make_shape(2, 8, 8, 128, 1, kv_head_stride=128 * 128, max_kv_len=100)
+    assert decode(strided, [0, 100, 228]) == bd.ERR_INVALID_ARG       # capacity 128 per head, offsets say 100
+    short = bd.make_shape(2, 8, 8, 128, 1, kv_head_stride=64 * 128, max_kv_len=100)
+    assert decode(short, [0, 128, 256]) == bd.ERR_INVALID_ARG         # stride shorter than the first sequence
+    # the same offsets are fine once they leave room (no GPU here: the call then fails later, at the device query)
+    assert decode(tight, [0, 100, 150]) != bd.ERR_INVALID_ARG
+    assert decode(strided, [0, 128, 256]) != bd.ERR_INVALID_ARG
+
+    ash = bd.KvAppendShape(2, 8, 128, 1, 4096, 1e-6, 0)
+
+    def append(shape, cu):
+        cu = np.asarray(cu, dtype=np.int32)
+        return L.yoco_kv_append(ctypes.byref(shape), p(16), p(16), p(16), p(16), p(16), p(cu.ctypes.data), pl, None)
+
+    assert append(ash, [0, 99, 150]) == bd.ERR_INVALID_ARG
+    assert append(ash, [0, 100, 149]) == bd.ERR_INVALID_ARG
+    assert append(bd.KvAppendShape(2, 8, 128, 1, 4096, 1e-6, 128 * 128), [0, 100, 228]) == bd.ERR_INVALID_ARG
+    assert append(ash, [0, 100, 150]) != bd.ERR_INVALID_ARG
+
+
+def test_status_word_names_the_wait_and_the_cta():
+    """0 is ok; otherwise the low byte is the kind of wait that ran out and the rest 1 + the CTA."""
+    assert bd.yoco_xattn_decode_status_word(0) == (bd.OK, 0, -1)
+    for wc in (bd.WAIT_ITEM_QUEUE, bd.WAIT_RING_FULL, bd.WAIT_RING_EMPTY, bd.WAIT_TENSOR, bd.WAIT_DRAIN,
+               bd.WAIT_MISALIGNED):
+        for cta in (0, 1, 147, 295, 70000):
+            word = wc | ((cta + 1) << 8)
+            assert bd.yoco_xattn_decode_status_word(word) == (bd.ERR_TIMEOUT, wc, cta)
+    # either output may be omitted
+    assert bd.lib().yoco_xattn_decode_status_word(2 | (5 << 8), None, None) == bd.ERR_TIMEOUT
+    # the header's names carry the same numbers
+    hdr = open(os.path.join(ROOT, "include", "yoco_xattn.h")).read()
+    for name, val in (("ITEM_QUEUE", 1), ("RING_FULL", 2), ("RING_EMPTY", 3), ("TENSOR", 4), ("DRAIN", 5),
+                      ("MISALIGNED", 6)):
+        assert re.search(rf"#define YOCO_WAIT_{name}\s+{val}\b", hdr), name
+    p = ctypes.c_void_p
+    shape = bd.make_shape(1, 8, 8, 128, 1, max_kv_len=64)
+    f = bd.lib().yoco_xattn_selftest_wait_expiry
+    for bad_limit in (0, -5, 1001):
+        assert f(ctypes.byref(shape), p(4096), p(4096), p(4096), None, None, p(4096), p(4096), 1 << 20, bad_limit,
+                 None) == bd.ERR_INVALID_ARG
+
+
 def test_public_header_is_plain_c_and_cxx(tmp_path):
     """The boundary is a C ABI: the header must compile on its own as C99 and as C++11, warnings
     as errors, and a C program must be able to link the planner (a pure host call) from the library."""
