@@ -4,19 +4,20 @@
 // that share every K/V tile brought into shared memory, and walks a contiguous range of 128-key
 // tiles.  Three warpgroups (384 threads):
 //   warpgroup 0   warp 0 = TMA producer (both Q tiles once per segment; K through a three-deep and
-//                 V through a two-deep ring), warps 1 and 2 = issuers of the score products of row
-//                 tiles 0 and 1, warp 3 = issuer of the PV products; gives most of its registers away
+//                 V through a two-deep ring), warps 1 and 2 = issuers of all tensor-core products of
+//                 row tiles 0 and 1; gives most of its registers away
 //   warpgroup 1   softmax of row tile 0 (thread = query row)
 //   warpgroup 2   softmax of row tile 1
 // Every 128-key tile is processed as two 64-key half steps.  Tensor memory (512 columns):
 //   S_0^0 S_0^1 | S_1^0 S_1^1 | O_0 | O_1      (64 fp32 columns per S buffer, 128 per O)
 // S_r^h receives the scores of row tile r against half h of the key tile, so the scores of the
-// next half step are already being computed while a warpgroup works on the current one: the
-// softmax never waits for the tensor pipe and the tensor pipe never waits for one particular
-// softmax.  A softmax thread reads its S row, keeps the running max / sum, and writes P (bf16,
-// two per 32-bit column) over the first 32 columns of the same S buffer; O_r += P_r V then takes
-// P straight from tensor memory as the A operand, so P never touches shared memory.
-// O in tensor memory is rescaled only when a row max outgrew the reference by more than 2^8.
+// next half step are already being computed while a warpgroup works on the current one.  A softmax
+// thread reads its S row, keeps the running max / sum, and writes P (bf16, two per 32-bit column)
+// over the first 32 columns of the same S buffer; O_r += P_r V then takes P straight from tensor
+// memory as the A operand, so P never touches shared memory.  The issuer of a row tile puts the
+// next score product of a buffer right behind the P V product that reads it: the tensor pipe runs
+// the products of one thread in the order issued, so the buffer needs no barrier round trip between
+// the two.  O in tensor memory is rescaled only when a row max outgrew the reference by more than 2^8.
 // Every wait is bounded and reports through the status word.
 #include "kernels.h"
 #include "ptx.cuh"
@@ -61,15 +62,6 @@ __host__ __device__ constexpr bool poly_pair(int j) {
     return ((j + 1) * kPolyPairs) / 16 != (j * kPolyPairs) / 16;
 }
 
-// position in the CTA's flat sequence of (segment, key tile) pairs
-struct TileCursor {
-    int si, k0, k_end, h;
-    uint32_t tp;                 // parity of the key tile number since the start of the CTA
-    uint32_t kb, kph, vb, vph;   // ring stage and phase parity of the K and V tiles
-    bool first_tile;             // first key tile of its segment
-    bool valid;
-};
-
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -113,7 +105,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         for (int b = 0; b < VS; ++b) {
             mbar_init(&v_full[b], 1);
-            mbar_init(&v_empty[b], 1);
+            mbar_init(&v_empty[b], 2);            // released by both issuers
         }
         for (int r = 0; r < 2; ++r) {
             for (int h = 0; h < 2; ++h) {
@@ -145,8 +137,8 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             bool ok = true;
             for (int si = seg_lo; si < seg_hi && ok; ++si) {
                 const DevSegment seg = p.segments[si];
-                const uint32_t sidx = si - seg_lo;
-                if (!(ok = wait_or_abort(q_empty, (sidx & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
+                if (seg.k_end <= seg.k_begin) continue;
+                if (!(ok = wait_or_abort(q_empty, (q_armed & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
                 ++q_armed;
                 mbar_expect_tx(q_full, 2 * C::TILE_BYTES);
                 for (int r = 0; r < 2; ++r)
@@ -178,124 +170,86 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 drained = drain_wait(&k_full[k % KS], (k / KS) & 1u, ab);
             for (uint32_t k = v_armed > (uint32_t)VS ? v_armed - VS : 0; drained && k < v_armed; ++k)
                 drained = drain_wait(&v_full[k % VS], (k / VS) & 1u, ab);
-        } else if (warp >= 1 && aligned_ok) {
+        } else if ((warp == 1 || warp == 2) && aligned_ok) {
             // =================================== MMA issuers =================================
-            // Issuing a tensor-core instruction costs a single warp tens of cycles (a chain of
-            // dependent scalar instructions), about as long as the instruction runs, so the work is
-            // spread over three warps: warps 1 and 2 issue S_r = Q_r K^T for row tiles 0 and 1,
-            // warp 3 issues O_r += P_r V for both.  Each whole warp walks the schedule (addresses
-            // and descriptors stay warp-uniform) and one elected lane issues.  Instructions of
-            // different threads are ordered only through the barriers: a score product waits for
-            // the product that last read its buffer (pv_done), a PV product for its P (p_full).
+            // Warp 1 + r issues every product of row tile r, half step by half step:
+            //   O_r += P_r^h V^h  (key tile j)   and right behind it   S_r^h = Q_r K^h^T  (key tile j + 1).
+            // The score product overwrites the buffer P_r^h sits in; the tensor pipe runs the products
+            // of one thread in the order issued, so no wait (and no hand-over between two warps) is
+            // needed between the two, which takes one barrier round trip out of the cycle
+            // scores -> softmax -> P V -> next scores of every buffer.  The whole warp walks the
+            // schedule (addresses and descriptors stay warp-uniform) and one elected lane issues:
+            // issued from a diverged lane the same instructions cost several times as much.
+            const int r = warp - 1;
             constexpr uint32_t idesc_qk = make_idesc(BH, false);
             constexpr uint32_t idesc_pv = make_idesc(D, true);
             const uint32_t sbase = smem_u32(smem);
-            TileCursor c;
-            c.si = seg_lo;
-            c.h = 0;
-            c.tp = 0;
-            c.kb = c.kph = c.vb = c.vph = 0;
-            c.first_tile = false;
-            auto cur_load = [&]() {
-                c.valid = c.si < seg_hi;
-                if (c.valid) {
-                    c.k0 = p.segments[c.si].k_begin;
-                    c.k_end = p.segments[c.si].k_end;
-                    c.first_tile = true;
-                }
-            };
-            auto cur_next = [&]() {      // one half step forward
-                if (c.h == 0) {
-                    c.h = 1;
-                    return;
-                }
-                c.h = 0;
-                c.tp ^= 1u;
-                if (++c.kb == KS) {
-                    c.kb = 0;
-                    c.kph ^= 1u;
-                }
-                if (++c.vb == VS) {
-                    c.vb = 0;
-                    c.vph ^= 1u;
-                }
-                c.first_tile = false;
-                c.k0 += BN;
-                if (c.k0 >= c.k_end) {
-                    ++c.si;
-                    cur_load();
-                }
-            };
-            cur_load();
+            const uint32_t q_lo = desc_lo(sbase + C::OFF_Q + r * C::TILE_BYTES, 16);
+            const uint32_t tmem_o = tmem_base + 2 * BN + r * BN;
             bool ok = true;
-            uint32_t tiles_seen = 0;     // key tiles finished by this warp (phase 0 has no predecessor)
+            uint32_t it = 0, n_seg = 0;
 
-            if (warp < 3) {
-                const int r = warp - 1;
-                const uint32_t q_lo = desc_lo(sbase + C::OFF_Q + r * C::TILE_BYTES, 16);
-                uint32_t seg_par = 0;
-                while (ok && c.valid) {
-                    if (c.h == 0) {
-                        if (c.first_tile) {
-                            ok = warp_wait(q_full, seg_par, ab, kWaitRingFull);
-                            seg_par ^= 1u;
-                        }
-                        ok = ok && warp_wait(&k_full[c.kb], c.kph, ab, kWaitRingFull);
-                    }
-                    // the buffer S_r^h still holds the P of the previous key tile until its product ran
-                    if (ok && tiles_seen > 0) ok = warp_wait(&pv_done[r * 2 + c.h], c.tp ^ 1u, ab, kWaitTensor);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t k_lo = desc_lo(sbase + C::OFF_K + c.kb * C::TILE_BYTES + c.h * BH * 128, 16);
-                    const uint32_t d_tmem = tmem_base + r * BN + c.h * BH;
-                    if (elect_one()) {
+            // scores of half h of key tile `tile` (its K stage must have landed)
+            auto issue_scores = [&](uint32_t tile, int h, bool last_of_segment) {
+                const uint32_t kb = tile % KS;
+                tc_fence_after();
+                const uint32_t k_lo = desc_lo(sbase + C::OFF_K + kb * C::TILE_BYTES + h * BH * 128, 16);
+                if (elect_one()) {
 #pragma unroll
-                        for (int ks = 0; ks < KSTEPS_QK; ++ks) {
-                            const uint32_t off = ((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4;
-                            umma_ss(d_tmem, desc_from_lo(q_lo + off, 1024), desc_from_lo(k_lo + off, 1024), idesc_qk,
-                                    ks > 0 ? 1u : 0u);
-                        }
-                        umma_commit(&s_full[r * 2 + c.h]);
-                        if (c.h == 1) {
-                            umma_commit(&k_empty[c.kb]);
-                            if (c.k0 + BN >= c.k_end) umma_commit(q_empty);   // both Q tiles may be replaced
-                        }
+                    for (int ks = 0; ks < KSTEPS_QK; ++ks) {
+                        const uint32_t off = ((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4;
+                        umma_ss(tmem_base + r * BN + h * BH, desc_from_lo(q_lo + off, 1024),
+                                desc_from_lo(k_lo + off, 1024), idesc_qk, ks > 0 ? 1u : 0u);
                     }
-                    __syncwarp();
-                    if (c.h == 1) ++tiles_seen;
-                    cur_next();
+                    umma_commit(&s_full[r * 2 + h]);
+                    if (h == 1) {
+                        umma_commit(&k_empty[kb]);
+                        if (last_of_segment) umma_commit(q_empty);   // this row tile's Q may be replaced
+                    }
                 }
-            } else {
-                while (ok && c.valid) {
-                    if (c.h == 0) ok = warp_wait(&v_full[c.vb], c.vph, ab, kWaitRingFull);
-                    const uint32_t v_lo = desc_lo(sbase + C::OFF_V + c.vb * C::TILE_BYTES + c.h * BH * 128, BN * 128);
-                    const uint32_t first = (c.first_tile && c.h == 0) ? 0u : 1u;
+                __syncwarp();
+            };
+
+            for (int si = seg_lo; si < seg_hi && ok; ++si) {
+                const int n_tiles = (p.segments[si].k_end - p.segments[si].k_begin + BN - 1) / BN;
+                if (n_tiles <= 0) continue;
+                // both halves of the first key tile of the segment (its Q and K have to be there)
+                if (!(ok = warp_wait(q_full, n_seg & 1u, ab, kWaitRingFull))) break;
+                ++n_seg;
+                if (!(ok = warp_wait(&k_full[it % KS], (it / KS) & 1u, ab, kWaitRingFull))) break;
+                issue_scores(it, 0, n_tiles == 1);
+                issue_scores(it, 1, n_tiles == 1);
+                for (int t = 0; t < n_tiles && ok; ++t, ++it) {
+                    const uint32_t vb = it % VS;
+                    if (!(ok = warp_wait(&v_full[vb], (it / VS) & 1u, ab, kWaitRingFull))) break;
+                    const bool more = t + 1 < n_tiles;
+                    if (more && !(ok = warp_wait(&k_full[(it + 1) % KS], ((it + 1) / KS) & 1u, ab, kWaitRingFull))) break;
 #pragma unroll
-                    for (int r = 0; r < 2; ++r) {
-                        ok = ok && warp_wait(&p_full[r * 2 + c.h], c.tp, ab, kWaitTensor);
-                        if (!ok) break;
+                    for (int h = 0; h < 2; ++h) {
+                        if (!(ok = warp_wait(&p_full[r * 2 + h], it & 1u, ab, kWaitTensor))) break;
                         tc_fence_after();
-                        const uint32_t a_tmem = tmem_base + r * BN + c.h * BH;
+                        const uint32_t v_lo = desc_lo(sbase + C::OFF_V + vb * C::TILE_BYTES + h * BH * 128, BN * 128);
+                        const uint32_t a_tmem = tmem_base + r * BN + h * BH;
                         if (elect_one()) {
 #pragma unroll
                             for (int ks = 0; ks < KSTEPS_PV; ++ks)
-                                umma_ts(tmem_base + 2 * BN + r * BN, a_tmem + ks * 8,
+                                umma_ts(tmem_o, a_tmem + ks * 8,
                                         desc_from_lo(v_lo + ((uint32_t)(ks * 16 * 128) >> 4), 1024), idesc_pv,
-                                        ks == 0 ? first : 1u);
-                            umma_commit(&pv_done[r * 2 + c.h]);
-                            if (r == 1 && c.h == 1) umma_commit(&v_empty[c.vb]);
+                                        (t == 0 && h == 0 && ks == 0) ? 0u : 1u);
+                            umma_commit(&pv_done[r * 2 + h]);
+                            if (h == 1) umma_commit(&v_empty[vb]);
                         }
                         __syncwarp();
+                        if (more) issue_scores(it + 1, h, t + 2 == n_tiles);
                     }
-                    cur_next();
                 }
             }
             // Nothing this warp issued may still be running (or still owe an arrive on one of this CTA's
             // barriers) when tensor memory is released and the CTA ends: one more commit, which
             // completes after every earlier product and commit of the issuing lane, and a wait for it.
             if (elect_one()) {
-                umma_commit(&drain_bar[warp - 1]);
-                drain_wait(&drain_bar[warp - 1], 0u, ab);
+                umma_commit(&drain_bar[r]);
+                drain_wait(&drain_bar[r], 0u, ab);
             }
             __syncwarp();
         }
@@ -322,9 +276,23 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const int lo_max = p.window > 0 ? seg.n_kv - p.window : 0;
             float m_ref = -INFINITY, l = 0.f;
             const uint32_t seg_first_it = it, seg_first_u = 2 * it;
+            int pending = -1;                          // half step whose P is stored but not yet announced
+
+            // The P of a half step is announced (wait for the stores, fence, arrive) only after the
+            // scores of the next half step have been fetched: the stores then have had time to land
+            // and their latency is not paid in line.
+            auto announce = [&]() {
+                if (pending >= 0) {
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&p_full[r * 2 + pending]);
+                    pending = -1;
+                }
+            };
 
             for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
-#pragma unroll
+#pragma unroll 1
                 for (int h = 0; h < 2; ++h) {
                     if (!ok) continue;
                     const uint32_t u = 2 * it + h;             // half step number
@@ -336,9 +304,10 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     for (int c = 0; c < BH / 32; ++c)
                         tmem_ld32(tmem_s + h * BH + c * 32, *reinterpret_cast<float(*)[32]>(&s[c * 32]));
                     tmem_wait_ld();
+                    announce();                                // the previous half step's P
 
-                    const bool unmasked = kh + BH <= n_full && kh >= lo_max;
-                    if (!unmasked) {           // causal edge, sequence end or window start
+                    const bool masked = !(kh + BH <= n_full && kh >= lo_max);   // causal edge, sequence end or window start
+                    if (masked) {
 #pragma unroll
                         for (int j = 0; j < BH; ++j) s[j] = (kh + j < vis && kh + j >= lo) ? s[j] : -INFINITY;
                     }
@@ -348,102 +317,85 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     for (int j = 0; j < BH; j += 2) mx4[(j >> 1) & 3] = fmax3(mx4[(j >> 1) & 3], s[j], s[j + 1]);
                     const float mx = fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * p.scale_log2;
                     // lazy rescale: the reference max moves only when the row max outgrew it by 2^8
-                    float alpha = 1.f;
                     const bool grow = mx > m_ref + kRescaleThreshold || (m_ref == -INFINITY && mx > -INFINITY);
-                    if (grow) {
-                        alpha = ex2_approx(m_ref - mx);               // 0 when m_ref = -inf
-                        m_ref = mx;
-                        l *= alpha;
-                    }
-                    if (__any_sync(0xffffffffu, grow) && u > seg_first_u) {
-                        // O_r holds the sums of the earlier half steps of this segment: wait for
-                        // the product of the previous one (the other buffer; it belongs to this key
-                        // tile when h = 1, to the previous one when h = 0)
-                        if (!(ok = warp_wait(&pv_done[r * 2 + (h ^ 1)], (it ^ (h ^ 1)) & 1u, ab, kWaitTensor))) continue;
-                        tc_fence_after();
+                    if (__any_sync(0xffffffffu, grow)) {
+                        float alpha = 1.f;
+                        if (grow) {
+                            alpha = ex2_approx(m_ref - mx);               // 0 when m_ref = -inf
+                            m_ref = mx;
+                            l *= alpha;
+                        }
+                        if (u > seg_first_u) {
+                            // O_r holds the sums of the earlier half steps of this segment: wait for
+                            // the product of the previous one (the other buffer; it belongs to this key
+                            // tile when h = 1, to the previous one when h = 0)
+                            if (!(ok = warp_wait(&pv_done[r * 2 + (h ^ 1)], (it ^ (h ^ 1)) & 1u, ab, kWaitTensor))) continue;
+                            tc_fence_after();
+#pragma unroll 1
+                            for (int c = 0; c < D / 32; ++c) {
+                                float o[32];
+                                tmem_ld32(tmem_o + c * 32, o);
+                                tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < D / 32; ++c) {
-                            float o[32];
-                            tmem_ld32(tmem_o + c * 32, o);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) o[j] *= alpha;
-                            tmem_st32(tmem_o + c * 32, o);
+                                for (int j = 0; j < 32; ++j) o[j] *= alpha;
+                                tmem_st32(tmem_o + c * 32, o);
+                            }
                         }
                     }
                     const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
 
-                    // P = 2^(s * scale - m_ref), two elements per instruction where the hardware
-                    // allows.  On tiles without masked keys, kPolyPairs of every 16 pairs take their
-                    // exponential on the FMA pipe so that the special-function unit (16 results per
-                    // clock per SM) is not the only limit.
-                    const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negm2 = f2_pack(neg_m, neg_m);
-                    uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};            // packed partial row sums
-#pragma unroll
-                    for (int c = 0; c < BH / 32; ++c) {                // 32 keys -> 16 packed columns
-                        uint32_t pk[16];
-                        if (unmasked) {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                const uint64_t x2 = f2_fma(f2_pack(s[c * 32 + 2 * j], s[c * 32 + 2 * j + 1]), scale2, negm2);
-                                uint64_t e2;
-                                if (poly_pair(j)) {
-                                    e2 = f2_exp2_poly(x2);
-                                } else {
-                                    float x0, x1;
-                                    f2_unpack(x2, x0, x1);
-                                    e2 = f2_pack(ex2_approx(x0), ex2_approx(x1));
-                                }
-                                ls2[j & 3] = f2_add(ls2[j & 3], e2);
-                                float e0, e1;
-                                f2_unpack(e2, e0, e1);
-                                pk[j] = pack_bf16x2(e0, e1);
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                const uint64_t x2 = f2_fma(f2_pack(s[c * 32 + 2 * j], s[c * 32 + 2 * j + 1]), scale2, negm2);
-                                float x0, x1;
-                                f2_unpack(x2, x0, x1);
-                                const uint64_t e2 = f2_pack(ex2_approx(x0), ex2_approx(x1));
-                                ls2[j & 3] = f2_add(ls2[j & 3], e2);
-                                float e0, e1;
-                                f2_unpack(e2, e0, e1);
-                                pk[j] = pack_bf16x2(e0, e1);
-                            }
-                        }
-                        tmem_st16(tmem_s + h * BH + c * 16, pk);
-                    }
-                    {
-                        float a0, a1, b0, b1;
-                        f2_unpack(f2_add(ls2[0], ls2[1]), a0, a1);
-                        f2_unpack(f2_add(ls2[2], ls2[3]), b0, b1);
-                        l += (a0 + a1) + (b0 + b1);
-                    }
-                    tmem_wait_st();
-                    tc_fence_before();
-
-                    // keys past the end of the sequence: their V rows may hold anything; zero them
-                    // so that 0 * garbage cannot make NaN.  Both warpgroups write the same zeros in
+                    // keys past the end of the sequence: their V rows may hold anything; zero them so
+                    // that 0 * garbage cannot make NaN.  Both warpgroups write the same zeros in
                     // the first half step, each before it releases its own first product on this tile.
                     if (h == 0 && k0 + BN > seg.n_kv) {
                         const uint32_t vb = it % VS, vn = it / VS;
                         if (!(ok = warp_wait(&v_full[vb], vn & 1u, ab, kWaitRingFull))) continue;
                         if (k0 + row >= seg.n_kv) {
                             uint8_t* vrow = smem + C::OFF_V + vb * C::TILE_BYTES + row * 128;
-#pragma unroll
-                            for (int hh = 0; hh < HALVES; ++hh)
-#pragma unroll
-                                for (int q = 0; q < 8; ++q)
-                                    *reinterpret_cast<uint4*>(vrow + hh * HALF_BYTES + q * 16) =
-                                        make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll 1
+                            for (int q = 0; q < 8 * HALVES; ++q)
+                                *reinterpret_cast<uint4*>(vrow + (q >> 3) * HALF_BYTES + (q & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
                         }
                         fence_proxy_async_smem();                   // generic writes -> tensor core reads
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&p_full[r * 2 + h]);
+
+                    // P = 2^(s * scale - m_ref), two elements per instruction where the hardware
+                    // allows.  kPolyPairs of every 16 pairs take their exponential on the FMA pipe
+                    // so that the special-function unit (16 results per clock per SM) is not the
+                    // only limit; a masked score (-inf) comes out as exactly 0 on both routes.
+                    const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negm2 = f2_pack(neg_m, neg_m);
+                    uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};            // packed partial row sums
+#pragma unroll
+                    for (int c = 0; c < BH / 32; ++c) {                // 32 keys -> 16 packed columns
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const uint64_t x2 = f2_fma(f2_pack(s[c * 32 + 2 * j], s[c * 32 + 2 * j + 1]), scale2, negm2);
+                            uint64_t e2;
+                            if (poly_pair(j)) {
+                                e2 = f2_exp2_poly(x2);
+                            } else {
+                                float x0, x1;
+                                f2_unpack(x2, x0, x1);
+                                e2 = f2_pack(ex2_approx(x0), ex2_approx(x1));
+                            }
+                            ls2[j & 3] = f2_add(ls2[j & 3], e2);
+                            float e0, e1;
+                            f2_unpack(e2, e0, e1);
+                            pk[j] = pack_bf16x2(e0, e1);
+                        }
+                        tmem_st16(tmem_s + h * BH + c * 16, pk);
+                    }
+                    pending = h;
+                    {
+                        float a0, a1, b0, b1;
+                        f2_unpack(f2_add(ls2[0], ls2[1]), a0, a1);
+                        f2_unpack(f2_add(ls2[2], ls2[3]), b0, b1);
+                        l += (a0 + a1) + (b0 + b1);
+                    }
                 }
             }
+            announce();
 
             // ---- end of segment: O_r is complete once the last PV has finished ----
             // (the products of one row tile complete in order, so the last one covers all)

@@ -125,12 +125,12 @@ __device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
 // 2^x for a pair on the FMA pipe instead of the special-function unit: x = n + f with n the nearest
 // integer (magic-number rounding) and f in [-0.5, 0.5]; 2^f by a cubic fitted to 7.5e-5 relative
 // error (far below the bf16 rounding that follows); n is added to the exponent field.  x is
-// clamped to >= -125 so that the exponent stays in range: anything below comes out as ~2^-125,
-// which vanishes against a row sum >= 2^-8 (callers must not use this on masked scores, which
-// have to come out as exactly 0).
+// clamped to >= -125 so that the exponent stays in range, and anything at or below the clamp (a
+// masked score is -inf) comes out as exactly 0, like the special-function unit's result.
 __device__ __forceinline__ uint64_t f2_exp2_poly(uint64_t x2) {
     float x0, x1;
     f2_unpack(x2, x0, x1);
+    const bool z0 = !(x0 > -125.f), z1 = !(x1 > -125.f);
     x2 = f2_pack(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
     const uint64_t magic = f2_pack(12582912.f, 12582912.f), neg_magic = f2_pack(-12582912.f, -12582912.f);
     const uint64_t t2 = f2_add(x2, magic);                         // low mantissa bits = round(x)
@@ -145,7 +145,7 @@ __device__ __forceinline__ uint64_t f2_exp2_poly(uint64_t x2) {
     f2_unpack(t2, t0, t1);
     const float e0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
     const float e1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
-    return f2_pack(e0, e1);
+    return f2_pack(z0 ? 0.f : e0, z1 ? 0.f : e1);
 }
 __device__ __forceinline__ float fmax3(float a, float b, float c) {   // one three-input max
     float d;
