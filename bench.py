@@ -113,7 +113,8 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sel), "window": window}
 
 
-from paper_2405_05254_b200.ranks import dist_env, job_throughput_gbs, max_over_ranks, replica_seed  # noqa: E402
+from paper_2405_05254_b200.ranks import (dist_env, job_throughput_gbs, max_over_ranks, replica_seed,  # noqa: E402
+                                         sharded_throughput_gbs)
 
 
 # ------------------------------------------------------------------------------------------
@@ -514,6 +515,101 @@ def measure_other_configs(dev, peak_gbs):
     return out
 
 
+def shard_keys_line(w, world, steps, warmup, total_ms, clocks, exchange_bytes):
+    """The JSON line of the key-range-sharded mode (pure host: also what the CPU test of this mode checks)."""
+    calls = steps * w.layers
+    value = sharded_throughput_gbs(w.kv_bytes, calls, total_ms)
+    return {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic", "us_per_token_layer": total_ms * 1e3 / calls / w.B,
+        "mode": "shard-keys",
+        "config": {"workload": f"{w.name}: B={w.B} Hq={w.Hq} Hkv={w.Hkv} d={w.d} T={w.T} kv_len={int(w.kv_len.max())} "
+                               f"x {w.layers} cross-decoder layers, the keys of every sequence split over {world} GPUs",
+                   "kv_bytes_per_layer_call": w.kv_bytes, "layers_per_step": w.layers,
+                   "l2": "each rank's share of K+V per call is larger than L2" if w.kv_bytes / world > 4 * 126e6
+                         else "each rank's share fits in L2: back-to-back calls re-read it from there",
+                   "parallelism": f"key-range sharding x{world}: per layer call every rank runs the partial decode on "
+                                  "its keys, one all-gather of the partial rows and their log-sum-exps (NCCL), and a "
+                                  "local merge"},
+        "clocks": clocks, "exchange_bytes_per_rank_per_call": exchange_bytes,
+        "gpu_launches": 3 * calls,
+    }
+
+
+def run_shard_keys(args):
+    """One long cache split by key range over the ranks (`torchrun ... bench.py --gpus N --shard-keys`): per
+    layer call yoco_xattn_decode_partial on the local keys, all-gather of the partials, local merge."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd, shard
+
+    rank, local_rank, world = dist_env()
+    if world != args.gpus and not (world == 1 and args.gpus == 1):
+        raise SystemExit("--gpus N > 1 must be launched with torchrun (one rank per GPU)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        # the communicator's own log (which shows the ranks and the transport picked) goes to a file, not to stdout
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_FILE", os.path.join(tempfile.gettempdir(), "nccl_shard_keys_%h_%p.log"))
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    w = si.workload(args.workload)
+    if w.B != 1 or w.T != 1:
+        raise SystemExit("--shard-keys runs the single-sequence decode workloads")
+    N = int(w.kv_len[0])
+    off, cnt = shard.key_range_shards([N], world)
+    o, n_local = int(off[rank, 0]), int(cnt[rank, 0])
+    # this rank's keys only: head c holds elements [c * N * d + o * d, ... + n_local * d) of the whole tensor
+    def local(tid, mult):
+        parts = [si.normal_bf16(w.seed, tid, n_local * w.d, mult=mult, first=(c * N + o) * w.d) for c in range(w.Hkv)]
+        return torch.from_numpy(np.concatenate(parts).view(np.int16)).to(dev).view(torch.bfloat16)
+    K, V = local(si.TID_K, w.k_mult), local(si.TID_V, 1.0)
+    Qd = [torch.from_numpy(w.make_q(l).reshape(-1).view(np.int16)).to(dev).view(torch.bfloat16) for l in range(w.layers)]
+    rows = w.B * w.Hq
+    lens = np.array([n_local], dtype=np.int32)
+    shape = bd.make_shape(1, w.Hq, w.Hkv, w.d, 1, max_kv_len=n_local)
+    ws = torch.empty(bd.yoco_xattn_workspace_size(shape, lens, bd.MODE_DECODE), dtype=torch.uint8, device=dev)
+    part_o = torch.empty((rows, w.d), dtype=torch.float32, device=dev)
+    part_l = torch.empty((rows,), dtype=torch.float32, device=dev)
+    Od = [torch.empty(rows * w.d, dtype=torch.bfloat16, device=dev) for _ in range(w.layers)]
+
+    def one_step():
+        for l in range(w.layers):
+            bd.yoco_xattn_decode_partial(shape, Qd[l], K, V, None, lens, part_o, part_l, ws)
+            all_o, all_l = shard.exchange_partials(part_o, part_l)
+            bd.yoco_xattn_combine_gathered(all_o, all_l, Od[l], None)
+
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        one_step()
+    assert bd.yoco_xattn_status(ws) == 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    ev0.record()
+    for _ in range(args.steps):
+        one_step()
+    ev1.record()
+    torch.cuda.synchronize()
+    barrier()
+    t1 = time.time()
+    total_ms = max_over_ranks([ev0.elapsed_time(ev1)], dev)[0]
+    assert bd.yoco_xattn_status(ws) == 0 and bool(torch.isfinite(Od[-1].float()).all())
+    clocks = sampler.stop(t0, t1) if sampler else None
+    if rank == 0:
+        print(json.dumps(shard_keys_line(w, world, args.steps, warm, total_ms, clocks, rows * (w.d + 1) * 4)), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
 def run_ours(args):
     import torch
     from paper_2405_05254_b200 import binding as bd
@@ -715,10 +811,15 @@ def main():
     ap.add_argument("--no-shard", action="store_true", help="skip the key-range-shard measurement")
     ap.add_argument("--no-window", action="store_true", help="skip the sliding-window decode measurement")
     ap.add_argument("--only-chunk", action="store_true", help="measure the chunk path alone")
+    ap.add_argument("--shard-keys", action="store_true",
+                    help="split the keys of the one long cache over the --gpus ranks (launch with torchrun): partial "
+                         "decode, all-gather of the partials, local merge; value = whole-cache bytes / slowest rank")
     ap.add_argument("--chunk-workload", default="chunk", choices=["chunk", "chunk_32k"])
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.shard_keys:
+        run_shard_keys(args)
     else:
         run_ours(args)
 

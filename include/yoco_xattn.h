@@ -242,20 +242,48 @@ int32_t yoco_xattn_combine_gathered(int64_t rows, int32_t S, int32_t d, const fl
                                     const float* part_lse, void* O, float* lse, void* stream);
 
 /* Decode over ONE SHARD of the keys, for key-range sharding of a long cache across GPUs (the
- * K^, V^ of Section 2.2 split along the sequence, as sequence-parallel prefill leaves them).
- * K, V, cu_kv_host, kv_len_host describe the keys this GPU holds (an ordinary packed cache,
- * kv_len[i] may be 0); the result is the attention over those keys only:
- *   part_o   [B*Hq, d] fp32, normalised over the shard's keys (0 where the shard is empty)
- *   part_lse [B*Hq]    fp32, natural-log sum of exp(score) over the shard's keys (-inf if empty)
+ * K^, V^ of Section 2.2 split along the sequence, as the chunk-parallel prefill of Appendix A leaves
+ * them before its all-gather).  K, V, cu_kv_host, kv_len_host describe the keys this GPU holds (an
+ * ordinary packed cache, kv_len[i] may be 0); the result is the attention over those keys only:
+ *   part_o   [B*Hq*T, d] fp32, normalised over the shard's keys (0 where the shard holds nothing a row sees)
+ *   part_lse [B*Hq*T]    fp32, natural-log sum of exp(score) over the shard's keys (-inf if none)
  * Exchanging (part_o, part_lse) between the shards and merging them with
  * yoco_xattn_combine_gathered gives exactly softmax(QK^T)V over the whole cache (the log-sum-exp
- * merge is algebraically exact).  Requires T = 1 and no window: with one query row per head every
- * key of a shard is visible whichever shard holds the row's own position.  Workspace as for
- * yoco_xattn_decode.  All pointers device unless marked host. */
+ * merge is algebraically exact).  Workspace as for yoco_xattn_decode.  All pointers device unless
+ * marked host.
+ *
+ * yoco_xattn_decode_partial knows nothing of where the shard sits in the sequence and therefore
+ * requires T = 1 and no window: with one query row per head every key of a shard is visible
+ * whichever shard holds the row's own position.
+ * The _at forms take the shard's place: key_offset_host[i] = index, in sequence i, of the first key
+ * held here, kv_total_host[i] = N_i of the whole sequence (host [B] each; key_offset + kv_len <=
+ * kv_total).  Query row t then sits at position N_i - T + t of the whole sequence and the causal
+ * rule and the window of shape->window apply to whole-sequence key positions, so any T and any
+ * window work: decode_partial_at for G*T <= 16 rows per KV head, chunk_partial_at (the tensor-core
+ * path) for any T.  Their workspace is sized by yoco_xattn_workspace_size_at. */
 int32_t yoco_xattn_decode_partial(const yoco_xattn_shape* shape, const void* Q, const void* K,
                                   const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
                                   float* part_o, float* part_lse, void* workspace,
                                   size_t workspace_bytes, void* stream);
+int32_t yoco_xattn_decode_partial_at(const yoco_xattn_shape* shape, const void* Q, const void* K,
+                                     const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
+                                     const int32_t* key_offset_host, const int32_t* kv_total_host,
+                                     float* part_o, float* part_lse, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+int32_t yoco_xattn_chunk_partial_at(const yoco_xattn_shape* shape, const void* Q, const void* K,
+                                    const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
+                                    const int32_t* key_offset_host, const int32_t* kv_total_host,
+                                    float* part_o, float* part_lse, void* workspace,
+                                    size_t workspace_bytes, void* stream);
+/* (No counterpart in the paper.)  yoco_xattn_plan and yoco_xattn_workspace_size for a shard at a given
+ * place (arguments as above): only the keys that some row of the call sees are planned. */
+int32_t yoco_xattn_plan_at(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
+                           const int32_t* key_offset_host, const int32_t* kv_total_host, int32_t sm_count,
+                           int32_t mode, yoco_xattn_plan_info* info, yoco_xattn_segment* segments_out,
+                           int32_t capacity);
+int32_t yoco_xattn_workspace_size_at(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
+                                     const int32_t* key_offset_host, const int32_t* kv_total_host,
+                                     int32_t sm_count, int32_t mode, size_t* bytes);
 
 /* ---- Writing the cache (Section 2.2, first cross-decoder equation) -------------------------
  *   K^ = LN(X) W_K,  V^ = LN(X) W_V,  LN = RMSNorm (Section 2.1), no bias:

@@ -74,6 +74,14 @@ def lib() -> ctypes.CDLL:
         L.yoco_xattn_combine.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
         L.yoco_xattn_combine_gathered.argtypes = [i64, i32, i32, vp, vp, vp, vp, vp]
         L.yoco_xattn_decode_partial.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        part_at = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.yoco_xattn_decode_partial_at.argtypes = part_at
+        L.yoco_xattn_chunk_partial_at.argtypes = part_at
+        L.yoco_xattn_workspace_size_at.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, i32, i32, ctypes.POINTER(sz)]
+        L.yoco_xattn_plan_at.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, i32, i32, ctypes.POINTER(PlanInfo), vp, i32]
+        for name in ("yoco_xattn_decode_partial_at", "yoco_xattn_chunk_partial_at", "yoco_xattn_workspace_size_at",
+                     "yoco_xattn_plan_at"):
+            getattr(L, name).restype = i32
         L.yoco_xattn_decode_fp8.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.yoco_xattn_decode_fp8.restype = i32
         L.yoco_kv_fold_gain.argtypes = [i64, i64, vp, vp, vp, vp]
@@ -130,6 +138,23 @@ def yoco_xattn_plan(shape: Shape, kv_len, sm_count: int, mode: int):
                                ctypes.cast(segs, ctypes.c_void_p), info.num_segments)
     if rc != OK:
         raise YocoError(rc, "yoco_xattn_plan")
+    return info, list(segs)[: info.num_segments]
+
+
+def yoco_xattn_plan_at(shape: Shape, kv_len, key_offset, kv_total, sm_count: int, mode: int):
+    """(PlanInfo, segments) for one key shard at a given place in the whole sequences; host only."""
+    keep, p_len = _host_i32(kv_len)
+    keep_off, p_off = _host_i32(key_offset)
+    keep_tot, p_tot = _host_i32(kv_total)
+    info = PlanInfo()
+    rc = lib().yoco_xattn_plan_at(ctypes.byref(shape), p_len, p_off, p_tot, sm_count, mode, ctypes.byref(info), None, 0)
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_plan_at")
+    segs = (Segment * max(1, info.num_segments))()
+    rc = lib().yoco_xattn_plan_at(ctypes.byref(shape), p_len, p_off, p_tot, sm_count, mode, ctypes.byref(info),
+                                  ctypes.cast(segs, ctypes.c_void_p), info.num_segments)
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_plan_at")
     return info, list(segs)[: info.num_segments]
 
 
@@ -225,6 +250,34 @@ def yoco_xattn_decode_partial(shape: Shape, Q, K, V, cu_kv, kv_len, part_o, part
                                          workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     if rc != OK:
         raise YocoError(rc, "yoco_xattn_decode_partial")
+
+
+def yoco_xattn_partial_at(shape: Shape, Q, K, V, cu_kv, kv_len, key_offset, kv_total, part_o, part_lse, workspace,
+                          mode: int = MODE_DECODE, stream=None) -> None:
+    """One key shard's partial result with the shard's place in the whole sequences (host int32 [B] each:
+    first key held here, length of the whole sequence): any T and any window.  ``mode`` picks the split-KV
+    decode kernel (G*T <= 16) or the tensor-core chunk kernel."""
+    keep_cu, p_cu = _host_i32(cu_kv)
+    keep_len, p_len = _host_i32(kv_len)
+    keep_off, p_off = _host_i32(key_offset)
+    keep_tot, p_tot = _host_i32(kv_total)
+    name = "yoco_xattn_decode_partial_at" if mode == MODE_DECODE else "yoco_xattn_chunk_partial_at"
+    rc = getattr(lib(), name)(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), p_cu, p_len, p_off, p_tot,
+                              _ptr(part_o), _ptr(part_lse), _ptr(workspace),
+                              workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, name)
+
+
+def yoco_xattn_workspace_size_at(shape: Shape, kv_len, key_offset, kv_total, mode: int, sm_count: int = 0) -> int:
+    keep_len, p_len = _host_i32(kv_len)
+    keep_off, p_off = _host_i32(key_offset)
+    keep_tot, p_tot = _host_i32(kv_total)
+    out = ctypes.c_size_t(0)
+    rc = lib().yoco_xattn_workspace_size_at(ctypes.byref(shape), p_len, p_off, p_tot, sm_count, mode, ctypes.byref(out))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_workspace_size_at")
+    return int(out.value)
 
 
 def yoco_xattn_decode_fp8(shape: Shape, Q, K8, V8, k_scale, v_scale, cu_kv, kv_len, O, lse, workspace,

@@ -62,10 +62,11 @@ int32_t device_state(DeviceState** out) {
 struct PlanKey {
     yoco_xattn_shape shape;
     int32_t sm_count, mode, max_sub;
-    std::vector<int32_t> lens, cu;
+    std::vector<int32_t> lens, cu, key_off, totals;
     bool operator==(const PlanKey& o) const {
         return std::memcmp(&shape, &o.shape, sizeof shape) == 0 && sm_count == o.sm_count &&
-               mode == o.mode && max_sub == o.max_sub && lens == o.lens && cu == o.cu;
+               mode == o.mode && max_sub == o.max_sub && lens == o.lens && cu == o.cu &&
+               key_off == o.key_off && totals == o.totals;
     }
 };
 // A cached plan with the launch-ready forms of its tables.
@@ -89,7 +90,8 @@ std::vector<std::shared_ptr<const ReadyPlan>> g_captured_plans;
 // Looks the plan up (most recently used first) or makes it.  The shared pointer keeps the entry
 // alive for the caller even if another thread evicts it from the cache meanwhile.
 int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t* lens, int32_t sm_count,
-                    int32_t mode, int32_t max_sub, std::shared_ptr<const ReadyPlan>& out) {
+                    int32_t mode, int32_t max_sub, std::shared_ptr<const ReadyPlan>& out,
+                    const int32_t* key_off = nullptr, const int32_t* totals = nullptr) {
     PlanKey key;
     std::memset(&key.shape, 0, sizeof key.shape);
     key.shape = s;
@@ -98,6 +100,8 @@ int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t*
     key.max_sub = max_sub;
     if (lens) key.lens.assign(lens, lens + s.B);
     if (cu) key.cu.assign(cu, cu + s.B + 1);
+    if (key_off) key.key_off.assign(key_off, key_off + s.B);
+    if (totals) key.totals.assign(totals, totals + s.B);
     {
         std::lock_guard<std::mutex> lock(g_mutex);
         for (auto it = g_plans.begin(); it != g_plans.end(); ++it)
@@ -108,7 +112,7 @@ int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t*
             }
     }
     auto ready = std::make_shared<ReadyPlan>();
-    int32_t rc = make_plan(s, cu, lens, sm_count, mode, ready->plan, max_sub);
+    int32_t rc = make_plan(s, cu, lens, sm_count, mode, ready->plan, max_sub, key_off, totals);
     if (rc != YOCO_OK) return rc;
     const Plan& plan = ready->plan;
     ready->blob.assign(kWorkspaceHeaderBytes / 4 + plan.table.size(), 0);
@@ -120,6 +124,8 @@ int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t*
         std::memset(&ready->combine_tab, 0, sizeof ready->combine_tab);
         std::memcpy(ready->decode_tab.seg, plan.table.data() + plan.off_segments,
                     (size_t)plan.coarse_segments * sizeof(DevSegment));
+        static_assert(sizeof(DecodeInlineTables) + sizeof(DecodeFp8Params) + 2 * sizeof(CUtensorMap) < 32000,
+                      "kernel parameter space");
         std::memcpy(ready->decode_tab.group_begin, plan.table.data() + plan.off_group_begin,
                     (size_t)(plan.info.num_groups + 1) * 4);
         std::memcpy(ready->combine_tab.stream_base, plan.table.data() + plan.off_stream_base,
@@ -255,11 +261,17 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 struct SelfTest {
     int64_t wait_limit_ns;
 };
+// where the keys of this call sit in the whole sequences (one shard of a key-range-sharded cache)
+struct ShardPos {
+    const int32_t* key_offset;   // host [B]
+    const int32_t* kv_total;     // host [B]
+};
 
 int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const void* K, const void* V,
             const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
             void* workspace, size_t workspace_bytes, void* stream_v, float* part_out = nullptr,
-            const Fp8Scales* fp8 = nullptr, int32_t max_sub = kMaxSubItems, const SelfTest* selftest = nullptr) {
+            const Fp8Scales* fp8 = nullptr, int32_t max_sub = kMaxSubItems, const SelfTest* selftest = nullptr,
+            const ShardPos* shard = nullptr) {
     // part_out != null: the result is a partial one (fp32 rows + their LSE in `lse`, no bf16 O)
     if (!shape) return YOCO_ERR_INVALID_ARG;
     int32_t rc = validate_shape(*shape, mode);
@@ -279,7 +291,8 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
     // The 8-bit kernel runs one piece per group: it is paced by its own instruction chains, evenly
     // on every SM, and handing out pieces made it slower (351 us against 331 us at 1M keys).
     if (fp8) max_sub = 1;
-    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, mode, max_sub, ready)) != YOCO_OK)
+    if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, mode, max_sub, ready,
+                          shard ? shard->key_offset : nullptr, shard ? shard->kv_total : nullptr)) != YOCO_OK)
         return rc;
     const Plan& plan = ready->plan;
     if ((int64_t)workspace_bytes < plan.info.workspace_bytes) return YOCO_ERR_WORKSPACE_TOO_SMALL;
@@ -383,6 +396,7 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             p.m_tiles = plan.info.m_tiles;
             p.d = shape->d;
             p.window = shape->window;
+            p.force_partial = part_out ? 1 : 0;
             if (plan.info.tile_m == kChunkPairTileM)
                 YOCO_CUDA_TRY(launch_chunk_pair(p, tmQ, tmK, tmV, plan.info.num_groups, stream));
             else
@@ -453,9 +467,16 @@ extern "C" {
 int32_t yoco_xattn_plan(const yoco_xattn_shape* shape, const int32_t* kv_len_host, int32_t sm_count,
                         int32_t mode, yoco_xattn_plan_info* info, yoco_xattn_segment* segments_out,
                         int32_t capacity) {
+    return yoco_xattn_plan_at(shape, kv_len_host, nullptr, nullptr, sm_count, mode, info, segments_out, capacity);
+}
+
+int32_t yoco_xattn_plan_at(const yoco_xattn_shape* shape, const int32_t* kv_len_host, const int32_t* key_offset_host,
+                           const int32_t* kv_total_host, int32_t sm_count, int32_t mode, yoco_xattn_plan_info* info,
+                           yoco_xattn_segment* segments_out, int32_t capacity) {
     if (!shape || !info || capacity < 0 || (capacity > 0 && !segments_out)) return YOCO_ERR_INVALID_ARG;
     Plan plan;
-    int32_t rc = make_plan(*shape, nullptr, kv_len_host, sm_count, mode, plan);
+    int32_t rc = make_plan(*shape, nullptr, kv_len_host, sm_count, mode, plan, kMaxSubItems, key_offset_host,
+                           kv_total_host);
     if (rc != YOCO_OK) return rc;
     *info = plan.info;
     const int32_t n = std::min<int32_t>(capacity, (int32_t)plan.segments.size());
@@ -470,6 +491,12 @@ int64_t yoco_xattn_sub_bound(int64_t n_tiles, int32_t sub_items, int32_t r) {
 
 int32_t yoco_xattn_workspace_size(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
                                   int32_t sm_count, int32_t mode, size_t* bytes) {
+    return yoco_xattn_workspace_size_at(shape, kv_len_host, nullptr, nullptr, sm_count, mode, bytes);
+}
+
+int32_t yoco_xattn_workspace_size_at(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
+                                     const int32_t* key_offset_host, const int32_t* kv_total_host,
+                                     int32_t sm_count, int32_t mode, size_t* bytes) {
     if (!shape || !bytes || sm_count < 0) return YOCO_ERR_INVALID_ARG;
     if (sm_count == 0) {
         int32_t rc = validate_shape(*shape, mode);
@@ -479,7 +506,8 @@ int32_t yoco_xattn_workspace_size(const yoco_xattn_shape* shape, const int32_t* 
         sm_count = dev->sm_count;
     }
     Plan plan;
-    int32_t rc = make_plan(*shape, nullptr, kv_len_host, sm_count, mode, plan);
+    int32_t rc = make_plan(*shape, nullptr, kv_len_host, sm_count, mode, plan, kMaxSubItems, key_offset_host,
+                           kv_total_host);
     if (rc != YOCO_OK) return rc;
     *bytes = (size_t)plan.info.workspace_bytes;
     return YOCO_OK;
@@ -557,15 +585,46 @@ int32_t yoco_xattn_combine_gathered(int64_t rows, int32_t S, int32_t d, const fl
     return combine_public(rows, S, d, part_o, part_lse, O, lse, stream, 1);
 }
 
+namespace {
+int32_t partial_impl(int32_t mode, const yoco_xattn_shape* shape, const void* Q, const void* K, const void* V,
+                     const int32_t* cu_kv_host, const int32_t* kv_len_host, const int32_t* key_offset_host,
+                     const int32_t* kv_total_host, float* part_o, float* part_lse, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    if (!shape || !part_o || !part_lse) return YOCO_ERR_INVALID_ARG;
+    if ((key_offset_host == nullptr) != (kv_total_host == nullptr)) return YOCO_ERR_INVALID_ARG;
+    // Without the shard's place in the sequence only T = 1 without a window can be answered: then every
+    // key of a shard is visible whatever follows it on other shards.
+    if (!key_offset_host && (shape->T != 1 || shape->window != 0)) return YOCO_ERR_UNSUPPORTED;
+    if (key_offset_host && !kv_len_host) return YOCO_ERR_INVALID_ARG;
+    const ShardPos pos{key_offset_host, kv_total_host};
+    return run(shape, mode, Q, K, V, cu_kv_host, kv_len_host, nullptr, part_lse, workspace, workspace_bytes, stream,
+               part_o, nullptr, kMaxSubItems, nullptr, key_offset_host ? &pos : nullptr);
+}
+}  // namespace
+
 int32_t yoco_xattn_decode_partial(const yoco_xattn_shape* shape, const void* Q, const void* K, const void* V,
                                   const int32_t* cu_kv_host, const int32_t* kv_len_host, float* part_o,
                                   float* part_lse, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!shape || !part_o || !part_lse) return YOCO_ERR_INVALID_ARG;
-    // one query row per head: then every key of a shard is visible whatever follows it on other
-    // shards, and a shard is an ordinary (shorter) cache; a window would need global positions
-    if (shape->T != 1 || shape->window != 0) return YOCO_ERR_UNSUPPORTED;
-    return run(shape, YOCO_MODE_DECODE, Q, K, V, cu_kv_host, kv_len_host, nullptr, part_lse, workspace,
-               workspace_bytes, stream, part_o);
+    return partial_impl(YOCO_MODE_DECODE, shape, Q, K, V, cu_kv_host, kv_len_host, nullptr, nullptr, part_o, part_lse,
+                        workspace, workspace_bytes, stream);
+}
+
+int32_t yoco_xattn_decode_partial_at(const yoco_xattn_shape* shape, const void* Q, const void* K, const void* V,
+                                     const int32_t* cu_kv_host, const int32_t* kv_len_host,
+                                     const int32_t* key_offset_host, const int32_t* kv_total_host, float* part_o,
+                                     float* part_lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!key_offset_host || !kv_total_host) return YOCO_ERR_INVALID_ARG;
+    return partial_impl(YOCO_MODE_DECODE, shape, Q, K, V, cu_kv_host, kv_len_host, key_offset_host, kv_total_host,
+                        part_o, part_lse, workspace, workspace_bytes, stream);
+}
+
+int32_t yoco_xattn_chunk_partial_at(const yoco_xattn_shape* shape, const void* Q, const void* K, const void* V,
+                                    const int32_t* cu_kv_host, const int32_t* kv_len_host,
+                                    const int32_t* key_offset_host, const int32_t* kv_total_host, float* part_o,
+                                    float* part_lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!key_offset_host || !kv_total_host) return YOCO_ERR_INVALID_ARG;
+    return partial_impl(YOCO_MODE_CHUNK, shape, Q, K, V, cu_kv_host, kv_len_host, key_offset_host, kv_total_host,
+                        part_o, part_lse, workspace, workspace_bytes, stream);
 }
 
 int32_t yoco_xattn_decode_fp8(const yoco_xattn_shape* shape, const void* Q, const void* K8, const void* V8,

@@ -269,11 +269,12 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
         for (int si = seg_lo; si < seg_hi; ++si) {
             const DevSegment seg = p.segments[si];
-            const int n_full = seg.n_kv - p.T + 1;     // keys visible to every row
+            const int n_full = seg.n_full;     // keys visible to row 0 (row t sees n_full + t), see DevSegment
+            const int n_edge = min(n_full, seg.n_kv);      // tiles that end at or below it need no mask
             const int vis = min(seg.n_kv, max(0, n_full + (r_local % p.T)));
             // sliding window: the row at position i keeps i - C < j; lo_max is the highest such bound
             const int lo = p.window > 0 ? max(0, n_full + (r_local % p.T) - p.window) : 0;
-            const int lo_max = p.window > 0 ? seg.n_kv - p.window : 0;
+            const int lo_max = p.window > 0 ? n_full + p.T - 1 - p.window : 0;
             float m_ref = -INFINITY, l = 0.f;
             const uint32_t seg_first_it = it, seg_first_u = 2 * it;
             int pending = -1;                          // half step whose P is stored but not yet announced
@@ -306,7 +307,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     tmem_wait_ld();
                     announce();                                // the previous half step's P
 
-                    const bool masked = !(kh + BH <= n_full && kh >= lo_max);   // causal edge, sequence end or window start
+                    const bool masked = !(kh + BH <= n_edge && kh >= lo_max);   // causal edge, sequence end or window start
                     if (masked) {
 #pragma unroll
                         for (int j = 0; j < BH; ++j) s[j] = (kh + j < vis && kh + j >= lo) ? s[j] : -INFINITY;
@@ -405,7 +406,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 const bool has = l > 0.f;
                 const float inv = has ? 1.f / l : 0.f;
                 const float lse = has ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
-                const bool final_out = seg.stream_nseg == 1;
+                const bool final_out = seg.stream_nseg == 1 && !p.force_partial;
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     float o[32];

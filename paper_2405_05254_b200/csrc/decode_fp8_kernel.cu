@@ -166,7 +166,8 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
                 bf16x4_to_f16x4(w1, qa[ks][1], qa[ks][3]);
             }
         }
-        const int n_full = seg.n_kv - p.T + 1;
+        const int n_full = seg.n_full;
+        const int n_edge = min(n_full, seg.n_kv);      // tiles that end at or below it need no mask
         const int vis0 = min(seg.n_kv, max(0, n_full + (g % p.T)));
         const int vis1 = min(seg.n_kv, max(0, n_full + ((g + 8) % p.T)));
 
@@ -206,7 +207,7 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
                 }
             }
             // ---- scale, mask (causal edge, sequence end, window start), online softmax ----
-            const bool need_mask = k0 + TILE_N > n_full || (p.window > 0 && k0 < seg.n_kv - p.window);
+            const bool need_mask = k0 + TILE_N > n_edge || (p.window > 0 && k0 < n_full + p.T - 1 - p.window);
             int lo0 = -1, lo1 = -1;
             if (need_mask && p.window > 0) {
                 lo0 = n_full + (g % p.T) - p.window;

@@ -219,8 +219,10 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
                     qa[ks][3] = v1 ? ld_global_u32(q1 + ks * 16 + 8) : 0u;
                 }
             }
-            // causal limits: row t sees keys j < n_kv - T + 1 + t
-            const int n_full = seg.n_kv - p.T + 1;
+            // causal limits: row t sees keys j < n_full + t (n_full = N - T + 1 for a whole cache; for a key
+            // shard the same count less the keys of earlier shards) and none past the keys held here
+            const int n_full = seg.n_full;
+            const int n_edge = min(n_full, seg.n_kv);      // tiles that end at or below it need no mask
             const int vis0 = min(seg.n_kv, max(0, n_full + (g % p.T)));
             const int vis1 = min(seg.n_kv, max(0, n_full + ((g + 8) % p.T)));
 
@@ -261,9 +263,9 @@ __device__ __forceinline__ void decode_body(const CUtensorMap& tmK, const CUtens
                         }
                     }
                     // ---- scale, mask, online softmax ----
-                    // sliding window: the row at position i = n_kv - T + t keeps i - C < j, i.e.
-                    // j >= i - C + 1 = n_full + t - C; the highest such bound of any row is n_kv - C
-                    const bool need_mask = kw + 16 > n_full || (p.window > 0 && kw < seg.n_kv - p.window);
+                    // sliding window: the row at position i keeps i - C < j, i.e. j >= i - C + 1 =
+                    // n_full + t - C; the highest such bound of any row is n_full + T - 1 - C
+                    const bool need_mask = kw + 16 > n_edge || (p.window > 0 && kw < n_full + p.T - 1 - p.window);
                     // window start of the two rows this lane holds (no window: below every key)
                     int lo0 = -1, lo1 = -1;
                     if (need_mask && p.window > 0) {

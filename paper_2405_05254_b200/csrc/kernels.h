@@ -130,6 +130,7 @@ struct ChunkParams {
     int32_t m_tiles;            // ceil(rows_per_stream / 128)
     int32_t d;
     int32_t window;             // sliding window C, 0 = none
+    int32_t force_partial;      // write every segment to its partial slot, even of an unsplit stream
 };
 // tmQ: [B*Hq*T, d] box {64, 128}; tmK / tmV: [rows, d] box {64, kChunkTileN}; 128-byte swizzle.
 // Grid = num_groups * m_tiles CTAs, the row tile varying fastest so that the CTAs that walk the

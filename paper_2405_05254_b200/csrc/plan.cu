@@ -2,6 +2,7 @@
 #include "plan.h"
 
 #include <algorithm>
+#include <climits>
 
 namespace yoco {
 
@@ -35,7 +36,8 @@ int32_t validate_layout(const yoco_xattn_shape& s, const int32_t* cu_kv_host, co
 }
 
 int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const int32_t* kv_len_host,
-                  int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items) {
+                  int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items,
+                  const int32_t* key_offset_host, const int32_t* kv_total_host) {
     int32_t rc = validate_shape(s, mode);
     if (rc != YOCO_OK) return rc;
     if (sm_count <= 0) return YOCO_ERR_INVALID_ARG;
@@ -50,11 +52,22 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     const int num_streams = s.B * s.Hkv;
 
     // per-sequence geometry
+    if ((key_offset_host == nullptr) != (kv_total_host == nullptr)) return YOCO_ERR_INVALID_ARG;
     std::vector<int64_t> tok_off(s.B + 1, 0);
     std::vector<int32_t> len(s.B, 0);
+    std::vector<int64_t> n_full(s.B, 0);     // keys of this cache that query row 0 sees (see DevSegment)
+    std::vector<int32_t> len_vis(s.B, 0);    // keys of this cache that at least the last row sees
     int64_t extent = 0;
     for (int i = 0; i < s.B; ++i) {
         len[i] = kv_len_host ? kv_len_host[i] : s.max_kv_len;
+        if (key_offset_host) {
+            if (key_offset_host[i] < 0 || len[i] < 0 || (int64_t)key_offset_host[i] + len[i] > kv_total_host[i])
+                return YOCO_ERR_INVALID_ARG;
+            n_full[i] = (int64_t)kv_total_host[i] - s.T + 1 - key_offset_host[i];
+        } else {
+            n_full[i] = (int64_t)len[i] - s.T + 1;
+        }
+        len_vis[i] = (int32_t)std::min<int64_t>(std::max<int64_t>(len[i], 0), std::max<int64_t>(n_full[i] + s.T - 1, 0));
         if (cu_kv_host) tok_off[i] = cu_kv_host[i];
         const int64_t head_rows = s.kv_head_stride ? s.kv_head_stride / s.d : len[i];
         if (!cu_kv_host) tok_off[i + 1] = tok_off[i] + head_rows;
@@ -69,10 +82,10 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     int64_t total_tiles = 0;
     for (int i = 0; i < s.B; ++i) {
         if (s.window > 0) {
-            const int64_t lo = (int64_t)len[i] - s.T - s.window + 1;
-            tile_lo[i] = std::min<int64_t>(std::max<int64_t>(lo, 0) / tile_n, (len[i] + tile_n - 1) / tile_n);
+            const int64_t lo = n_full[i] - s.window;      // lowest key row 0 sees
+            tile_lo[i] = std::min<int64_t>(std::max<int64_t>(lo, 0) / tile_n, (len_vis[i] + tile_n - 1) / tile_n);
         }
-        total_tiles += (int64_t)s.Hkv * ((len[i] + tile_n - 1) / tile_n - tile_lo[i]);
+        total_tiles += (int64_t)s.Hkv * ((len_vis[i] + tile_n - 1) / tile_n - tile_lo[i]);
     }
 
     // number of CTA groups
@@ -95,7 +108,7 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     int64_t g = 0;          // current group
     auto group_lo = [&](int64_t p) { return p * total_tiles / num_groups; };
     for (int b = 0; b < s.B; ++b) {
-        const int64_t nt = (len[b] + tile_n - 1) / tile_n;
+        const int64_t nt = (len_vis[b] + tile_n - 1) / tile_n;
         const int64_t head_rows = s.kv_head_stride ? s.kv_head_stride / s.d : len[b];
         for (int c = 0; c < s.Hkv; ++c) {
             const int stream = b * s.Hkv + c;
@@ -107,12 +120,13 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
                 const int64_t t_end = std::min<int64_t>(nt, group_lo(g + 1) - flat + t0);
                 DevSegment d{};
                 d.k_begin = (int32_t)(t * tile_n);
-                d.k_end = (int32_t)std::min<int64_t>(t_end * tile_n, len[b]);
+                d.k_end = (int32_t)std::min<int64_t>(t_end * tile_n, len_vis[b]);
                 d.kv_row0 = (int32_t)(tok_off[b] * s.Hkv + c * head_rows + d.k_begin);
                 d.q_row0 = (b * s.Hq + c * G) * s.T;
                 d.slot = (int32_t)dev.size();
                 d.n_kv = len[b];
                 d.stream = stream;
+                d.n_full = (int32_t)std::max<int64_t>(std::min<int64_t>(n_full[b], INT32_MAX), INT32_MIN / 2);
                 yoco_xattn_segment pub{(int32_t)g, b, c, d.k_begin, d.k_end, d.slot};
                 plan.segments.push_back(pub);
                 dev.push_back(d);
@@ -175,14 +189,14 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
 
     // device blob
     plan.off_segments = 0;
-    plan.off_group_begin = (int32_t)(dev.size() * 8);
+    plan.off_group_begin = (int32_t)(dev.size() * kSegmentWords);
     plan.off_stream_base = plan.off_group_begin + (int32_t)group_begin.size();
     plan.off_stream_nseg = plan.off_stream_base + num_streams;
     plan.table.resize(plan.off_stream_nseg + num_streams);
-    static_assert(sizeof(DevSegment) == 32, "DevSegment is 8 int32");
+    static_assert(sizeof(DevSegment) == 4 * kSegmentWords, "DevSegment is kSegmentWords int32");
     for (size_t k = 0; k < dev.size(); ++k) {
         const int32_t* w = reinterpret_cast<const int32_t*>(&dev[k]);
-        std::copy(w, w + 8, plan.table.begin() + k * 8);
+        std::copy(w, w + kSegmentWords, plan.table.begin() + k * kSegmentWords);
     }
     std::copy(group_begin.begin(), group_begin.end(), plan.table.begin() + plan.off_group_begin);
     std::copy(stream_base.begin(), stream_base.end(), plan.table.begin() + plan.off_stream_base);

@@ -57,7 +57,7 @@ inline int choose_sub_items(int64_t tiles_per_group, int max_sub) {
     return R < 1 ? 1 : R;
 }
 
-// One work segment as the kernels read it (8 x int32 = 32 bytes).
+// One work segment as the kernels read it (10 x int32 = 40 bytes).
 struct DevSegment {
     int32_t kv_row0;     // row of key k_begin in the [rows, d] view of the packed K/V buffers
     int32_t k_begin;     // first key of the range inside its sequence
@@ -67,7 +67,12 @@ struct DevSegment {
     int32_t n_kv;        // N_i of the sequence
     int32_t stream_nseg; // segments of this stream (1: the kernel writes the final output)
     int32_t stream;      // b * Hkv + c
+    int32_t n_full;      // keys (counted from key 0 of this cache) that query row 0 sees: N_i - T + 1 for a
+                         // whole cache; for one shard of a key-range-sharded cache the same count minus
+                         // the keys held by earlier shards (may be <= 0 or exceed n_kv).  Row t sees n_full + t.
+    int32_t pad_;
 };
+constexpr int kSegmentWords = 10;
 
 struct Plan {
     yoco_xattn_plan_info info{};
@@ -86,8 +91,12 @@ struct Plan {
 
 // Returns YOCO_OK or an error code; fills `plan`.  cu_kv_host may be null (tight packing).
 // max_sub_items: upper limit of pieces per decode group (1 = every group is one piece).
+// key_offset_host / kv_total_host (both null, or both [B]): the cache described by kv_len_host is
+// keys [key_offset[i], key_offset[i] + kv_len[i]) of a sequence of kv_total[i] keys; the causal and
+// window masks then use the rows' positions in the whole sequence.
 int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const int32_t* kv_len_host,
-                  int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items = kMaxSubItems);
+                  int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items = kMaxSubItems,
+                  const int32_t* key_offset_host = nullptr, const int32_t* kv_total_host = nullptr);
 
 int32_t validate_shape(const yoco_xattn_shape& s, int32_t mode);
 // Lengths, head stride and token offsets must describe sequences that do not overlap (pure host).

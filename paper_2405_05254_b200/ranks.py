@@ -33,3 +33,9 @@ def max_over_ranks(values, device=None):
 def job_throughput_gbs(bytes_per_call: int, calls_per_rank: int, world: int, slowest_ms: float) -> float:
     """Aggregate K/V GB/s of the whole job: all ranks' bytes over the slowest rank's time."""
     return bytes_per_call * calls_per_rank * world / (slowest_ms * 1e-3) / 1e9
+
+
+def sharded_throughput_gbs(whole_cache_bytes: int, calls: int, slowest_ms: float) -> float:
+    """K/V GB/s of a key-range-sharded job: the whole cache is streamed once per layer call, each rank
+    reading its own share, and a call is over when the slowest rank has merged the gathered partials."""
+    return whole_cache_bytes * calls / (slowest_ms * 1e-3) / 1e9

@@ -60,6 +60,55 @@ def test_sharded_decode_merges_to_the_unsharded_attention(world):
         assert (all_o[r].reshape(w.B, w.Hq, w.d)[~live[..., 0]] == 0).all()
 
 
+def sharded_at(w, world, mode, window=0, layer=0):
+    """Every rank's call with the shard's place in the sequence (any T, any window), gathered and merged."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd, shard
+    K, V, Qb = w.make_k(), w.make_v(), w.make_q(layer)
+    Q = to_dev_bf16(Qb.reshape(-1))
+    rows = w.B * w.Hq * w.T
+    tile = 64 if mode == "decode" else 128
+    m = bd.MODE_DECODE if mode == "decode" else bd.MODE_CHUNK
+    off, cnt = shard.key_range_shards(w.kv_len, world, tile=tile)
+    all_o = torch.full((world, rows, w.d), 7.0, dtype=torch.float32, device="cuda")
+    all_l = torch.full((world, rows), 7.0, dtype=torch.float32, device="cuda")
+    for r in range(world):
+        Kr = shard.take_key_range(K, w.kv_len, w.Hkv, w.d, off[r], cnt[r])
+        Vr = shard.take_key_range(V, w.kv_len, w.Hkv, w.d, off[r], cnt[r])
+        Kd = to_dev_bf16(Kr if Kr.size else np.zeros(8, dtype=np.uint16))
+        Vd = to_dev_bf16(Vr if Vr.size else np.zeros(8, dtype=np.uint16))
+        shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(cnt[r].max()), window=window)
+        ws = torch.empty(bd.yoco_xattn_workspace_size_at(shape, cnt[r], off[r], w.kv_len, m), dtype=torch.uint8,
+                         device="cuda")
+        bd.yoco_xattn_partial_at(shape, Q, Kd, Vd, None, cnt[r], off[r], w.kv_len, all_o[r], all_l[r], ws, mode=m)
+        assert bd.yoco_xattn_status(ws) == 0
+    O = torch.empty(rows * w.d, dtype=torch.bfloat16, device="cuda")
+    L = torch.empty(rows, dtype=torch.float32, device="cuda")
+    bd.yoco_xattn_combine_gathered(all_o, all_l, O, L)
+    torch.cuda.synchronize()
+    o_ref, lse_ref = oracle.xattn(Qb, K, V, w.cu, w.kv_len, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T, window=window)
+    assert_close(bf16_dev_to_f64(O).reshape(o_ref.shape), o_ref, f"{mode} x{world} T={w.T} C={window}")
+    assert_lse_close(L.cpu().numpy().reshape(lse_ref.shape), lse_ref, f"{mode} x{world} T={w.T} C={window}")
+    return all_l.cpu().numpy()
+
+
+@pytest.mark.parametrize("world,T,window", [(2, 2, 0), (3, 4, 0), (3, 1, 700), (4, 2, 129), (2, 3, 1)])
+def test_sharded_decode_with_several_rows_and_windows(world, T, window):
+    """Rows of a sharded call sit at their positions in the WHOLE sequence: the causal edge falls into
+    the last shard only, a window may start in any shard, and shards wholly outside a row's window
+    contribute -inf.  Merged result against the oracle on the unsharded cache."""
+    w = si.Workload("shard_t", B=4, Hq=8, Hkv=2, d=128, T=T, layers=1, seed=62, kv_len=[5000, 64 + T, 700, T])
+    all_l = sharded_at(w, world, "decode", window)
+    if window and window < 600:
+        assert np.isneginf(all_l[0].reshape(w.B, w.Hq, T)[0]).all()     # first shard of the long sequence: out of every window
+
+
+@pytest.mark.parametrize("world,T,window", [(2, 40, 0), (3, 200, 0), (2, 130, 300), (3, 64, 2000)])
+def test_sharded_chunk_through_the_tensor_core_path(world, T, window):
+    w = si.Workload("shard_c", B=2, Hq=8, Hkv=2, d=128, T=T, layers=1, seed=63, kv_len=[3000 + T, 517 + T])
+    sharded_at(w, world, "chunk", window)
+
+
 def test_partial_entry_rejects_several_rows_and_windows():
     import torch
     from paper_2405_05254_b200 import binding as bd

@@ -330,6 +330,46 @@ def test_overlapping_offsets_and_a_stride_too_short_are_rejected_on_the_host():
     assert append(ash, [0, 100, 150]) != bd.ERR_INVALID_ARG
 
 
+@pytest.mark.parametrize("T,C", [(1, 0), (5, 0), (1, 300), (7, 300), (40, 1), (3, 100000)])
+def test_plan_of_a_key_shard_covers_exactly_the_keys_some_row_sees(T, C):
+    """A shard holds keys [off, off + n) of a sequence of N keys; query row t sits at position N - T + t
+    of the whole sequence.  The plan of the shard must cover, tile by tile, exactly the local keys from
+    the tile of the lowest key row 0 sees up to the last key the last row sees, for every KV head --
+    restated here from the mask inequalities, not from the planner's code."""
+    N = 20000
+    mode = bd.MODE_DECODE if T * 2 <= 16 else bd.MODE_CHUNK
+    tile = 64 if mode == bd.MODE_DECODE else 128
+    shape = bd.make_shape(3, 4, 2, 128, T, window=C)
+    shards = [(0, 7000), (7000, 9000), (16000, 4000)]          # (offset, count) of the three "sequences"
+    lens = [n for _, n in shards]
+    offs = [o for o, _ in shards]
+    info, segs = bd.yoco_xattn_plan_at(shape, lens, offs, [N] * 3, 148, mode)
+    for b, (off, n) in enumerate(shards):
+        pos0, pos_last = N - T, N - 1                          # whole-sequence positions of the first / last row
+        lo_seen = max(pos0 - C + 1, 0) if C > 0 else 0         # lowest whole-sequence key row 0 sees
+        first = max(lo_seen - off, 0)                          # ... as a local key
+        last = min(pos_last - off, n - 1)                      # highest local key the last row sees
+        for c in range(2):
+            mine = sorted((s.k_begin, s.k_end) for s in segs if s.b == b and s.c == c)
+            if last < first:
+                assert mine == []
+                continue
+            assert mine[0][0] == first // tile * tile and mine[-1][1] == last + 1
+            for (a0, a1), (b0, b1) in zip(mine, mine[1:]):
+                assert a1 == b0 and a1 % tile == 0
+    # offsets and totals come together, and a shard may not reach past its sequence
+    L = bd.lib()
+    p = ctypes.c_void_p
+    a = np.array(lens, dtype=np.int32)
+    o = np.array(offs, dtype=np.int32)
+    t_bad = np.array([N, N, 19999], dtype=np.int32)
+    pi = bd.PlanInfo()
+    assert L.yoco_xattn_plan_at(ctypes.byref(shape), p(a.ctypes.data), p(o.ctypes.data), None, 148, mode,
+                                ctypes.byref(pi), None, 0) == bd.ERR_INVALID_ARG
+    assert L.yoco_xattn_plan_at(ctypes.byref(shape), p(a.ctypes.data), p(o.ctypes.data), p(t_bad.ctypes.data), 148, mode,
+                                ctypes.byref(pi), None, 0) == bd.ERR_INVALID_ARG
+
+
 def test_status_word_names_the_wait_and_the_cta():
     """0 is ok; otherwise the low byte is the kind of wait that ran out and the rest 1 + the CTA."""
     assert bd.yoco_xattn_decode_status_word(0) == (bd.OK, 0, -1)
