@@ -277,6 +277,39 @@ def measure_chunk(dev, peaks, name="chunk"):
             "kv_bytes": w.kv_bytes}
 
 
+def measure_chunk_fp8(dev, peaks, name="chunk"):
+    """The multi-token path over an 8-bit cache on the chunk workload: the same K/V draws quantised to
+    E4M3 with per-head amax / 448 scales, widened to fp16 inside the kernel."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    w = si.workload(name)
+    K8h, V8h, ks, vs = w.make_kv_fp8()
+    K8, V8 = torch.from_numpy(K8h).to(dev), torch.from_numpy(V8h).to(dev)
+    Q = torch.from_numpy(w.make_q(0).reshape(-1).view(np.int16)).to(dev).view(torch.bfloat16)
+    shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(w.kv_len.max()))
+    ws = torch.empty(bd.yoco_xattn_workspace_size_chunk_fp8(shape, w.kv_len), dtype=torch.uint8, device=dev)
+    O = torch.empty(w.B * w.Hq * w.T * w.d, dtype=torch.bfloat16, device=dev)
+
+    def call():
+        bd.yoco_xattn_chunk_fp8(shape, Q, K8, V8, ks, vs, w.cu, w.kv_len, O, None, ws)
+
+    for _ in range(3):
+        call()
+    assert bd.yoco_xattn_status(ws) == 0 and bool(torch.isfinite(O.float()).all())
+    n = 10
+    bd.yoco_xattn_profile_enable(n)
+    for _ in range(n):
+        call()
+    k_ms = float(bd.yoco_xattn_profile_collect(n).mean())
+    bd.yoco_xattn_profile_enable(0)
+    flop = sum(w.Hq * (w.T * (int(nk) - w.T) + w.T * (w.T + 1) / 2) * 4 * w.d for nk in w.kv_len)
+    tf = flop / (k_ms * 1e-3) / 1e12
+    burst = float(peaks.get("bf16_tflops", 1590.0))
+    return {"workload": f"{w.name} over an FP8 E4M3 cache: B={w.B} T={w.T} kv_len={int(w.kv_len[0])}", "kernel_ms": k_ms,
+            "bound": "tensor", "achieved": tf, "unit": "TFLOP/s", "peak": burst, "frac": tf / burst,
+            "kv_bytes": int(K8h.size + V8h.size)}
+
+
 def measure_window(dev, peak_gbs, name="swa"):
     """Batched decode under the sliding-window mask: 128 sequences, window 1,024.  Only the keys
     inside a window are planned and read, so the algorithmic bytes are those of the windows."""
@@ -781,6 +814,8 @@ def run_ours(args):
             del K, V
             torch.cuda.empty_cache()
             line["chunk"] = measure_chunk(dev, peaks, args.chunk_workload)
+            if not args.no_fp8:
+                line["chunk_fp8"] = measure_chunk_fp8(dev, peaks, args.chunk_workload)
         if world == 1 and not args.no_append:
             line["kv_append"] = measure_kv_append(dev, peaks, peak)
         if world == 1 and not args.no_window:

@@ -235,6 +235,19 @@ int32_t yoco_xattn_decode_fp8(const yoco_xattn_shape* shape, const void* Q, cons
                               const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/* The multi-token path over the same 8-bit cache (arguments as yoco_xattn_decode_fp8, any T >= 1): a
+ * prefill or verification chunk against a cache written by yoco_kv_append_fp8.  The bytes are widened
+ * to fp16 inside the kernel (exact), Q and P are rounded to fp16 (|Q| < 65504) and the products run on
+ * the tensor cores as fp16 x fp16 with fp32 accumulation.  d = 128 only, Hkv <= 64.  The workspace is
+ * sized by yoco_xattn_workspace_size_chunk_fp8 (this path always plans two 128-row tiles per CTA, so the
+ * size can differ from that of yoco_xattn_chunk for small T). */
+int32_t yoco_xattn_chunk_fp8(const yoco_xattn_shape* shape, const void* Q, const void* K8, const void* V8,
+                             const float* k_scale_host, const float* v_scale_host,
+                             const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O, float* lse,
+                             void* workspace, size_t workspace_bytes, void* stream);
+int32_t yoco_xattn_workspace_size_chunk_fp8(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
+                                            int32_t sm_count, size_t* bytes);
+
 /* (No counterpart in the paper.)  The same merge for pieces laid out piece-major: part_o [S, rows, d], part_lse [S, rows] -- what
  * an all-gather over S ranks leaves when every rank contributes its [rows, d] partial result and
  * its [rows] log-sum-exp.  Otherwise as yoco_xattn_combine. */

@@ -84,6 +84,10 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).restype = i32
         L.yoco_xattn_decode_fp8.argtypes = [ctypes.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.yoco_xattn_decode_fp8.restype = i32
+        L.yoco_xattn_chunk_fp8.argtypes = L.yoco_xattn_decode_fp8.argtypes
+        L.yoco_xattn_chunk_fp8.restype = i32
+        L.yoco_xattn_workspace_size_chunk_fp8.argtypes = [ctypes.POINTER(Shape), vp, i32, ctypes.POINTER(sz)]
+        L.yoco_xattn_workspace_size_chunk_fp8.restype = i32
         L.yoco_kv_fold_gain.argtypes = [i64, i64, vp, vp, vp, vp]
         L.yoco_kv_append.argtypes = [ctypes.POINTER(KvAppendShape), vp, vp, vp, vp, vp, vp, vp, vp]
         L.yoco_xattn_sub_bound.argtypes = [ctypes.c_int64, i32, i32]
@@ -293,6 +297,30 @@ def yoco_xattn_decode_fp8(shape: Shape, Q, K8, V8, k_scale, v_scale, cu_kv, kv_l
                                      workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     if rc != OK:
         raise YocoError(rc, "yoco_xattn_decode_fp8")
+
+
+def yoco_xattn_chunk_fp8(shape: Shape, Q, K8, V8, k_scale, v_scale, cu_kv, kv_len, O, lse, workspace,
+                         stream=None) -> None:
+    """The multi-token (tensor-core) path over an FP8 E4M3 cache with per-head scales; any T."""
+    keep_cu, p_cu = _host_i32(cu_kv)
+    keep_len, p_len = _host_i32(kv_len)
+    ks = np.ascontiguousarray(k_scale, dtype=np.float32)
+    vs = np.ascontiguousarray(v_scale, dtype=np.float32)
+    rc = lib().yoco_xattn_chunk_fp8(ctypes.byref(shape), _ptr(Q), _ptr(K8), _ptr(V8),
+                                    ctypes.c_void_p(ks.ctypes.data), ctypes.c_void_p(vs.ctypes.data), p_cu, p_len,
+                                    _ptr(O), _ptr(lse), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_chunk_fp8")
+
+
+def yoco_xattn_workspace_size_chunk_fp8(shape: Shape, kv_len, sm_count: int = 0) -> int:
+    keep, p_len = _host_i32(kv_len)
+    out = ctypes.c_size_t(0)
+    rc = lib().yoco_xattn_workspace_size_chunk_fp8(ctypes.byref(shape), p_len, sm_count, ctypes.byref(out))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_workspace_size_chunk_fp8")
+    return int(out.value)
 
 
 def yoco_kv_fold_gain(g, W, Wg, stream=None) -> None:

@@ -61,11 +61,11 @@ int32_t device_state(DeviceState** out) {
 // ---- plan cache ---------------------------------------------------------------------------
 struct PlanKey {
     yoco_xattn_shape shape;
-    int32_t sm_count, mode, max_sub;
+    int32_t sm_count, mode, max_sub, two_tiles;
     std::vector<int32_t> lens, cu, key_off, totals;
     bool operator==(const PlanKey& o) const {
         return std::memcmp(&shape, &o.shape, sizeof shape) == 0 && sm_count == o.sm_count &&
-               mode == o.mode && max_sub == o.max_sub && lens == o.lens && cu == o.cu &&
+               mode == o.mode && max_sub == o.max_sub && two_tiles == o.two_tiles && lens == o.lens && cu == o.cu &&
                key_off == o.key_off && totals == o.totals;
     }
 };
@@ -91,13 +91,14 @@ std::vector<std::shared_ptr<const ReadyPlan>> g_captured_plans;
 // alive for the caller even if another thread evicts it from the cache meanwhile.
 int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t* lens, int32_t sm_count,
                     int32_t mode, int32_t max_sub, std::shared_ptr<const ReadyPlan>& out,
-                    const int32_t* key_off = nullptr, const int32_t* totals = nullptr) {
+                    const int32_t* key_off = nullptr, const int32_t* totals = nullptr, bool two_tiles = false) {
     PlanKey key;
     std::memset(&key.shape, 0, sizeof key.shape);
     key.shape = s;
     key.sm_count = sm_count;
     key.mode = mode;
     key.max_sub = max_sub;
+    key.two_tiles = two_tiles ? 1 : 0;
     if (lens) key.lens.assign(lens, lens + s.B);
     if (cu) key.cu.assign(cu, cu + s.B + 1);
     if (key_off) key.key_off.assign(key_off, key_off + s.B);
@@ -112,7 +113,7 @@ int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t*
             }
     }
     auto ready = std::make_shared<ReadyPlan>();
-    int32_t rc = make_plan(s, cu, lens, sm_count, mode, ready->plan, max_sub, key_off, totals);
+    int32_t rc = make_plan(s, cu, lens, sm_count, mode, ready->plan, max_sub, key_off, totals, two_tiles);
     if (rc != YOCO_OK) return rc;
     const Plan& plan = ready->plan;
     ready->blob.assign(kWorkspaceHeaderBytes / 4 + plan.table.size(), 0);
@@ -290,9 +291,10 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
     std::shared_ptr<const ReadyPlan> ready;
     // The 8-bit kernel runs one piece per group: it is paced by its own instruction chains, evenly
     // on every SM, and handing out pieces made it slower (351 us against 331 us at 1M keys).
-    if (fp8) max_sub = 1;
+    if (fp8 && mode == YOCO_MODE_DECODE) max_sub = 1;
     if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, mode, max_sub, ready,
-                          shard ? shard->key_offset : nullptr, shard ? shard->kv_total : nullptr)) != YOCO_OK)
+                          shard ? shard->key_offset : nullptr, shard ? shard->kv_total : nullptr,
+                          fp8 && mode == YOCO_MODE_CHUNK)) != YOCO_OK)
         return rc;
     const Plan& plan = ready->plan;
     if ((int64_t)workspace_bytes < plan.info.workspace_bytes) return YOCO_ERR_WORKSPACE_TOO_SMALL;
@@ -380,8 +382,13 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             CUtensorMap tmQ, tmK, tmV;
             const int64_t q_rows = (int64_t)shape->B * shape->Hq * shape->T;
             if ((rc = make_map_2d(&tmQ, Q, q_rows, shape->d, kChunkTileM)) != YOCO_OK) return rc;
-            if ((rc = make_map_2d(&tmK, K, plan.kv_rows_extent, shape->d, kChunkTileN)) != YOCO_OK) return rc;
-            if ((rc = make_map_2d(&tmV, V, plan.kv_rows_extent, shape->d, kChunkTileN)) != YOCO_OK) return rc;
+            if (fp8) {
+                if ((rc = make_map_2d_u8(&tmK, K, plan.kv_rows_extent, kChunkTileN)) != YOCO_OK) return rc;
+                if ((rc = make_map_2d_u8(&tmV, V, plan.kv_rows_extent, kChunkTileN)) != YOCO_OK) return rc;
+            } else {
+                if ((rc = make_map_2d(&tmK, K, plan.kv_rows_extent, shape->d, kChunkTileN)) != YOCO_OK) return rc;
+                if ((rc = make_map_2d(&tmV, V, plan.kv_rows_extent, shape->d, kChunkTileN)) != YOCO_OK) return rc;
+            }
             ChunkParams p{};
             p.O = static_cast<__nv_bfloat16*>(O);
             p.lse = lse;
@@ -397,7 +404,15 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
             p.d = shape->d;
             p.window = shape->window;
             p.force_partial = part_out ? 1 : 0;
-            if (plan.info.tile_m == kChunkPairTileM)
+            if (fp8) {
+                ChunkFp8Scales cs{};
+                cs.Hkv = shape->Hkv;
+                for (int c = 0; c < shape->Hkv; ++c) {
+                    cs.score_scale_log2[c] = scale * fp8->k_scale[c] * 1.4426950408889634f;
+                    cs.v_scale[c] = fp8->v_scale[c];
+                }
+                YOCO_CUDA_TRY(launch_chunk_pair(p, tmQ, tmK, tmV, plan.info.num_groups, stream, &cs));
+            } else if (plan.info.tile_m == kChunkPairTileM)
                 YOCO_CUDA_TRY(launch_chunk_pair(p, tmQ, tmK, tmV, plan.info.num_groups, stream));
             else
                 YOCO_CUDA_TRY(launch_chunk(p, tmQ, tmK, tmV, plan.info.num_groups, stream));
@@ -640,6 +655,39 @@ int32_t yoco_xattn_decode_fp8(const yoco_xattn_shape* shape, const void* Q, cons
     const Fp8Scales sc{k_scale_host, v_scale_host};
     return run(shape, YOCO_MODE_DECODE, Q, K8, V8, cu_kv_host, kv_len_host, O, lse, workspace, workspace_bytes,
                stream, nullptr, &sc);
+}
+
+int32_t yoco_xattn_chunk_fp8(const yoco_xattn_shape* shape, const void* Q, const void* K8, const void* V8,
+                             const float* k_scale_host, const float* v_scale_host, const int32_t* cu_kv_host,
+                             const int32_t* kv_len_host, void* O, float* lse, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    if (!shape || !k_scale_host || !v_scale_host) return YOCO_ERR_INVALID_ARG;
+    if (shape->d != 128 || shape->Hkv > kFp8MaxHeads) return YOCO_ERR_UNSUPPORTED;
+    for (int c = 0; c < shape->Hkv; ++c)
+        if (!(k_scale_host[c] > 0.f) || !(v_scale_host[c] > 0.f) || !std::isfinite(k_scale_host[c]) ||
+            !std::isfinite(v_scale_host[c]))
+            return YOCO_ERR_INVALID_ARG;
+    const Fp8Scales sc{k_scale_host, v_scale_host};
+    return run(shape, YOCO_MODE_CHUNK, Q, K8, V8, cu_kv_host, kv_len_host, O, lse, workspace, workspace_bytes,
+               stream, nullptr, &sc);
+}
+
+int32_t yoco_xattn_workspace_size_chunk_fp8(const yoco_xattn_shape* shape, const int32_t* kv_len_host,
+                                            int32_t sm_count, size_t* bytes) {
+    if (!shape || !bytes || sm_count < 0) return YOCO_ERR_INVALID_ARG;
+    if (sm_count == 0) {
+        int32_t rc = validate_shape(*shape, YOCO_MODE_CHUNK);
+        if (rc != YOCO_OK) return rc;
+        DeviceState* dev = nullptr;
+        if ((rc = device_state(&dev)) != YOCO_OK) return rc;
+        sm_count = dev->sm_count;
+    }
+    Plan plan;
+    int32_t rc = make_plan(*shape, nullptr, kv_len_host, sm_count, YOCO_MODE_CHUNK, plan, kMaxSubItems, nullptr, nullptr,
+                           true);
+    if (rc != YOCO_OK) return rc;
+    *bytes = (size_t)plan.info.workspace_bytes;
+    return YOCO_OK;
 }
 
 int32_t yoco_kv_fold_gain(int64_t d_model, int64_t n_out, const void* g, const void* W, void* Wg, void* stream) {

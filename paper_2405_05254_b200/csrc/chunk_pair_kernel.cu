@@ -19,6 +19,16 @@
 // the products of one thread in the order issued, so the buffer needs no barrier round trip between
 // the two.  O in tensor memory is rescaled only when a row max outgrew the reference by more than 2^8.
 // Every wait is bounded and reports through the status word.
+//
+// FP8 = true reads an 8-bit cache (FP8 E4M3 bytes, one fp32 scale per KV head, head dimension 128):
+// the producer brings a 128-key tile of bytes (16 KB) into the upper half of a ring stage, warp 3
+// widens it in place to fp16 in the layout the tensor-core descriptors read (every E4M3 value is an
+// fp16 value, so this is exact; row r of the bytes sits exactly where row r of the second 64-channel
+// half goes, so a thread only ever overwrites its own source row), Q is converted bf16 -> fp16 in
+// place once per segment, P is rounded to fp16, and all products run fp16 x fp16.  k_scale folds
+// into the softmax scale, v_scale multiplies the normalised output.
+#include <cuda_fp16.h>
+
 #include "kernels.h"
 #include "ptx.cuh"
 #include "tcgen05.cuh"
@@ -50,7 +60,7 @@ struct PCfg {
     static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
     static constexpr int OFF_V = OFF_K + K_STAGES * TILE_BYTES;
     static constexpr int OFF_BAR = OFF_V + V_STAGES * TILE_BYTES;
-    static constexpr int NUM_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 12 + 3;
+    static constexpr int NUM_BARS = 2 + 2 * K_STAGES + 2 * V_STAGES + 12 + 3 + (K_STAGES + V_STAGES + 1);
     static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16;
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
 };
@@ -62,10 +72,27 @@ __host__ __device__ constexpr bool poly_pair(int j) {
     return ((j + 1) * kPolyPairs) / 16 != (j * kPolyPairs) / 16;
 }
 
-template <int D>
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// two E4M3 bytes (low byte first) -> two fp16 (exact)
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_bytes) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"((uint16_t)two_bytes));
+    return r;
+}
+// two bf16 -> two fp16 (round to nearest; |x| < 65504 required of Q)
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
+    return pack_f16x2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+}
+
+template <int D, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                  const __grid_constant__ CUtensorMap tmV, const ChunkParams p) {
+                  const __grid_constant__ CUtensorMap tmV, const ChunkParams p,
+                  const __grid_constant__ ChunkFp8Scales sc) {
+    static_assert(!FP8 || D == 128, "the 8-bit cache path is built for head dimension 128");
     using C = PCfg<D>;
     constexpr int HALVES = C::HALVES;
     constexpr int KS = C::K_STAGES, VS = C::V_STAGES;
@@ -84,6 +111,13 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     uint64_t* p_full = s_full + 4;           // [2][2]  P_r^h has been written over S_r^h
     uint64_t* pv_done = p_full + 4;          // [2][2]  O_r includes the current half step; P_r^h is dead
     uint64_t* drain_bar = pv_done + 4;       // [3]     everything issuer warp 1 + i started has finished
+    uint64_t* k_ready = drain_bar + 3;       // [KS]    8-bit cache: the K tile has been widened to fp16
+    uint64_t* v_ready = k_ready + KS;        // [VS]    ... the V tile
+    uint64_t* q_ready = v_ready + VS;        //         ... both Q tiles have been converted to fp16
+    // what the issuers and the softmax warpgroups wait on for an operand tile
+    uint64_t* k_use = FP8 ? k_ready : k_full;
+    uint64_t* v_use = FP8 ? v_ready : v_full;
+    uint64_t* q_use = FP8 ? q_ready : q_full;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -99,6 +133,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mbar_init(q_full, 1);
         mbar_init(q_empty, 2);
         for (int b = 0; b < 3; ++b) mbar_init(&drain_bar[b], 1);
+        for (int b = 0; b < KS + VS + 1; ++b) mbar_init(&k_ready[b], 1);
         for (int b = 0; b < KS; ++b) {
             mbar_init(&k_full[b], 1);
             mbar_init(&k_empty[b], 2);            // released by both issuers
@@ -150,17 +185,27 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     const uint32_t kb = it % KS, kn = it / KS;
                     if (!(ok = wait_or_abort(&k_empty[kb], (kn & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
                     ++k_armed;
-                    mbar_expect_tx(&k_full[kb], C::TILE_BYTES);
-                    for (int h = 0; h < HALVES; ++h)
-                        tma_load_2d(smem + C::OFF_K + kb * C::TILE_BYTES + h * HALF_BYTES, &tmK, h * 64, row,
-                                    &k_full[kb]);
+                    if (FP8) {      // 128 keys x 128 bytes into the upper half of the stage
+                        mbar_expect_tx(&k_full[kb], HALF_BYTES);
+                        tma_load_2d(smem + C::OFF_K + kb * C::TILE_BYTES + HALF_BYTES, &tmK, 0, row, &k_full[kb]);
+                    } else {
+                        mbar_expect_tx(&k_full[kb], C::TILE_BYTES);
+                        for (int h = 0; h < HALVES; ++h)
+                            tma_load_2d(smem + C::OFF_K + kb * C::TILE_BYTES + h * HALF_BYTES, &tmK, h * 64, row,
+                                        &k_full[kb]);
+                    }
                     const uint32_t vb = it % VS, vn = it / VS;
                     if (!(ok = wait_or_abort(&v_empty[vb], (vn & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
                     ++v_armed;
-                    mbar_expect_tx(&v_full[vb], C::TILE_BYTES);
-                    for (int h = 0; h < HALVES; ++h)
-                        tma_load_2d(smem + C::OFF_V + vb * C::TILE_BYTES + h * HALF_BYTES, &tmV, h * 64, row,
-                                    &v_full[vb]);
+                    if (FP8) {
+                        mbar_expect_tx(&v_full[vb], HALF_BYTES);
+                        tma_load_2d(smem + C::OFF_V + vb * C::TILE_BYTES + HALF_BYTES, &tmV, 0, row, &v_full[vb]);
+                    } else {
+                        mbar_expect_tx(&v_full[vb], C::TILE_BYTES);
+                        for (int h = 0; h < HALVES; ++h)
+                            tma_load_2d(smem + C::OFF_V + vb * C::TILE_BYTES + h * HALF_BYTES, &tmV, h * 64, row,
+                                        &v_full[vb]);
+                    }
                 }
             }
             // Every copy this thread started must have landed before the CTA may end (at once when all
@@ -181,8 +226,8 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             // schedule (addresses and descriptors stay warp-uniform) and one elected lane issues:
             // issued from a diverged lane the same instructions cost several times as much.
             const int r = warp - 1;
-            constexpr uint32_t idesc_qk = make_idesc(BH, false);
-            constexpr uint32_t idesc_pv = make_idesc(D, true);
+            constexpr uint32_t idesc_qk = make_idesc(BH, false, FP8);
+            constexpr uint32_t idesc_pv = make_idesc(D, true, FP8);
             const uint32_t sbase = smem_u32(smem);
             const uint32_t q_lo = desc_lo(sbase + C::OFF_Q + r * C::TILE_BYTES, 16);
             const uint32_t tmem_o = tmem_base + 2 * BN + r * BN;
@@ -214,16 +259,16 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 const int n_tiles = (p.segments[si].k_end - p.segments[si].k_begin + BN - 1) / BN;
                 if (n_tiles <= 0) continue;
                 // both halves of the first key tile of the segment (its Q and K have to be there)
-                if (!(ok = warp_wait(q_full, n_seg & 1u, ab, kWaitRingFull))) break;
+                if (!(ok = warp_wait(q_use, n_seg & 1u, ab, kWaitRingFull))) break;
                 ++n_seg;
-                if (!(ok = warp_wait(&k_full[it % KS], (it / KS) & 1u, ab, kWaitRingFull))) break;
+                if (!(ok = warp_wait(&k_use[it % KS], (it / KS) & 1u, ab, kWaitRingFull))) break;
                 issue_scores(it, 0, n_tiles == 1);
                 issue_scores(it, 1, n_tiles == 1);
                 for (int t = 0; t < n_tiles && ok; ++t, ++it) {
                     const uint32_t vb = it % VS;
-                    if (!(ok = warp_wait(&v_full[vb], (it / VS) & 1u, ab, kWaitRingFull))) break;
+                    if (!(ok = warp_wait(&v_use[vb], (it / VS) & 1u, ab, kWaitRingFull))) break;
                     const bool more = t + 1 < n_tiles;
-                    if (more && !(ok = warp_wait(&k_full[(it + 1) % KS], ((it + 1) / KS) & 1u, ab, kWaitRingFull))) break;
+                    if (more && !(ok = warp_wait(&k_use[(it + 1) % KS], ((it + 1) / KS) & 1u, ab, kWaitRingFull))) break;
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         if (!(ok = warp_wait(&p_full[r * 2 + h], it & 1u, ab, kWaitTensor))) break;
@@ -252,6 +297,66 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 drain_wait(&drain_bar[r], 0u, ab);
             }
             __syncwarp();
+        } else if (FP8 && warp == 3 && aligned_ok) {
+            // =================================== widening warp (8-bit cache) =================
+            // Lane l handles rows l, l + 32, l + 64, l + 96 of a tile.  The bytes of row r were written
+            // by TMA with the 128-byte swizzle (16-byte chunk c at position c ^ (r & 7)); the fp16 row
+            // goes out in the same swizzle, channels 0-63 to row r of the lower half tile and 64-127
+            // to row r of the upper one, i.e. over the bytes just read.
+            auto widen_tile = [&](uint8_t* tile) {
+#pragma unroll 1
+                for (int pass = 0; pass < 4; ++pass) {
+                    const int rr = pass * 32 + lane;
+                    uint8_t* src = tile + HALF_BYTES + rr * 128;
+                    uint4 raw[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) raw[c] = *reinterpret_cast<const uint4*>(src + ((c ^ (rr & 7)) << 4));
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {                 // 16 elements: channels 16 c .. 16 c + 15
+                        const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+                        uint32_t f[8];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            f[2 * q] = e4m3x2_to_f16x2(w[q]);
+                            f[2 * q + 1] = e4m3x2_to_f16x2(w[q] >> 16);
+                        }
+                        uint8_t* dst = tile + (c >> 2) * HALF_BYTES + rr * 128;
+                        const int c0 = (c & 3) * 2;
+                        *reinterpret_cast<uint4*>(dst + (((c0) ^ (rr & 7)) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
+                        *reinterpret_cast<uint4*>(dst + (((c0 + 1) ^ (rr & 7)) << 4)) = make_uint4(f[4], f[5], f[6], f[7]);
+                    }
+                }
+                fence_proxy_async_smem();                          // generic writes -> tensor core reads
+                __syncwarp();
+            };
+            uint32_t it = 0, n_seg = 0;
+            bool ok = true;
+            for (int si = seg_lo; si < seg_hi && ok; ++si) {
+                const int n_tiles = (p.segments[si].k_end - p.segments[si].k_begin + BN - 1) / BN;
+                if (n_tiles <= 0) continue;
+                // Q: bf16 -> fp16 in place (element by element, so the swizzle does not matter)
+                if (!(ok = warp_wait(q_full, n_seg & 1u, ab, kWaitRingFull))) break;
+                ++n_seg;
+#pragma unroll 1
+                for (int off = lane * 16; off < 2 * C::TILE_BYTES; off += 32 * 16) {
+                    uint4 v = *reinterpret_cast<const uint4*>(smem + C::OFF_Q + off);
+                    v.x = bf16x2_to_f16x2(v.x); v.y = bf16x2_to_f16x2(v.y);
+                    v.z = bf16x2_to_f16x2(v.z); v.w = bf16x2_to_f16x2(v.w);
+                    *reinterpret_cast<uint4*>(smem + C::OFF_Q + off) = v;
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(q_ready);
+                for (int t = 0; t < n_tiles && ok; ++t, ++it) {
+                    const uint32_t kb = it % KS, vb = it % VS;
+                    if (!(ok = warp_wait(&k_full[kb], (it / KS) & 1u, ab, kWaitRingFull))) break;
+                    widen_tile(smem + C::OFF_K + kb * C::TILE_BYTES);
+                    if (lane == 0) mbar_arrive(&k_ready[kb]);
+                    if (!(ok = warp_wait(&v_full[vb], (it / VS) & 1u, ab, kWaitRingFull))) break;
+                    widen_tile(smem + C::OFF_V + vb * C::TILE_BYTES);
+                    if (lane == 0) mbar_arrive(&v_ready[vb]);
+                }
+            }
         }
     } else {
         // ======================================= softmax warpgroups ==========================
@@ -277,6 +382,11 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const int lo_max = p.window > 0 ? n_full + p.T - 1 - p.window : 0;
             float m_ref = -INFINITY, l = 0.f;
             const uint32_t seg_first_it = it, seg_first_u = 2 * it;
+            // 8-bit cache: the key scale of this KV head folds into the softmax scale, the value scale
+            // multiplies the normalised output
+            const int head = FP8 ? seg.stream % sc.Hkv : 0;
+            const float scale_log2 = FP8 ? sc.score_scale_log2[head] : p.scale_log2;
+            const float out_scale = FP8 ? sc.v_scale[head] : 1.f;
             int pending = -1;                          // half step whose P is stored but not yet announced
 
             // The P of a half step is announced (wait for the stores, fence, arrive) only after the
@@ -316,7 +426,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
                     for (int j = 0; j < BH; j += 2) mx4[(j >> 1) & 3] = fmax3(mx4[(j >> 1) & 3], s[j], s[j + 1]);
-                    const float mx = fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * p.scale_log2;
+                    const float mx = fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * scale_log2;
                     // lazy rescale: the reference max moves only when the row max outgrew it by 2^8
                     const bool grow = mx > m_ref + kRescaleThreshold || (m_ref == -INFINITY && mx > -INFINITY);
                     if (__any_sync(0xffffffffu, grow)) {
@@ -350,7 +460,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     // the first half step, each before it releases its own first product on this tile.
                     if (h == 0 && k0 + BN > seg.n_kv) {
                         const uint32_t vb = it % VS, vn = it / VS;
-                        if (!(ok = warp_wait(&v_full[vb], vn & 1u, ab, kWaitRingFull))) continue;
+                        if (!(ok = warp_wait(&v_use[vb], vn & 1u, ab, kWaitRingFull))) continue;
                         if (k0 + row >= seg.n_kv) {
                             uint8_t* vrow = smem + C::OFF_V + vb * C::TILE_BYTES + row * 128;
 #pragma unroll 1
@@ -364,7 +474,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     // allows.  kPolyPairs of every 16 pairs take their exponential on the FMA pipe
                     // so that the special-function unit (16 results per clock per SM) is not the
                     // only limit; a masked score (-inf) comes out as exactly 0 on both routes.
-                    const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negm2 = f2_pack(neg_m, neg_m);
+                    const uint64_t scale2 = f2_pack(scale_log2, scale_log2), negm2 = f2_pack(neg_m, neg_m);
                     uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};            // packed partial row sums
 #pragma unroll
                     for (int c = 0; c < BH / 32; ++c) {                // 32 keys -> 16 packed columns
@@ -383,7 +493,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                             ls2[j & 3] = f2_add(ls2[j & 3], e2);
                             float e0, e1;
                             f2_unpack(e2, e0, e1);
-                            pk[j] = pack_bf16x2(e0, e1);
+                            pk[j] = FP8 ? pack_f16x2(e0, e1) : pack_bf16x2(e0, e1);
                         }
                         tmem_st16(tmem_s + h * BH + c * 16, pk);
                     }
@@ -404,7 +514,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             if (ok) {
                 tc_fence_after();
                 const bool has = l > 0.f;
-                const float inv = has ? 1.f / l : 0.f;
+                const float inv = has ? out_scale / l : 0.f;
                 const float lse = has ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
                 const bool final_out = seg.stream_nseg == 1 && !p.force_partial;
 #pragma unroll
@@ -454,37 +564,44 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
 }
 
-template <int D>
+template <int D, bool FP8>
 cudaError_t launch_one(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                       const CUtensorMap& tmV, int num_groups, cudaStream_t stream) {
-    chunk_pair_kernel<D><<<num_groups * p.m_tiles, kThreads, PCfg<D>::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, p);
+                       const CUtensorMap& tmV, int num_groups, cudaStream_t stream, const ChunkFp8Scales& sc) {
+    chunk_pair_kernel<D, FP8><<<num_groups * p.m_tiles, kThreads, PCfg<D>::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, p, sc);
     return cudaGetLastError();
 }
 
-
-template <int D>
+template <int D, bool FP8>
 cudaError_t setup_one() {
-    cudaError_t e = cudaFuncSetAttribute(chunk_pair_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(chunk_pair_kernel<D, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          PCfg<D>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     // the register split inside the kernel assumes the launch allocation it was written for
     cudaFuncAttributes attr;
-    if ((e = cudaFuncGetAttributes(&attr, chunk_pair_kernel<D>)) != cudaSuccess) return e;
+    if ((e = cudaFuncGetAttributes(&attr, chunk_pair_kernel<D, FP8>)) != cudaSuccess) return e;
     return attr.numRegs >= kRegsLaunch ? cudaSuccess : cudaErrorLaunchOutOfResources;
 }
 
 }  // namespace
 
 cudaError_t chunk_pair_kernel_setup() {
-    cudaError_t e = setup_one<128>();
-    return e != cudaSuccess ? e : setup_one<64>();
+    cudaError_t e = setup_one<128, false>();
+    if (e != cudaSuccess) return e;
+    if ((e = setup_one<64, false>()) != cudaSuccess) return e;
+    return setup_one<128, true>();
 }
 
 cudaError_t launch_chunk_pair(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                              const CUtensorMap& tmV, int num_groups, cudaStream_t stream) {
+                              const CUtensorMap& tmV, int num_groups, cudaStream_t stream,
+                              const ChunkFp8Scales* fp8_scales) {
     if (num_groups <= 0) return cudaSuccess;
-    return p.d == 128 ? launch_one<128>(p, tmQ, tmK, tmV, num_groups, stream)
-                      : launch_one<64>(p, tmQ, tmK, tmV, num_groups, stream);
+    if (fp8_scales) {
+        if (p.d != 128) return cudaErrorInvalidValue;
+        return launch_one<128, true>(p, tmQ, tmK, tmV, num_groups, stream, *fp8_scales);
+    }
+    const ChunkFp8Scales none{};
+    return p.d == 128 ? launch_one<128, false>(p, tmQ, tmK, tmV, num_groups, stream, none)
+                      : launch_one<64, false>(p, tmQ, tmK, tmV, num_groups, stream, none);
 }
 
 }  // namespace yoco

@@ -140,8 +140,16 @@ cudaError_t launch_chunk(const ChunkParams& p, const CUtensorMap& tmQ, const CUt
 cudaError_t chunk_kernel_setup();
 // Same interface for streams with more than 128 rows: one CTA owns two 128-row tiles (m_tiles =
 // ceil(rows_per_stream / 256)), tmQ box is still {64, 128}.
+// fp8_scales (host, may be null): K and V are an 8-bit cache (tmK / tmV then are uint8 maps over the
+// [rows, 128] byte view, box {128, kChunkTileN}); head dimension 128 only.
+struct ChunkFp8Scales {
+    int32_t Hkv;
+    float score_scale_log2[kFp8MaxHeads]; // per KV head: softmax scale * k_scale[c] * log2(e)
+    float v_scale[kFp8MaxHeads];          // per KV head
+};
 cudaError_t launch_chunk_pair(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                              const CUtensorMap& tmV, int num_groups, cudaStream_t stream);
+                              const CUtensorMap& tmV, int num_groups, cudaStream_t stream,
+                              const ChunkFp8Scales* fp8_scales = nullptr);
 cudaError_t chunk_pair_kernel_setup();
 
 // ---- writing the cache: K^ = RMSNorm(X) W_K, V^ = RMSNorm(X) W_V appended head-major ------------

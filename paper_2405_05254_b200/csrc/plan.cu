@@ -37,7 +37,7 @@ int32_t validate_layout(const yoco_xattn_shape& s, const int32_t* cu_kv_host, co
 
 int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const int32_t* kv_len_host,
                   int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items,
-                  const int32_t* key_offset_host, const int32_t* kv_total_host) {
+                  const int32_t* key_offset_host, const int32_t* kv_total_host, bool chunk_two_tiles_always) {
     int32_t rc = validate_shape(s, mode);
     if (rc != YOCO_OK) return rc;
     if (sm_count <= 0) return YOCO_ERR_INVALID_ARG;
@@ -47,7 +47,7 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     const int rows_per_stream = G * s.T;
     const int tile_n = mode == YOCO_MODE_DECODE ? kDecodeTileN : kChunkTileN;
     const int tile_m = mode == YOCO_MODE_DECODE ? kDecodeTileM
-                       : rows_per_stream > kChunkTileM ? kChunkPairTileM : kChunkTileM;
+                       : (rows_per_stream > kChunkTileM || chunk_two_tiles_always) ? kChunkPairTileM : kChunkTileM;
     const int m_tiles = (rows_per_stream + tile_m - 1) / tile_m;
     const int num_streams = s.B * s.Hkv;
 

@@ -175,10 +175,11 @@ __device__ __forceinline__ uint64_t desc_from_lo(uint32_t lo, uint32_t sbo_bytes
     const uint32_t hi = (sbo_bytes >> 4) | (1u << 14) | (2u << 29);
     return ((uint64_t)hi << 32) | lo;
 }
-// Instruction descriptor: f32 accumulate, bf16 x bf16, M = 128, given N and B major-ness.
-__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
-           ((uint32_t)(128 >> 4) << 24);
+// Instruction descriptor: f32 accumulate, bf16 x bf16 (or fp16 x fp16: both operands of one product have
+// the same type), M = 128, given N and B major-ness.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major, bool fp16 = false) {
+    return (1u << 4) | ((fp16 ? 0u : 1u) << 7) | ((fp16 ? 0u : 1u) << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
 }  // namespace yoco
