@@ -65,8 +65,10 @@ struct PCfg {
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
 };
 
-// Which of the 16 score pairs of a 32-key chunk take the polynomial exponential: spread evenly so
-// that the two instruction streams interleave.
+// Which of the 16 score pairs of a 32-key chunk take their exponential on the FMA pipe (a cubic, see
+// f2_exp2_poly) instead of the special-function unit (16 results per clock per SM), spread evenly so
+// that the two instruction streams interleave.  Measured on the 32K-cache chunk case with the turns
+// described below in place, 0 / 2 / 4 of 16: 974 / 1,055 / 1,125 TFLOP/s.
 constexpr int kPolyPairs = 4;
 __host__ __device__ constexpr bool poly_pair(int j) {
     return ((j + 1) * kPolyPairs) / 16 != (j * kPolyPairs) / 16;
@@ -372,6 +374,31 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         uint32_t it = 0;
         bool ok = aligned_ok;
 
+        // The exponentials of the two row tiles take turns.  The two softmax warps that share a
+        // scheduler (same quadrant, row tiles 0 and 1) would otherwise run their exponentials at the
+        // same time -- both are released by score products that complete back to back -- and then
+        // share the special-function unit (4 results per clock and scheduler) while the rest of their
+        // half step (fetch, row max, hand-overs) leaves it idle: measured, a 32-key group costs ~230
+        // cycles alone and 430-500 next to its neighbour.  With turns (row tile 0, row tile 1, row tile 0,
+        // ...) one warp's exponentials overlap the other's remaining work.  A turn is passed with a
+        // named barrier of the two warps: the passer arrives without waiting, the taker waits.  Both
+        // warps walk the same half steps, and a warp that has given up still takes and passes its
+        // turns, so neither can be left waiting.
+        const int bar_to_1 = 1 + quad, bar_to_0 = 5 + quad;     // barrier ids 1..8
+        auto take_turn = [&](uint32_t u) {
+            if (r == 1) named_barrier_sync(bar_to_1, 64);
+            else if (u > 0) named_barrier_sync(bar_to_0, 64);
+        };
+        uint32_t turns = 0;
+        auto pass_turn = [&]() {
+            named_barrier_arrive(r == 0 ? bar_to_1 : bar_to_0, 64);
+            ++turns;
+        };
+        auto skip_turn = [&](uint32_t u) {
+            take_turn(u);
+            pass_turn();
+        };
+
         for (int si = seg_lo; si < seg_hi; ++si) {
             const DevSegment seg = p.segments[si];
             const int n_full = seg.n_full;     // keys visible to row 0 (row t sees n_full + t), see DevSegment
@@ -387,35 +414,25 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             const int head = FP8 ? seg.stream % sc.Hkv : 0;
             const float scale_log2 = FP8 ? sc.score_scale_log2[head] : p.scale_log2;
             const float out_scale = FP8 ? sc.v_scale[head] : 1.f;
-            int pending = -1;                          // half step whose P is stored but not yet announced
-
-            // The P of a half step is announced (wait for the stores, fence, arrive) only after the
-            // scores of the next half step have been fetched: the stores then have had time to land
-            // and their latency is not paid in line.
-            auto announce = [&]() {
-                if (pending >= 0) {
-                    tmem_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&p_full[r * 2 + pending]);
-                    pending = -1;
-                }
-            };
-
             for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
 #pragma unroll 1
                 for (int h = 0; h < 2; ++h) {
-                    if (!ok) continue;
                     const uint32_t u = 2 * it + h;             // half step number
+                    if (!ok) {
+                        skip_turn(u);
+                        continue;
+                    }
                     const int kh = k0 + h * BH;                // first key of the half step
-                    if (!(ok = warp_wait(&s_full[r * 2 + h], it & 1u, ab, kWaitTensor))) continue;
+                    if (!(ok = warp_wait(&s_full[r * 2 + h], it & 1u, ab, kWaitTensor))) {
+                        skip_turn(u);
+                        continue;
+                    }
                     tc_fence_after();
                     float s[BH];
 #pragma unroll
                     for (int c = 0; c < BH / 32; ++c)
                         tmem_ld32(tmem_s + h * BH + c * 32, *reinterpret_cast<float(*)[32]>(&s[c * 32]));
                     tmem_wait_ld();
-                    announce();                                // the previous half step's P
 
                     const bool masked = !(kh + BH <= n_edge && kh >= lo_max);   // causal edge, sequence end or window start
                     if (masked) {
@@ -440,7 +457,10 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                             // O_r holds the sums of the earlier half steps of this segment: wait for
                             // the product of the previous one (the other buffer; it belongs to this key
                             // tile when h = 1, to the previous one when h = 0)
-                            if (!(ok = warp_wait(&pv_done[r * 2 + (h ^ 1)], (it ^ (h ^ 1)) & 1u, ab, kWaitTensor))) continue;
+                            if (!(ok = warp_wait(&pv_done[r * 2 + (h ^ 1)], (it ^ (h ^ 1)) & 1u, ab, kWaitTensor))) {
+                                skip_turn(u);
+                                continue;
+                            }
                             tc_fence_after();
 #pragma unroll 1
                             for (int c = 0; c < D / 32; ++c) {
@@ -460,7 +480,10 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     // the first half step, each before it releases its own first product on this tile.
                     if (h == 0 && k0 + BN > seg.n_kv) {
                         const uint32_t vb = it % VS, vn = it / VS;
-                        if (!(ok = warp_wait(&v_use[vb], vn & 1u, ab, kWaitRingFull))) continue;
+                        if (!(ok = warp_wait(&v_use[vb], vn & 1u, ab, kWaitRingFull))) {
+                            skip_turn(u);
+                            continue;
+                        }
                         if (k0 + row >= seg.n_kv) {
                             uint8_t* vrow = smem + C::OFF_V + vb * C::TILE_BYTES + row * 128;
 #pragma unroll 1
@@ -471,11 +494,10 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     }
 
                     // P = 2^(s * scale - m_ref), two elements per instruction where the hardware
-                    // allows.  kPolyPairs of every 16 pairs take their exponential on the FMA pipe
-                    // so that the special-function unit (16 results per clock per SM) is not the
-                    // only limit; a masked score (-inf) comes out as exactly 0 on both routes.
+                    // allows; a masked score (-inf) comes out as exactly 0.
                     const uint64_t scale2 = f2_pack(scale_log2, scale_log2), negm2 = f2_pack(neg_m, neg_m);
                     uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};            // packed partial row sums
+                    take_turn(u);
 #pragma unroll
                     for (int c = 0; c < BH / 32; ++c) {                // 32 keys -> 16 packed columns
                         uint32_t pk[16];
@@ -497,7 +519,14 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                         }
                         tmem_st16(tmem_s + h * BH + c * 16, pk);
                     }
-                    pending = h;
+                    pass_turn();
+                    // announce P (announcing it only after the next half step's scores had been fetched,
+                    // to keep the wait for the stores out of line, was measured slower: the product
+                    // that frees this buffer for the scores after next then starts later)
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&p_full[r * 2 + h]);
                     {
                         float a0, a1, b0, b1;
                         f2_unpack(f2_add(ls2[0], ls2[1]), a0, a1);
@@ -506,8 +535,6 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                     }
                 }
             }
-            announce();
-
             // ---- end of segment: O_r is complete once the last PV has finished ----
             // (the products of one row tile complete in order, so the last one covers all)
             if (ok && it > seg_first_it) ok = warp_wait(&pv_done[r * 2 + 1], (it - 1) & 1u, ab, kWaitTensor);
@@ -554,6 +581,9 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 tc_fence_before();
             }
         }
+        // the last turn row tile 1 passed has no taker: take it, so that no barrier is left half complete
+        if (r == 0 && turns > 0) named_barrier_sync(bar_to_0, 64);
+
     }
 
     tc_fence_before();

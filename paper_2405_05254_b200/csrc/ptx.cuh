@@ -152,6 +152,10 @@ __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// Arrival at a named barrier without waiting for it (the other side waits with named_barrier_sync).
+__device__ __forceinline__ void named_barrier_arrive(int id, int threads) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 // Barrier over `threads` threads that also ORs a predicate: every participant gets the same answer.
 __device__ __forceinline__ bool named_barrier_or(int id, int threads, bool pred) {
     uint32_t r;
