@@ -6,7 +6,7 @@ import pytest
 
 import oracle
 import synth_inputs as si
-from helpers import GpuRunner, assert_close, assert_lse_close, errors, to_dev_bf16
+from helpers import GpuRunner, assert_close, assert_lse_close, bf16_dev_to_f64, errors, to_dev_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -247,6 +247,49 @@ def test_layer_calls_replay_bit_identically_from_a_cuda_graph(lens):
         assert bd.yoco_xattn_status(ws, side) == 0
         for a, b in zip(eager, Os):
             assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+def test_a_recorded_call_with_tables_in_the_workspace_survives_plan_cache_eviction():
+    """A problem too large for kernel-parameter tables uploads them from the library's plan cache.  Recorded
+    into a graph, that copy reads the plan's host memory again at every replay, so the library keeps such a
+    plan for good: after enough other shapes to push it out of the 16-entry cache the replay must still give
+    the oracle's result.  (Where the CUDA runtime refuses to record a copy from pageable memory the call must
+    fail with an error code and leave the context usable.)"""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    w = si.Workload("graph_big", B=25, Hq=8, Hkv=8, d=128, T=1, layers=1, seed=30,
+                    kv_len=[4000 + 137 * i for i in range(25)])          # 200 streams, ~490 segments
+    Kb, Vb, Qb = w.make_k(), w.make_v(), w.make_q(0)
+    K, V, Q = to_dev_bf16(Kb), to_dev_bf16(Vb), to_dev_bf16(Qb.reshape(-1))
+    O = torch.empty(w.B * w.Hq * w.d, dtype=torch.bfloat16, device="cuda")
+    shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, 1, max_kv_len=int(w.kv_len.max()))
+    ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_DECODE), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        bd.yoco_xattn_decode(shape, Q, K, V, w.cu, w.kv_len, O, None, ws, side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    try:
+        with torch.cuda.graph(graph, stream=side):
+            bd.yoco_xattn_decode(shape, Q, K, V, w.cu, w.kv_len, O, None, ws, side)
+    except (bd.YocoError, RuntimeError) as e:
+        torch.cuda.synchronize()
+        assert int(torch.zeros(1, device="cuda").item()) == 0          # refused cleanly, context alive
+        pytest.skip(f"the runtime does not record this copy: {e}")
+    # 20 other shapes through the same entry point: the recorded plan leaves the cache
+    small = torch.zeros(64 * 8 * 128, dtype=torch.bfloat16, device="cuda")
+    for n in range(1, 21):
+        sh = bd.make_shape(1, 8, 8, 128, 1, max_kv_len=n)
+        wsn = torch.empty(bd.yoco_xattn_workspace_size(sh, [n], bd.MODE_DECODE), dtype=torch.uint8, device="cuda")
+        bd.yoco_xattn_decode(sh, small, small, small, None, [n], small.clone(), None, wsn)
+    torch.cuda.synchronize()
+    o_ref, _ = oracle_full(w, Qb, Kb, Vb)
+    for _ in range(2):
+        O.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert bd.yoco_xattn_status(ws, side) == 0
+        assert_close(bf16_dev_to_f64(O).reshape(o_ref.shape), o_ref, "replay after eviction")
 
 
 def test_calls_on_two_streams_with_their_own_workspaces_do_not_interfere():
