@@ -7,12 +7,21 @@
 //
 // The bytes are widened to fp16 in registers (cvt.rn.f16x2.e4m3x2 is exact) and the small
 // products run as m16n8k16 fp16 MMAs with fp32 accumulation; Q is converted bf16 -> fp16 once per
-// segment and P is rounded to fp16.  Because ldmatrix moves 16-bit units, a lane receives four
-// consecutive channels of a key (K) or two channels of two consecutive keys (V, transposed); the
-// reduction index of an MMA may be permuted freely as long as both operands agree, so Q is loaded
-// with the matching channel order and the output channels are put back in order when the
-// accumulators are written out.  The scales multiply the scores (k_scale, folded into the softmax
-// scale) and the output (v_scale).
+// segment and P is rounded to fp16.  With at most 16 query rows per stream the products are taken
+// transposed, keys and channels on the 16-wide side of the instruction:
+//   S^T (keys x rows)     = K (keys x channels)      Q^T
+//   O^T (channels x rows) = V^T (channels x keys)    P^T
+// so that no tensor-core row is padding when there are 8 rows or fewer: half the products of the
+// rows-on-the-16-side form, and these warp-level products are what a consumer warp spends most of
+// its time on (measured: the same kernel with half the products issued ran 6 % faster, while
+// removing two fifths of its other instructions changed nothing).  P^T comes out of the score
+// product with a key per lane group and has to become an operand with a query row per lane group: one
+// movmatrix (8 x 8 transpose of 16-bit units) per 8 keys.  Because ldmatrix moves 16-bit units, a lane
+// receives four consecutive channels of a key (K) or two channels of two consecutive keys (V,
+// transposed); the reduction index of a product may be permuted freely as long as both operands
+// agree, and so may the order of the output channels: Q is loaded with the matching channel order
+// and the output channels are put back in order when the accumulators are written out.  The
+// scales multiply the scores (k_scale, folded into the softmax scale) and the output (v_scale).
 #include <cuda_fp16.h>
 
 #include "kernels.h"
@@ -35,19 +44,27 @@ struct Cfg8 {
     static constexpr int MERGE_ML_BYTES = kConsumerWarps * ROWS * 2 * 4;
     static constexpr int BUDGET = 113 * 1024;     // two CTAs per SM
     static constexpr int STAGES_FIT = (BUDGET - MERGE_O_BYTES - MERGE_ML_BYTES - 128) / STAGE_BYTES;
-    static constexpr int STAGES = STAGES_FIT > 5 ? 5 : STAGES_FIT;
+    static constexpr int STAGES = STAGES_FIT > 6 ? 6 : STAGES_FIT;
     static_assert(STAGES >= kConsumerWarps, "every consumer warp needs a tile in flight");
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + MERGE_O_BYTES + MERGE_ML_BYTES + 128;
     static_assert(STAGES >= 2, "need at least a double buffer");
 };
 
 // D(16x8, f32) += A(16x16, f16, row) * B(16x8, f16, col)
-__device__ __forceinline__ void mma_f16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
         "{%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// 8 x 8 transpose of 16-bit units across the warp: lane (g, tq) gives row g, columns 2 tq and 2 tq + 1,
+// and receives the same positions of the transposed matrix.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
 }
 // two E4M3 bytes (low byte first) -> two fp16 (exact)
 __device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_bytes) {
@@ -59,10 +76,34 @@ __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
     __half2 v = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
-// four bf16 (two 32-bit words) -> two fp16x2 words
-__device__ __forceinline__ void bf16x4_to_f16x4(uint2 w, uint32_t& lo, uint32_t& hi) {
-    lo = pack_f16x2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u));
-    hi = pack_f16x2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
+__device__ __forceinline__ float ex2_fast(float x) {   // 2^x, one special-function op; 2^-inf = 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ void st_release_shared(uint32_t* p, uint32_t v) {
+    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_acquire_shared(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    return v;
+}
+// Waits (bounded, like every wait) until the producer's count of armed tiles has reached `want`.
+__device__ __forceinline__ bool wait_armed(const uint32_t* armed, uint32_t want, const Abort& ab) {
+    if (ld_acquire_shared(armed) >= want) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t i = 1;; ++i) {
+        if (ld_acquire_shared(armed) >= want) return true;
+        if ((i & 63u) == 0) {
+            if (*ab.flag) return false;
+            if ((int64_t)(global_timer_ns() - t0) > ab.limit_ns || i >= kWaitMaxPolls) {
+                report_give_up(ab, kWaitItemQueue);
+                return false;
+            }
+        }
+    }
 }
 
 template <int ROWS>
@@ -80,7 +121,8 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES + C::MERGE_O_BYTES + C::MERGE_ML_BYTES);
     uint64_t* empty_bar = full_bar + STAGES;
     volatile int* give_up = reinterpret_cast<volatile int*>(empty_bar + STAGES);   // some thread ran out of patience
-    static_assert(2 * STAGES * 8 + 4 <= 128, "barrier block");
+    uint32_t* armed = reinterpret_cast<uint32_t*>(empty_bar + STAGES) + 1;         // tiles the producer has armed so far
+    static_assert(2 * STAGES * 8 + 8 <= 128, "barrier block");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int seg_lo = group_begin[blockIdx.x], seg_hi = group_begin[blockIdx.x + 1];
@@ -93,6 +135,7 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
     const Abort ab{give_up, p.status, p.wait_limit_ns > 0 ? p.wait_limit_ns : kWaitLimitNs};
     if (threadIdx.x == 0) {
         *give_up = 0;
+        *armed = 0u;
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);                 // released by the one warp that read the tile
@@ -121,6 +164,7 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
                     const int row = seg.kv_row0 + (k0 - seg.k_begin);
                     tma_load_2d(kdst, &tmK, 0, row, &full_bar[stage]);
                     tma_load_2d(kdst + TENSOR_BYTES, &tmV, 0, row, &full_bar[stage]);
+                    st_release_shared(armed, it + 1);        // tiles 0 .. it have their barriers armed
                 }
             }
             // every copy this thread armed must have landed before it leaves (the CTA ends with its last
@@ -137,9 +181,10 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
     // one softmax for 64 keys instead of one per 16, which matters here because at half the bytes
     // per key the chain of dependent latencies per tile (products, shuffles, exponentials), not
     // the memory, would otherwise set the pace.  A tile is released by the one warp that read it.
+    constexpr int NT = ROWS / 8;                       // 8-row groups on the narrow side of the products
     const int g = lane >> 2, tq = lane & 3;
     const int n_rows = p.rows_per_stream;
-    // row address this lane supplies to ldmatrix.x4: matrix (lane >> 3) = (chunk pair member, key half)
+    // row address this lane supplies to ldmatrix.x4 for K: matrix (lane >> 3) = (16-byte chunk of the pair, key half)
     const int ld_key16 = ((lane >> 3) & 1) * 8 + (lane & 7);            // key row inside a 16-key group
     const int ld_chunk = lane >> 4;                                      // 0: first chunk of the pair, 1: second
     uint32_t it = 0;
@@ -150,128 +195,152 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
         const int head = seg.stream % pp.Hkv;
         const float sscale = pp.score_scale_log2[head], vscale = pp.v_scale[head];
 
-        // Q as the fp16 A operand.  Reduction step ks covers channels 16 ks .. 16 ks + 15, and this
-        // lane's four reduction slots (k = 2 tq, 2 tq + 1, 2 tq + 8, 2 tq + 9) stand for the four
-        // consecutive channels 16 ks + 4 tq + {0, 1, 2, 3}: the order in which ldmatrix hands it K bytes.
-        uint32_t qa[8][4];
-        {
-            const __nv_bfloat16* q0 = p.Q + ((int64_t)seg.q_row0 + g) * D + tq * 4;
-            const __nv_bfloat16* q1 = q0 + 8 * D;
-            const bool v0 = g < n_rows, v1 = ROWS == 16 && (g + 8) < n_rows;
+        // Q^T as the second operand of the score product (fp16).  Reduction step ks covers channels
+        // 16 ks .. 16 ks + 15, and this lane's four reduction slots (k = 2 tq, 2 tq + 1, 2 tq + 8, 2 tq + 9)
+        // stand for the four consecutive channels 16 ks + 4 tq + {0, 1, 2, 3} of query row 8 nt + g: the
+        // order in which ldmatrix hands it K bytes.
+        uint32_t qb[NT][8][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int row = 8 * nt + g;
+            const __nv_bfloat16* q = p.Q + ((int64_t)seg.q_row0 + row) * D + tq * 4;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-                const uint2 w0 = v0 ? *reinterpret_cast<const uint2*>(q0 + ks * 16) : make_uint2(0u, 0u);
-                const uint2 w1 = v1 ? *reinterpret_cast<const uint2*>(q1 + ks * 16) : make_uint2(0u, 0u);
-                bf16x4_to_f16x4(w0, qa[ks][0], qa[ks][2]);
-                bf16x4_to_f16x4(w1, qa[ks][1], qa[ks][3]);
+                const uint2 w = row < n_rows ? *reinterpret_cast<const uint2*>(q + ks * 16) : make_uint2(0u, 0u);
+                qb[nt][ks][0] = pack_f16x2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u));
+                qb[nt][ks][1] = pack_f16x2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
             }
         }
         const int n_full = seg.n_full;
         const int n_edge = min(n_full, seg.n_kv);      // tiles that end at or below it need no mask
-        const int vis0 = min(seg.n_kv, max(0, n_full + (g % p.T)));
-        const int vis1 = min(seg.n_kv, max(0, n_full + ((g + 8) % p.T)));
+        int vis[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) vis[nt][e] = min(seg.n_kv, max(0, n_full + ((8 * nt + 2 * tq + e) % p.T)));
 
-        float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-        float o[8][2][4];      // [16-channel chunk][even / odd channels][c fragment]
+        // running max and (this lane's part of the) sum of rows 8 nt + 2 tq + {0, 1}
+        float m[NT][2], l[NT][2];
+        // O^T: acc[nt][j][e] is the product tile whose channel slot i stands for channel 32 j + 2 i + e
+        // (i < 8) or 32 j + 16 + 2 (i - 8) + e: elements 0, 1 = (slot g, rows 2 tq, 2 tq + 1), elements
+        // 2, 3 = (slot g + 8, same rows)
+        float acc[NT][4][2][4];
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
+        for (int nt = 0; nt < NT; ++nt) {
+            m[nt][0] = m[nt][1] = -INFINITY;
+            l[nt][0] = l[nt][1] = 0.f;
 #pragma unroll
-            for (int h = 0; h < 2; ++h) o[c][h][0] = o[c][h][1] = o[c][h][2] = o[c][h][3] = 0.f;
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) acc[nt][j][e][0] = acc[nt][j][e][1] = acc[nt][j][e][2] = acc[nt][j][e][3] = 0.f;
+        }
 
         for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += TILE_N, ++it) {
             if (!ok || (int)(it % kConsumerWarps) != warp) continue;       // not this warp's tile
+            // A parity wait only tells the phase of a barrier apart from the one before it.  A warp
+            // that takes every fourth tile could ask for round r of a stage whose round r - 1 has not
+            // landed yet (copies complete in any order, and when a kernel starts all of them queue at
+            // once): it would be let through at once, read a tile that is still being written and
+            // release the stage a second time.  So it first waits until the producer has armed
+            // THIS tile: the producer can only have done so after the previous tile of the stage was
+            // released, i.e. after its round completed, and the barrier is then in the round asked for.
             const uint32_t stage = it % STAGES, round = it / STAGES;
-            if (!wait_or_abort(&full_bar[stage], round & 1u, ab, kWaitRingFull)) {
+            if (!wait_armed(armed, it + 1, ab) || !wait_or_abort(&full_bar[stage], round & 1u, ab, kWaitRingFull)) {
                 ok = false;         // this warp touches no tile any more; it still walks to the barriers below
                 continue;
             }
             const uint32_t kbase = smem_u32(stage_mem + stage * STAGE_BYTES);
             const uint32_t vbase = kbase + TENSOR_BYTES;
 
-            // ---- S = Q K^T for 64 keys: four 16-key groups, two n-tiles of 8 keys each ----
-            float s[8][4];
+            // ---- S^T = K Q^T for 64 keys: four 16-key groups, eight 16-channel reduction steps.
+            //      (The key groups of a step are fetched first and their products issued side by
+            //      side: products into the same accumulator wait for one another.) ----
+            float s[NT][4][4];     // [row group][16-key group]: (key g, rows 2 tq, 2 tq + 1), (key g + 8, same rows)
 #pragma unroll
-            for (int nt = 0; nt < 8; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int kg = 0; kg < 4; ++kg) {
-                const int key = kg * 16 + ld_key16;
+                for (int mt = 0; mt < 4; ++mt) s[nt][mt][0] = s[nt][mt][1] = s[nt][mt][2] = s[nt][mt][3] = 0.f;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int chunk = 2 * j + ld_chunk;
-                    uint32_t r0, r1, r2, r3;   // (keys 0-7, chunk 2j) (keys 8-15, 2j) (keys 0-7, 2j+1) (keys 8-15, 2j+1)
-                    ldmatrix_x4(kbase + key * 128 + (((chunk ^ key) & 7) << 4), r0, r1, r2, r3);
-                    mma_f16_16816(s[2 * kg], qa[2 * j], e4m3x2_to_f16x2(r0), e4m3x2_to_f16x2(r0 >> 16));
-                    mma_f16_16816(s[2 * kg + 1], qa[2 * j], e4m3x2_to_f16x2(r1), e4m3x2_to_f16x2(r1 >> 16));
-                    mma_f16_16816(s[2 * kg], qa[2 * j + 1], e4m3x2_to_f16x2(r2), e4m3x2_to_f16x2(r2 >> 16));
-                    mma_f16_16816(s[2 * kg + 1], qa[2 * j + 1], e4m3x2_to_f16x2(r3), e4m3x2_to_f16x2(r3 >> 16));
+            for (int j = 0; j < 4; ++j) {
+                const int chunk = 2 * j + ld_chunk;
+                uint32_t r[4][4];   // per key group: (keys 0-7, chunk 2 j) (keys 8-15, 2 j) (keys 0-7, 2 j + 1) (keys 8-15, 2 j + 1)
+#pragma unroll
+                for (int mt = 0; mt < 4; ++mt) {
+                    const int key = mt * 16 + ld_key16;
+                    ldmatrix_x4(kbase + key * 128 + (((chunk ^ key) & 7) << 4), r[mt][0], r[mt][1], r[mt][2], r[mt][3]);
                 }
+#pragma unroll
+                for (int h = 0; h < 2; ++h)                // chunk 2 j + h = reduction step ks
+#pragma unroll
+                    for (int mt = 0; mt < 4; ++mt) {
+                        const uint32_t lo = r[mt][2 * h], hi = r[mt][2 * h + 1];     // key g, key g + 8
+                        const uint32_t a0 = e4m3x2_to_f16x2(lo), a2 = e4m3x2_to_f16x2(lo >> 16);
+                        const uint32_t a1 = e4m3x2_to_f16x2(hi), a3 = e4m3x2_to_f16x2(hi >> 16);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt)
+                            mma_f16_16816(s[nt][mt], a0, a1, a2, a3, qb[nt][2 * j + h][0], qb[nt][2 * j + h][1]);
+                    }
             }
             // ---- scale, mask (causal edge, sequence end, window start), online softmax ----
             const bool need_mask = k0 + TILE_N > n_edge || (p.window > 0 && k0 < n_full + p.T - 1 - p.window);
-            int lo0 = -1, lo1 = -1;
-            if (need_mask && p.window > 0) {
-                lo0 = n_full + (g % p.T) - p.window;
-                lo1 = n_full + ((g + 8) % p.T) - p.window;
-            }
-            float mx0 = -INFINITY, mx1 = -INFINITY;
+            float alpha[NT][2];
+            bool any_alpha = false;
+            uint32_t pb[NT][4][2];     // P^T (fp16) as the second operand of O^T += V^T P^T: [16-key group][keys 0-7 / 8-15]
 #pragma unroll
-            for (int nt = 0; nt < 8; ++nt)
+            for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float v = s[nt][e] * sscale;
-                    if (need_mask) {
-                        const int j = k0 + nt * 8 + tq * 2 + (e & 1);
-                        v = (j < ((e & 2) ? vis1 : vis0) && j >= ((e & 2) ? lo1 : lo0)) ? v : -INFINITY;
-                    }
-                    s[nt][e] = v;
-                    if (e & 2) mx1 = fmaxf(mx1, v);
-                    else mx0 = fmaxf(mx0, v);
+                for (int e = 0; e < 2; ++e) {
+                    const int lo = (need_mask && p.window > 0) ? n_full + ((8 * nt + 2 * tq + e) % p.T) - p.window : -1;
+                    float mx = -INFINITY;
+#pragma unroll
+                    for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            float v = s[nt][mt][2 * hh + e] * sscale;
+                            if (need_mask) {
+                                const int jj = k0 + mt * 16 + hh * 8 + g;
+                                v = (jj < vis[nt][e] && jj >= lo) ? v : -INFINITY;
+                            }
+                            s[nt][mt][2 * hh + e] = v;
+                            mx = fmaxf(mx, v);
+                        }
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                    const float mn = fmaxf(m[nt][e], mx);
+                    const float ms = mn == -INFINITY ? 0.f : mn;
+                    alpha[nt][e] = ex2_fast(m[nt][e] - ms);
+                    any_alpha |= alpha[nt][e] != 1.f;
+                    m[nt][e] = mn;
+                    float sum = 0.f;
+#pragma unroll
+                    for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            const float pv = ex2_fast(s[nt][mt][2 * hh + e] - ms);
+                            s[nt][mt][2 * hh + e] = pv;
+                            sum += pv;
+                        }
+                    l[nt][e] = l[nt][e] * alpha[nt][e] + sum;
                 }
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-            const float mn0 = fmaxf(m0, mx0);
-            const float ms0 = mn0 == -INFINITY ? 0.f : mn0;
-            const float alpha0 = exp2f(m0 - ms0);
-            m0 = mn0;
-            float alpha1 = 1.f, ms1 = 0.f;
-            if (ROWS == 16) {
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-                const float mn1 = fmaxf(m1, mx1);
-                ms1 = mn1 == -INFINITY ? 0.f : mn1;
-                alpha1 = exp2f(m1 - ms1);
-                m1 = mn1;
-            }
-            // P in [0, 1], rounded to fp16, as the A operands of the four 16-key reduction steps
-            uint32_t pa[4][4];
-            float sum0 = 0.f, sum1 = 0.f;
+                // (key g, rows 2 tq, 2 tq + 1) -> (row g, keys 2 tq, 2 tq + 1), for the first and the second
+                // eight keys of every 16-key group
 #pragma unroll
-            for (int kg = 0; kg < 4; ++kg) {
-                const float p00 = exp2f(s[2 * kg][0] - ms0), p01 = exp2f(s[2 * kg][1] - ms0);
-                const float p10 = exp2f(s[2 * kg + 1][0] - ms0), p11 = exp2f(s[2 * kg + 1][1] - ms0);
-                sum0 += (p00 + p01) + (p10 + p11);
-                pa[kg][0] = pack_f16x2(p00, p01);
-                pa[kg][2] = pack_f16x2(p10, p11);
-                if (ROWS == 16) {
-                    const float q00 = exp2f(s[2 * kg][2] - ms1), q01 = exp2f(s[2 * kg][3] - ms1);
-                    const float q10 = exp2f(s[2 * kg + 1][2] - ms1), q11 = exp2f(s[2 * kg + 1][3] - ms1);
-                    sum1 += (q00 + q01) + (q10 + q11);
-                    pa[kg][1] = pack_f16x2(q00, q01);
-                    pa[kg][3] = pack_f16x2(q10, q11);
-                } else {
-                    pa[kg][1] = pa[kg][3] = 0u;
+                for (int mt = 0; mt < 4; ++mt) {
+                    pb[nt][mt][0] = movmatrix_trans(pack_f16x2(s[nt][mt][0], s[nt][mt][1]));
+                    pb[nt][mt][1] = movmatrix_trans(pack_f16x2(s[nt][mt][2], s[nt][mt][3]));
                 }
             }
-            l0 = l0 * alpha0 + sum0;
-            l1 = l1 * alpha1 + sum1;
-            if (__any_sync(0xffffffffu, alpha0 != 1.f || alpha1 != 1.f)) {
+            if (__any_sync(0xffffffffu, any_alpha)) {
 #pragma unroll
-                for (int c = 0; c < 8; ++c)
+                for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        o[c][h][0] *= alpha0; o[c][h][1] *= alpha0;
-                        o[c][h][2] *= alpha1; o[c][h][3] *= alpha1;
-                    }
+                    for (int j = 0; j < 4; ++j)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            acc[nt][j][e][0] *= alpha[nt][0]; acc[nt][j][e][1] *= alpha[nt][1];
+                            acc[nt][j][e][2] *= alpha[nt][0]; acc[nt][j][e][3] *= alpha[nt][1];
+                        }
             }
             // ---- rows past the end of the sequence may hold anything (an FP8 NaN included):
             //      zero them so that 0 * garbage cannot produce NaN in O += P V ----
@@ -283,9 +352,10 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
                         *reinterpret_cast<uint4*>(vrow + r * 128 + lane * 16) = make_uint4(0u, 0u, 0u, 0u);
                 __syncwarp();
             }
-            // ---- O += P V.  The transposed ldmatrix hands this lane, for keys 2 tq and 2 tq + 1,
-            //      the two channels 16 c + 2 g and 16 c + 2 g + 1: the even channels of a chunk
-            //      form one n-tile, the odd ones the other ----
+            // ---- O^T += V^T P^T.  The transposed ldmatrix hands this lane, for keys 2 tq and 2 tq + 1 of
+            //      an 8-key group, the two channels 2 g and 2 g + 1 of a 16-byte chunk: the even channels of
+            //      a pair of chunks form one product tile (slots 0-7 from the first chunk, 8-15 from the
+            //      second), the odd ones another ----
 #pragma unroll
             for (int kg = 0; kg < 4; ++kg) {
                 const int key = kg * 16 + ld_key16;
@@ -299,10 +369,15 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
                     r1 = __byte_perm(r1, 0u, 0x3120);
                     r2 = __byte_perm(r2, 0u, 0x3120);
                     r3 = __byte_perm(r3, 0u, 0x3120);
-                    mma_f16_16816(o[2 * j][0], pa[kg], e4m3x2_to_f16x2(r0), e4m3x2_to_f16x2(r1));
-                    mma_f16_16816(o[2 * j][1], pa[kg], e4m3x2_to_f16x2(r0 >> 16), e4m3x2_to_f16x2(r1 >> 16));
-                    mma_f16_16816(o[2 * j + 1][0], pa[kg], e4m3x2_to_f16x2(r2), e4m3x2_to_f16x2(r3));
-                    mma_f16_16816(o[2 * j + 1][1], pa[kg], e4m3x2_to_f16x2(r2 >> 16), e4m3x2_to_f16x2(r3 >> 16));
+                    const uint32_t e0 = e4m3x2_to_f16x2(r0), e1 = e4m3x2_to_f16x2(r2);          // even channels
+                    const uint32_t e2 = e4m3x2_to_f16x2(r1), e3 = e4m3x2_to_f16x2(r3);
+                    const uint32_t o0 = e4m3x2_to_f16x2(r0 >> 16), o1 = e4m3x2_to_f16x2(r2 >> 16);   // odd channels
+                    const uint32_t o2 = e4m3x2_to_f16x2(r1 >> 16), o3 = e4m3x2_to_f16x2(r3 >> 16);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        mma_f16_16816(acc[nt][j][0], e0, e1, e2, e3, pb[nt][kg][0], pb[nt][kg][1]);
+                        mma_f16_16816(acc[nt][j][1], o0, o1, o2, o3, pb[nt][kg][0], pb[nt][kg][1]);
+                    }
                 }
             }
             if (k0 + TILE_N > seg.n_kv) fence_proxy_async_smem();   // generic writes before TMA reuse
@@ -311,32 +386,28 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
         }
 
         // ---- merge the four warps' states, write the final rows or this segment's partial ----
-        l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-        l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-        if (ROWS == 16) {
-            l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-            l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-        }
         {
-            // accumulator (chunk c, even / odd tile, column 2 tq + j) is channel 16 c + 4 tq + 2 j (+ 1 if odd):
-            // this lane's four values of a chunk are four consecutive channels
             float* mo = merge_o + (warp * ROWS) * D;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                *reinterpret_cast<float4*>(mo + g * D + c * 16 + tq * 4) =
-                    make_float4(o[c][0][0], o[c][1][0], o[c][0][1], o[c][1][1]);
-                if (ROWS == 16)
-                    *reinterpret_cast<float4*>(mo + (g + 8) * D + c * 16 + tq * 4) =
-                        make_float4(o[c][0][2], o[c][1][2], o[c][0][3], o[c][1][3]);
-            }
-            if (tq == 0) {
-                merge_ml[(warp * ROWS + g) * 2] = m0;
-                merge_ml[(warp * ROWS + g) * 2 + 1] = l0;
-                if (ROWS == 16) {
-                    merge_ml[(warp * ROWS + g + 8) * 2] = m1;
-                    merge_ml[(warp * ROWS + g + 8) * 2 + 1] = l1;
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    l[nt][e] += __shfl_xor_sync(0xffffffffu, l[nt][e], 4);
+                    l[nt][e] += __shfl_xor_sync(0xffffffffu, l[nt][e], 8);
+                    l[nt][e] += __shfl_xor_sync(0xffffffffu, l[nt][e], 16);
+                    const int row = 8 * nt + 2 * tq + e;
+                    // the even and the odd tile of a chunk pair hold neighbouring channels
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh)
+                            *reinterpret_cast<float2*>(mo + row * D + 32 * j + 16 * hh + 2 * g) =
+                                make_float2(acc[nt][j][0][2 * hh + e], acc[nt][j][1][2 * hh + e]);
+                    if (g == 0) {
+                        merge_ml[(warp * ROWS + row) * 2] = m[nt][e];
+                        merge_ml[(warp * ROWS + row) * 2 + 1] = l[nt][e];
+                    }
                 }
-            }
         }
         named_barrier_sync(1, kConsumerWarps * 32);
         const bool final_out = seg.stream_nseg == 1 && !p.force_partial;
