@@ -132,8 +132,9 @@ typedef struct yoco_xattn_plan_info {
  * stream at the same rate, so CTA g runs piece 0 of its own group and the remaining pieces
  * are handed out, in item order, to whichever CTA is free.  The pieces, their slots and the
  * merge order are fixed here, so the result is the same whoever runs a piece; segments_out
- * then lists the pieces.  (yoco_xattn_decode_fp8 and yoco_xattn_decode_static run with
- * sub_items = 1.)
+ * then lists the pieces.  (yoco_xattn_decode_static runs with sub_items = 1;
+ * yoco_xattn_decode_fp8 chooses the pieces as for half as many tiles, a tile of an 8-bit cache
+ * being half the bytes.)
  * kv_len_host: [B] or NULL (every N_i = shape->max_kv_len).
  * segments_out: optional array of `capacity` entries; at most `capacity` are written,
  * info->num_segments tells how many exist.  */

@@ -61,11 +61,11 @@ int32_t device_state(DeviceState** out) {
 // ---- plan cache ---------------------------------------------------------------------------
 struct PlanKey {
     yoco_xattn_shape shape;
-    int32_t sm_count, mode, max_sub, two_tiles;
+    int32_t sm_count, mode, max_sub, eight_bit;
     std::vector<int32_t> lens, cu, key_off, totals;
     bool operator==(const PlanKey& o) const {
         return std::memcmp(&shape, &o.shape, sizeof shape) == 0 && sm_count == o.sm_count &&
-               mode == o.mode && max_sub == o.max_sub && two_tiles == o.two_tiles && lens == o.lens && cu == o.cu &&
+               mode == o.mode && max_sub == o.max_sub && eight_bit == o.eight_bit && lens == o.lens && cu == o.cu &&
                key_off == o.key_off && totals == o.totals;
     }
 };
@@ -91,14 +91,14 @@ std::vector<std::shared_ptr<const ReadyPlan>> g_captured_plans;
 // alive for the caller even if another thread evicts it from the cache meanwhile.
 int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t* lens, int32_t sm_count,
                     int32_t mode, int32_t max_sub, std::shared_ptr<const ReadyPlan>& out,
-                    const int32_t* key_off = nullptr, const int32_t* totals = nullptr, bool two_tiles = false) {
+                    const int32_t* key_off = nullptr, const int32_t* totals = nullptr, bool eight_bit = false) {
     PlanKey key;
     std::memset(&key.shape, 0, sizeof key.shape);
     key.shape = s;
     key.sm_count = sm_count;
     key.mode = mode;
     key.max_sub = max_sub;
-    key.two_tiles = two_tiles ? 1 : 0;
+    key.eight_bit = eight_bit ? 1 : 0;
     if (lens) key.lens.assign(lens, lens + s.B);
     if (cu) key.cu.assign(cu, cu + s.B + 1);
     if (key_off) key.key_off.assign(key_off, key_off + s.B);
@@ -113,7 +113,7 @@ int32_t cached_plan(const yoco_xattn_shape& s, const int32_t* cu, const int32_t*
             }
     }
     auto ready = std::make_shared<ReadyPlan>();
-    int32_t rc = make_plan(s, cu, lens, sm_count, mode, ready->plan, max_sub, key_off, totals, two_tiles);
+    int32_t rc = make_plan(s, cu, lens, sm_count, mode, ready->plan, max_sub, key_off, totals, eight_bit);
     if (rc != YOCO_OK) return rc;
     const Plan& plan = ready->plan;
     ready->blob.assign(kWorkspaceHeaderBytes / 4 + plan.table.size(), 0);
@@ -289,12 +289,9 @@ int32_t run(const yoco_xattn_shape* shape, int32_t mode, const void* Q, const vo
     if ((rc = device_state(&dev)) != YOCO_OK) return rc;
 
     std::shared_ptr<const ReadyPlan> ready;
-    // The 8-bit kernel runs one piece per group: it is paced by its own instruction chains, evenly
-    // on every SM, and handing out pieces made it slower (351 us against 331 us at 1M keys).
-    if (fp8 && mode == YOCO_MODE_DECODE) max_sub = 1;
     if ((rc = cached_plan(*shape, cu_kv_host, kv_len_host, dev->sm_count, mode, max_sub, ready,
                           shard ? shard->key_offset : nullptr, shard ? shard->kv_total : nullptr,
-                          fp8 && mode == YOCO_MODE_CHUNK)) != YOCO_OK)
+                          fp8 != nullptr)) != YOCO_OK)
         return rc;
     const Plan& plan = ready->plan;
     if ((int64_t)workspace_bytes < plan.info.workspace_bytes) return YOCO_ERR_WORKSPACE_TOO_SMALL;

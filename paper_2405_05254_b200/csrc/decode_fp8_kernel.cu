@@ -43,10 +43,10 @@ struct Cfg8 {
     static constexpr int MERGE_O_BYTES = kConsumerWarps * ROWS * D * 4;
     static constexpr int MERGE_ML_BYTES = kConsumerWarps * ROWS * 2 * 4;
     static constexpr int BUDGET = 113 * 1024;     // two CTAs per SM
-    static constexpr int STAGES_FIT = (BUDGET - MERGE_O_BYTES - MERGE_ML_BYTES - 128) / STAGE_BYTES;
+    static constexpr int STAGES_FIT = (BUDGET - MERGE_O_BYTES - MERGE_ML_BYTES - 256) / STAGE_BYTES;
     static constexpr int STAGES = STAGES_FIT > 6 ? 6 : STAGES_FIT;
     static_assert(STAGES >= kConsumerWarps, "every consumer warp needs a tile in flight");
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + MERGE_O_BYTES + MERGE_ML_BYTES + 128;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + MERGE_O_BYTES + MERGE_ML_BYTES + 256;
     static_assert(STAGES >= 2, "need at least a double buffer");
 };
 
@@ -122,10 +122,21 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
     uint64_t* empty_bar = full_bar + STAGES;
     volatile int* give_up = reinterpret_cast<volatile int*>(empty_bar + STAGES);   // some thread ran out of patience
     uint32_t* armed = reinterpret_cast<uint32_t*>(empty_bar + STAGES) + 1;         // tiles the producer has armed so far
-    static_assert(2 * STAGES * 8 + 8 <= 128, "barrier block");
+    uint64_t* item_full = empty_bar + STAGES + 1;  // [2] producer -> consumers: queue entry written
+    uint64_t* item_empty = item_full + 2;          // [2] consumers -> producer: entry read
+    volatile int32_t* item_q = reinterpret_cast<volatile int32_t*>(item_empty + 2);   // [2] item ids
+    static_assert(2 * STAGES * 8 + 8 + 32 + 8 <= 256, "barrier block");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int seg_lo = group_begin[blockIdx.x], seg_hi = group_begin[blockIdx.x + 1];
+    // Work items as in the bf16 kernel: with R = p.sub_items > 1 every group's range is cut into R
+    // pieces; CTA g starts with piece 0 of group g and its producer, once the last copy of an item
+    // is on its way, claims the next unclaimed piece from a global counter and tells the consumers
+    // through a two-entry queue, so that the ring never drains between items and a fast SM takes
+    // more pieces than a slow one.  What a piece computes and where its partial result goes is
+    // fixed by the plan.
+    const int R = p.sub_items > 1 ? p.sub_items : 1;
+    const int n_groups = gridDim.x;
+    const int n_items = n_groups * R;
     asm volatile("griddepcontrol.launch_dependents;");
 
     if ((smem_u32(smem) & 1023u) != 0) {   // the swizzle arithmetic below needs 1 KB alignment
@@ -140,6 +151,10 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);                 // released by the one warp that read the tile
         }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&item_full[s], 1);
+            mbar_init(&item_empty[s], kConsumerWarps);
+        }
         mbar_fence_init();
     }
     __syncthreads();
@@ -151,21 +166,47 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
             tma_prefetch_desc(&tmV);
             uint32_t it = 0;
             bool ok = true;
-            for (int si = seg_lo; si < seg_hi && ok; ++si) {
-                const DevSegment seg = segments[si];
-                for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += TILE_N, ++it) {
-                    const uint32_t stage = it % STAGES, round = it / STAGES;
-                    if (!wait_or_abort(&empty_bar[stage], (round & 1u) ^ 1u, ab, kWaitRingEmpty)) {
-                        ok = false;
-                        break;
-                    }
-                    uint8_t* kdst = stage_mem + stage * STAGE_BYTES;
-                    mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
-                    const int row = seg.kv_row0 + (k0 - seg.k_begin);
-                    tma_load_2d(kdst, &tmK, 0, row, &full_bar[stage]);
-                    tma_load_2d(kdst + TENSOR_BYTES, &tmV, 0, row, &full_bar[stage]);
-                    st_release_shared(armed, it + 1);        // tiles 0 .. it have their barriers armed
+            int item = blockIdx.x;
+            for (uint32_t n = 0; ok; ++n) {
+                // hand the item (or the end mark) to the consumers
+                if (!wait_or_abort(&item_empty[n & 1u], ((n >> 1) & 1u) ^ 1u, ab, kWaitItemQueue)) break;
+                item_q[n & 1u] = item;
+                mbar_arrive(&item_full[n & 1u]);
+                if (item >= n_items) break;
+                const int grp = item % n_groups, piece = item / n_groups;
+                const int seg_lo = group_begin[grp], seg_hi = group_begin[grp + 1];
+                int t_lo = 0, t_hi = 0x7fffffff, t_acc = 0;     // the piece's tiles inside the group
+                if (R > 1) {
+                    int n_g = 0;
+                    for (int si = seg_lo; si < seg_hi; ++si)
+                        n_g += (segments[si].k_end - segments[si].k_begin + TILE_N - 1) / TILE_N;
+                    t_lo = (int)sub_bound(n_g, R, piece);
+                    t_hi = (int)sub_bound(n_g, R, piece + 1);
                 }
+                for (int si = seg_lo; si < seg_hi && ok; ++si) {
+                    const DevSegment seg = segments[si];
+                    const int seg_tiles = (seg.k_end - seg.k_begin + TILE_N - 1) / TILE_N;
+                    const int s_lo = max(t_lo - t_acc, 0), s_hi = min(t_hi - t_acc, seg_tiles);
+                    t_acc += seg_tiles;
+                    if (s_lo >= s_hi) continue;
+                    const int k_lo = seg.k_begin + s_lo * TILE_N;
+                    const int k_hi = min(seg.k_begin + s_hi * TILE_N, seg.k_end);
+                    for (int k0 = k_lo; k0 < k_hi; k0 += TILE_N, ++it) {
+                        const uint32_t stage = it % STAGES, round = it / STAGES;
+                        if (!wait_or_abort(&empty_bar[stage], (round & 1u) ^ 1u, ab, kWaitRingEmpty)) {
+                            ok = false;
+                            break;
+                        }
+                        uint8_t* kdst = stage_mem + stage * STAGE_BYTES;
+                        mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
+                        const int row = seg.kv_row0 + (k0 - seg.k_begin);
+                        tma_load_2d(kdst, &tmK, 0, row, &full_bar[stage]);
+                        tma_load_2d(kdst + TENSOR_BYTES, &tmV, 0, row, &full_bar[stage]);
+                        st_release_shared(armed, it + 1);        // tiles 0 .. it have their barriers armed
+                    }
+                }
+                // all loads of this item are on their way: claim the next one
+                item = R > 1 ? n_groups + atomicAdd(p.work_counter, 1) : n_items;
             }
             // every copy this thread armed must have landed before it leaves (the CTA ends with its last
             // thread, and its shared memory then belongs to another CTA); at once when all went well
@@ -190,8 +231,38 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
     uint32_t it = 0;
     bool ok = true;
 
+    for (uint32_t n_item = 0;; ++n_item) {
+    // the next item from the producer; the four warps must take the same decision, so a warp
+    // that gives up waiting says so before the barrier and all of them leave together
+    const bool got_item = wait_or_abort(&item_full[n_item & 1u], (n_item >> 1) & 1u, ab, kWaitItemQueue);
+    const int item = item_q[n_item & 1u];
+    if (named_barrier_or(1, kConsumerWarps * 32, !got_item || !ok)) break;
+    if (lane == 0) mbar_arrive(&item_empty[n_item & 1u]);
+    if (item >= n_items) break;
+    const int grp = item % n_groups, piece = item / n_groups;
+    const int seg_lo = group_begin[grp], seg_hi = group_begin[grp + 1];
+    int t_lo = 0, t_hi = 0x7fffffff, t_acc = 0;       // the piece's tiles inside the group
+    if (R > 1) {
+        int n_g = 0;
+        for (int si = seg_lo; si < seg_hi; ++si)
+            n_g += (segments[si].k_end - segments[si].k_begin + TILE_N - 1) / TILE_N;
+        t_lo = (int)sub_bound(n_g, R, piece);
+        t_hi = (int)sub_bound(n_g, R, piece + 1);
+    }
+
     for (int si = seg_lo; si < seg_hi; ++si) {
         const DevSegment seg = segments[si];
+        const int seg_tiles = (seg.k_end - seg.k_begin + TILE_N - 1) / TILE_N;
+        const int s_lo = max(t_lo - t_acc, 0), s_hi = min(t_hi - t_acc, seg_tiles);
+        t_acc += seg_tiles;
+        const int slot = seg.slot * R + piece;
+        if (s_lo >= s_hi) {
+            // this piece holds nothing of the segment: its slot must say so to the merge
+            if (R > 1 && threadIdx.x < p.rows_per_stream) p.part_lse[(int64_t)slot * p.rows_per_stream + threadIdx.x] = -INFINITY;
+            continue;
+        }
+        const int k_lo = seg.k_begin + s_lo * TILE_N;
+        const int k_hi = min(seg.k_begin + s_hi * TILE_N, seg.k_end);
         const int head = seg.stream % pp.Hkv;
         const float sscale = pp.score_scale_log2[head], vscale = pp.v_scale[head];
 
@@ -235,7 +306,7 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
                 for (int e = 0; e < 2; ++e) acc[nt][j][e][0] = acc[nt][j][e][1] = acc[nt][j][e][2] = acc[nt][j][e][3] = 0.f;
         }
 
-        for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += TILE_N, ++it) {
+        for (int k0 = k_lo; k0 < k_hi; k0 += TILE_N, ++it) {
             if (!ok || (int)(it % kConsumerWarps) != warp) continue;       // not this warp's tile
             // A parity wait only tells the phase of a barrier apart from the one before it.  A warp
             // that takes every fourth tile could ask for round r of a stage whose round r - 1 has not
@@ -410,7 +481,7 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
                 }
         }
         named_barrier_sync(1, kConsumerWarps * 32);
-        const bool final_out = seg.stream_nseg == 1 && !p.force_partial;
+        const bool final_out = seg.stream_nseg == 1 && !p.force_partial && R == 1;
         for (int idx = threadIdx.x; idx < n_rows * D; idx += kConsumerWarps * 32) {
             const int r = idx / D, col = idx - r * D;
             float M = -INFINITY;
@@ -431,11 +502,12 @@ __device__ __forceinline__ void decode_fp8_body(const CUtensorMap& tmK, const CU
                 p.O[((int64_t)seg.q_row0 + r) * D + col] = __float2bfloat16(outv);
                 if (p.lse && col == 0) p.lse[seg.q_row0 + r] = lse;
             } else {
-                p.part_o[((int64_t)seg.slot * n_rows + r) * D + col] = outv;
-                if (col == 0) p.part_lse[(int64_t)seg.slot * n_rows + r] = lse;
+                p.part_o[((int64_t)slot * n_rows + r) * D + col] = outv;
+                if (col == 0) p.part_lse[(int64_t)slot * n_rows + r] = lse;
             }
         }
         named_barrier_sync(1, kConsumerWarps * 32);
+    }
     }
 }
 

@@ -37,7 +37,7 @@ int32_t validate_layout(const yoco_xattn_shape& s, const int32_t* cu_kv_host, co
 
 int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const int32_t* kv_len_host,
                   int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items,
-                  const int32_t* key_offset_host, const int32_t* kv_total_host, bool chunk_two_tiles_always) {
+                  const int32_t* key_offset_host, const int32_t* kv_total_host, bool eight_bit_cache) {
     int32_t rc = validate_shape(s, mode);
     if (rc != YOCO_OK) return rc;
     if (sm_count <= 0) return YOCO_ERR_INVALID_ARG;
@@ -47,7 +47,7 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     const int rows_per_stream = G * s.T;
     const int tile_n = mode == YOCO_MODE_DECODE ? kDecodeTileN : kChunkTileN;
     const int tile_m = mode == YOCO_MODE_DECODE ? kDecodeTileM
-                       : (rows_per_stream > kChunkTileM || chunk_two_tiles_always) ? kChunkPairTileM : kChunkTileM;
+                       : (rows_per_stream > kChunkTileM || eight_bit_cache) ? kChunkPairTileM : kChunkTileM;
     const int m_tiles = (rows_per_stream + tile_m - 1) / tile_m;
     const int num_streams = s.B * s.Hkv;
 
@@ -139,7 +139,7 @@ int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const in
     // Pieces pay when a group is one long run of a stream.  When groups are chains of short streams
     // (more than two segments per group on average) most streams are not split at all and are written
     // without a merge; pieces would split every one of them.
-    int R = mode == YOCO_MODE_DECODE ? choose_sub_items(total_tiles / num_groups, max_sub_items) : 1;
+    int R = mode == YOCO_MODE_DECODE ? choose_sub_items(total_tiles / num_groups / (eight_bit_cache ? 2 : 1), max_sub_items) : 1;
     if ((int64_t)dev.size() > 2 * num_groups) R = 1;
     int32_t max_splits = 0, needs_combine = R > 1 ? 1 : 0;
     for (int st = 0; st < num_streams; ++st) {

@@ -91,15 +91,17 @@ struct Plan {
 
 // Returns YOCO_OK or an error code; fills `plan`.  cu_kv_host may be null (tight packing).
 // max_sub_items: upper limit of pieces per decode group (1 = every group is one piece).
-// chunk_two_tiles_always: chunk plans use the two-row-tile CTA (kChunkPairTileM) whatever G*T is (the
-// 8-bit cache is read by that kernel only).
+// eight_bit_cache: the plan is for an 8-bit cache.  Chunk plans then use the two-row-tile CTA
+// (kChunkPairTileM) whatever G*T is (the 8-bit cache is read by that kernel only); decode plans choose
+// the pieces per group as for half as many tiles (a tile is half the bytes, and the pieces pay by bytes:
+// measured at 55 tiles per group, one piece 51.0 us, two 52.9 us).
 // key_offset_host / kv_total_host (both null, or both [B]): the cache described by kv_len_host is
 // keys [key_offset[i], key_offset[i] + kv_len[i]) of a sequence of kv_total[i] keys; the causal and
 // window masks then use the rows' positions in the whole sequence.
 int32_t make_plan(const yoco_xattn_shape& s, const int32_t* cu_kv_host, const int32_t* kv_len_host,
                   int32_t sm_count, int32_t mode, Plan& plan, int32_t max_sub_items = kMaxSubItems,
                   const int32_t* key_offset_host = nullptr, const int32_t* kv_total_host = nullptr,
-                  bool chunk_two_tiles_always = false);
+                  bool eight_bit_cache = false);
 
 int32_t validate_shape(const yoco_xattn_shape& s, int32_t mode);
 // Lengths, head stride and token offsets must describe sequences that do not overlap (pure host).
