@@ -104,30 +104,81 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             tma_prefetch_desc(&tmQ);
             tma_prefetch_desc(&tmK);
             tma_prefetch_desc(&tmV);
-            uint32_t it = 0;
-            uint32_t q_armed = 0, k_armed = 0, v_armed = 0;   // copies started, for the drain on the way out
+            // Two cursors walk the tiles of the group, one for K (which also brings a segment's Q, ahead of
+            // its first K tile) and one for V, each as far ahead as its ring has room: the score
+            // product frees a K stage long before the second product frees the V stage of the same
+            // tile, and K should not wait for V.  A stage that is not free yet is looked at again on the
+            // next turn; like every wait, the turns without progress are bounded.
+            struct Cursor {
+                int si, k0, k_end, row0;       // segment, next key, end of the segment's keys, K/V row of key 0
+                bool fresh;                    // the segment's Q has not been requested yet (K cursor)
+            };
+            auto enter = [&](Cursor& c) {      // c.si < seg_hi: read the segment
+                const DevSegment sg = p.segments[c.si];
+                c.k0 = sg.k_begin;
+                c.k_end = sg.k_end;
+                c.row0 = sg.kv_row0 - sg.k_begin;
+                c.fresh = true;
+            };
+            Cursor ck{seg_lo, 0, 0, 0, false}, cv{seg_lo, 0, 0, 0, false};
+            if (seg_lo < seg_hi) {
+                enter(ck);
+                enter(cv);
+            }
+            uint32_t q_armed = 0, k_armed = 0, v_armed = 0;   // copies started (also for the drain on the way out)
             bool ok = true;
-            for (int si = seg_lo; si < seg_hi && ok; ++si) {
-                const DevSegment seg = p.segments[si];
-                const uint32_t sidx = si - seg_lo;
-                if (!(ok = wait_or_abort(q_empty, (sidx & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
-                ++q_armed;
-                mbar_expect_tx(q_full, C::TILE_BYTES);
-                for (int h = 0; h < HALVES; ++h)
-                    tma_load_2d(smem + C::OFF_Q + h * HALF_BYTES, &tmQ, h * 64, seg.q_row0 + m_tile * BM, q_full);
-                for (int k0 = seg.k_begin; k0 < seg.k_end; k0 += BN, ++it) {
-                    const uint32_t b = it & 1u, n = it >> 1;
-                    const int row = seg.kv_row0 + (k0 - seg.k_begin);
-                    if (!(ok = wait_or_abort(&k_empty[b], (n & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
-                    ++k_armed;
-                    mbar_expect_tx(&k_full[b], C::TILE_BYTES);
-                    for (int h = 0; h < HALVES; ++h)
-                        tma_load_2d(smem + C::OFF_K + b * C::TILE_BYTES + h * HALF_BYTES, &tmK, h * 64, row, &k_full[b]);
-                    if (!(ok = wait_or_abort(&v_empty[b], (n & 1u) ^ 1u, ab, kWaitRingEmpty))) break;
-                    ++v_armed;
-                    mbar_expect_tx(&v_full[b], C::TILE_BYTES);
-                    for (int h = 0; h < HALVES; ++h)
-                        tma_load_2d(smem + C::OFF_V + b * C::TILE_BYTES + h * HALF_BYTES, &tmV, h * 64, row, &v_full[b]);
+            uint64_t t0 = global_timer_ns();
+            uint32_t idle = 0;
+            while (ok && (ck.si < seg_hi || cv.si < seg_hi)) {
+                bool moved = false;
+                if (ck.si < seg_hi) {
+                    if (ck.fresh) {            // every segment, also one without keys, gets its Q (the others wait for it)
+                        if (mbar_try_wait(q_empty, (q_armed & 1u) ^ 1u)) {
+                            ++q_armed;
+                            mbar_expect_tx(q_full, C::TILE_BYTES);
+                            for (int h = 0; h < HALVES; ++h)
+                                tma_load_2d(smem + C::OFF_Q + h * HALF_BYTES, &tmQ, h * 64,
+                                            p.segments[ck.si].q_row0 + m_tile * BM, q_full);
+                            ck.fresh = false;
+                            moved = true;
+                        }
+                    } else if (ck.k0 >= ck.k_end) {
+                        if (++ck.si < seg_hi) enter(ck);
+                        moved = true;
+                    } else if (mbar_try_wait(&k_empty[k_armed & 1u], ((k_armed >> 1) & 1u) ^ 1u)) {
+                        const uint32_t b = k_armed & 1u;
+                        ++k_armed;
+                        mbar_expect_tx(&k_full[b], C::TILE_BYTES);
+                        for (int h = 0; h < HALVES; ++h)
+                            tma_load_2d(smem + C::OFF_K + b * C::TILE_BYTES + h * HALF_BYTES, &tmK, h * 64, ck.row0 + ck.k0, &k_full[b]);
+                        ck.k0 += BN;
+                        moved = true;
+                    }
+                }
+                if (cv.si < seg_hi) {
+                    if (cv.k0 >= cv.k_end) {
+                        if (++cv.si < seg_hi) enter(cv);
+                        moved = true;
+                    } else if (mbar_try_wait(&v_empty[v_armed & 1u], ((v_armed >> 1) & 1u) ^ 1u)) {
+                        const uint32_t b = v_armed & 1u;
+                        ++v_armed;
+                        mbar_expect_tx(&v_full[b], C::TILE_BYTES);
+                        for (int h = 0; h < HALVES; ++h)
+                            tma_load_2d(smem + C::OFF_V + b * C::TILE_BYTES + h * HALF_BYTES, &tmV, h * 64, cv.row0 + cv.k0, &v_full[b]);
+                        cv.k0 += BN;
+                        moved = true;
+                    }
+                }
+                if (moved) {
+                    idle = 0;
+                } else if ((++idle & 63u) == 0) {
+                    if (idle == 64u) t0 = global_timer_ns();
+                    if (*ab.flag) {
+                        ok = false;
+                    } else if ((int64_t)(global_timer_ns() - t0) > ab.limit_ns || idle >= kWaitMaxPolls) {
+                        report_give_up(ab, kWaitRingEmpty);
+                        ok = false;
+                    }
                 }
             }
             // Every copy this thread started must have landed before the CTA may end (at once when all
@@ -261,8 +312,8 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 }
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int j = 0; j < BN; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], s[j]);
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+                for (int j = 0; j < BN; j += 2) mx4[(j >> 1) & 3] = fmax3(mx4[(j >> 1) & 3], s[j], s[j + 1]);
+                const float mx = fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * p.scale_log2;
                 // lazy rescale: the reference max moves only when the row max outgrew it by 2^8
                 float alpha = 1.f;
                 bool grow = mx > m_ref + kRescaleThreshold || (m_ref == -INFINITY && mx > -INFINITY);
@@ -293,25 +344,29 @@ chunk_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 // P buffer b is free once PV of tile it-2 has completed
                 if (!(ok = warp_wait(&p_empty[b], (n & 1u) ^ 1u, ab, kWaitTensor))) continue;
                 uint8_t* prow = smem + C::OFF_P + b * C::P_BYTES + row * 128;
-                float ls4[4] = {0.f, 0.f, 0.f, 0.f};
-                const float neg_m = -m_use;
+                // two elements per instruction where the hardware allows (packed fp32 multiply-add and add)
+                const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negm2 = f2_pack(-m_use, -m_use);
+                uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
                 for (int c = 0; c < BN / 8; ++c) {                 // 8 keys = one 16-byte chunk
-                    float e[8];
+                    uint32_t w[4];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        e[j] = ex2_approx(fmaf(s[c * 8 + j], p.scale_log2, neg_m));
-                        ls4[j & 3] += e[j];
+                    for (int j = 0; j < 4; ++j) {
+                        float x0, x1;
+                        f2_unpack(f2_fma(f2_pack(s[c * 8 + 2 * j], s[c * 8 + 2 * j + 1]), scale2, negm2), x0, x1);
+                        const float e0 = ex2_approx(x0), e1 = ex2_approx(x1);
+                        ls2[j] = f2_add(ls2[j], f2_pack(e0, e1));
+                        w[j] = pack_bf16x2(e0, e1);
                     }
-                    uint4 pk;
-                    pk.x = pack_bf16x2(e[0], e[1]);
-                    pk.y = pack_bf16x2(e[2], e[3]);
-                    pk.z = pack_bf16x2(e[4], e[5]);
-                    pk.w = pack_bf16x2(e[6], e[7]);
-                    *reinterpret_cast<uint4*>(prow + (c >> 3) * HALF_BYTES + (((c & 7) ^ (row & 7)) << 4)) = pk;
+                    *reinterpret_cast<uint4*>(prow + (c >> 3) * HALF_BYTES + (((c & 7) ^ (row & 7)) << 4)) =
+                        make_uint4(w[0], w[1], w[2], w[3]);
                 }
-                const float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-                l += lsum;
+                {
+                    float a0, a1, b0, b1;
+                    f2_unpack(f2_add(ls2[0], ls2[1]), a0, a1);
+                    f2_unpack(f2_add(ls2[2], ls2[3]), b0, b1);
+                    l += (a0 + a1) + (b0 + b1);
+                }
 
                 // keys past the end of the sequence: their V rows may hold anything; zero them so
                 // that 0 * garbage cannot make NaN
