@@ -124,6 +124,32 @@ def test_fp8_cache_decode_at_one_million_tokens():
     assert_lse_close(L.cpu().numpy().reshape(lse_ref.shape), lse_ref, "fp8 cache, 1M keys")
 
 
+@pytest.mark.parametrize("name", ["ragged", "256k"])
+def test_fp8_cache_decode_where_the_plan_cuts_pieces(name):
+    """The 8-bit-cache decode on plans with run-time work pieces other than the 1M case: the ragged batch
+    (four pieces per group, groups that span several streams, pieces that hold nothing of a segment) and one
+    sequence of 262,144 keys (two pieces per group), every head, against the oracle reading the same bytes."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    from helpers import bf16_dev_to_f64, to_dev_bf16
+    w = si.workload("ragged") if name == "ragged" else si.Workload("256k", B=1, Hq=32, Hkv=8, d=128, T=1, layers=1,
+                                                                      seed=11, kv_len=[262144])
+    K8, V8, ks, vs = w.make_kv_fp8()
+    Q = w.make_q(0)
+    shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(w.kv_len.max()))
+    n = w.B * w.Hq * w.T
+    ws = torch.empty(bd.yoco_xattn_workspace_size(shape, w.kv_len, bd.MODE_DECODE), dtype=torch.uint8, device="cuda")
+    O = torch.empty(n * w.d, dtype=torch.bfloat16, device="cuda")
+    L = torch.empty(n, dtype=torch.float32, device="cuda")
+    K8d, V8d, Qd = torch.from_numpy(K8).cuda(), torch.from_numpy(V8).cuda(), to_dev_bf16(Q.reshape(-1))
+    for _ in range(2):          # the second call finds the workspace as the first one left it
+        bd.yoco_xattn_decode_fp8(shape, Qd, K8d, V8d, ks, vs, w.cu, w.kv_len, O, L, ws)
+        assert bd.yoco_xattn_status(ws) == 0
+    o_ref, lse_ref = oracle.xattn_fp8(Q, K8, V8, ks, vs, w.cu, w.kv_len, B=w.B, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=w.T)
+    assert_close(bf16_dev_to_f64(O).reshape(o_ref.shape), o_ref, f"fp8 cache, {name}")
+    assert_lse_close(L.cpu().numpy().reshape(lse_ref.shape), lse_ref, f"fp8 cache, {name}")
+
+
 @pytest.mark.parametrize("T", [8, 32])
 def test_few_new_rows_over_a_long_cache(T):
     """T = 8 and 32 new positions per sequence (32 and 128 rows per KV head: the one-tile tensor-core
