@@ -377,6 +377,15 @@ int32_t yoco_xattn_selftest_wait_expiry(const yoco_xattn_shape* shape, const voi
                                         const void* V, const int32_t* cu_kv_host, const int32_t* kv_len_host,
                                         void* O, void* workspace, size_t workspace_bytes, int32_t limit_ms,
                                         void* stream);
+/* The same for the decode kernel of the 8-bit cache (arguments as for yoco_xattn_decode_fp8; no
+ * counterpart in the paper).  Its consumer warps take every fourth tile and first wait for the
+ * producer to have armed their tile; with a producer that arms nothing that is the wait that runs
+ * out, so the status reads YOCO_ERR_TIMEOUT with YOCO_WAIT_ITEM_QUEUE. */
+int32_t yoco_xattn_selftest_wait_expiry_fp8(const yoco_xattn_shape* shape, const void* Q, const void* K8,
+                                            const void* V8, const float* k_scale_host, const float* v_scale_host,
+                                            const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O,
+                                            void* workspace, size_t workspace_bytes, int32_t limit_ms,
+                                            void* stream);
 
 /* Measurement aid (no counterpart in the paper).  After yoco_xattn_profile_enable(n), each of
  * the next n decode/chunk calls records a CUDA event pair on its stream around the attention

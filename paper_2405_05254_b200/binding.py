@@ -406,6 +406,23 @@ def yoco_xattn_selftest_wait_expiry(shape: Shape, Q, K, V, cu_kv, kv_len, O, wor
         raise YocoError(rc, "yoco_xattn_selftest_wait_expiry")
 
 
+def yoco_xattn_selftest_wait_expiry_fp8(shape: Shape, Q, K8, V8, k_scale, v_scale, cu_kv, kv_len, O, workspace,
+                                        limit_ms: int, stream=None) -> None:
+    """The same self-test for the decode kernel of the 8-bit cache: the wait that runs out is the consumers'
+    wait for the producer to arm their tile.  O is left undefined."""
+    keep_cu, p_cu = _host_i32(cu_kv)
+    keep_len, p_len = _host_i32(kv_len)
+    ks = np.ascontiguousarray(k_scale, dtype=np.float32)
+    vs = np.ascontiguousarray(v_scale, dtype=np.float32)
+    rc = lib().yoco_xattn_selftest_wait_expiry_fp8(ctypes.byref(shape), _ptr(Q), _ptr(K8), _ptr(V8),
+                                                   ctypes.c_void_p(ks.ctypes.data), ctypes.c_void_p(vs.ctypes.data),
+                                                   p_cu, p_len, _ptr(O), _ptr(workspace),
+                                                   workspace.numel() * workspace.element_size(), int(limit_ms),
+                                                   _stream_ptr(stream))
+    if rc != OK:
+        raise YocoError(rc, "yoco_xattn_selftest_wait_expiry_fp8")
+
+
 def yoco_xattn_profile_enable(max_records: int) -> None:
     rc = lib().yoco_xattn_profile_enable(max_records)
     if rc != OK:

@@ -835,6 +835,17 @@ int32_t yoco_xattn_selftest_wait_expiry(const yoco_xattn_shape* shape, const voi
                stream, nullptr, nullptr, 1, &st);
 }
 
+int32_t yoco_xattn_selftest_wait_expiry_fp8(const yoco_xattn_shape* shape, const void* Q, const void* K8,
+                                            const void* V8, const float* k_scale_host, const float* v_scale_host,
+                                            const int32_t* cu_kv_host, const int32_t* kv_len_host, void* O,
+                                            void* workspace, size_t workspace_bytes, int32_t limit_ms, void* stream) {
+    if (limit_ms <= 0 || limit_ms > 1000 || !k_scale_host || !v_scale_host) return YOCO_ERR_INVALID_ARG;
+    const SelfTest st{(int64_t)limit_ms * 1000000ll};
+    const Fp8Scales sc{k_scale_host, v_scale_host};
+    return run(shape, YOCO_MODE_DECODE, Q, K8, V8, cu_kv_host, kv_len_host, O, nullptr, workspace, workspace_bytes,
+               stream, nullptr, &sc, 1, &st);
+}
+
 int32_t yoco_xattn_profile_enable(int32_t max_records) {
     if (max_records < 0) return YOCO_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lock(g_mutex);
