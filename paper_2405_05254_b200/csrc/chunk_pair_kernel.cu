@@ -21,7 +21,8 @@
 // Every wait is bounded and reports through the status word.
 //
 // FP8 = true reads an 8-bit cache (FP8 E4M3 bytes, one fp32 scale per KV head, head dimension 128):
-// the producer brings a 128-key tile of bytes (16 KB) into the upper half of a ring stage, warp 3
+// the producer brings a 128-key tile of bytes (16 KB) into the upper half of a ring stage, a fourth
+// warpgroup (512 threads then; one warp per scheduler, 32 rows of every tile each)
 // widens it in place to fp16 in the layout the tensor-core descriptors read (every E4M3 value is an
 // fp16 value, so this is exact; row r of the bytes sits exactly where row r of the second 64-channel
 // half goes, so a thread only ever overwrites its own source row), Q is converted bf16 -> fp16 in
@@ -40,16 +41,22 @@ namespace {
 constexpr int BM = 128;                        // rows of one tensor-core tile
 constexpr int BN = kChunkTileN;                // 128 keys per shared-memory tile
 constexpr int BH = BN / 2;                     // keys per half step
-constexpr int kThreads = 384;
+// three warpgroups for a bf16 cache; a fourth one widens the tiles of an 8-bit cache
+template <bool FP8>
+constexpr int kThreadsOf = FP8 ? 512 : 384;
 constexpr int HALF_BYTES = 128 * 128;          // 128 rows x 64 bf16: one swizzled half tile
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float kRescaleThreshold = 8.f;       // in log2 units: P stays below 2^8
-// Register split after launch.  The CTA starts with 168 registers per thread (what 384 threads
-// allow); warpgroup 0 gives back down to kRegsOther and the softmax warpgroups grow to
-// kRegsSoftmax.  The total must fit in what the CTA was launched with, or the request to grow
-// would never be granted.
-constexpr int kRegsLaunch = 168, kRegsSoftmax = 224, kRegsOther = 56;
-static_assert(128 * kRegsOther + 256 * kRegsSoftmax <= kRegsLaunch * kThreads, "register pool of the CTA");
+// Register split after launch.  The CTA starts with what its thread count allows (168 registers per
+// thread for 384 threads, 128 for 512); warpgroup 0 (and the widening warpgroup) give back down to
+// kOther / kWiden and the softmax warpgroups grow to kSoftmax.  The total must fit in what the CTA
+// was launched with, or the request to grow would never be granted.
+template <bool FP8>
+struct Regs {
+    static constexpr int kLaunch = FP8 ? 128 : 168, kSoftmax = FP8 ? 192 : 224, kOther = 56, kWiden = 64;
+    static_assert(128 * kOther + 256 * kSoftmax + (FP8 ? 128 * kWiden : 0) <= kLaunch * kThreadsOf<FP8>,
+                  "register pool of the CTA");
+};
 
 template <int D>
 struct PCfg {
@@ -90,7 +97,7 @@ __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
 }
 
 template <int D, bool FP8>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsOf<FP8>, 1)
 chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const ChunkParams p,
                   const __grid_constant__ ChunkFp8Scales sc) {
@@ -135,7 +142,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         mbar_init(q_full, 1);
         mbar_init(q_empty, 2);
         for (int b = 0; b < 3; ++b) mbar_init(&drain_bar[b], 1);
-        for (int b = 0; b < KS + VS + 1; ++b) mbar_init(&k_ready[b], 1);
+        for (int b = 0; b < KS + VS + 1; ++b) mbar_init(&k_ready[b], 4);      // the four widening warps
         for (int b = 0; b < KS; ++b) {
             mbar_init(&k_full[b], 1);
             mbar_init(&k_empty[b], 2);            // released by both issuers
@@ -163,7 +170,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp < 4) {
-        setmaxnreg_dec<kRegsOther>();
+        setmaxnreg_dec<Regs<FP8>::kOther>();
         if (warp == 0 && lane == 0 && aligned_ok) {
             // =================================== TMA producer ================================
             tma_prefetch_desc(&tmQ);
@@ -299,16 +306,22 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 drain_wait(&drain_bar[r], 0u, ab);
             }
             __syncwarp();
-        } else if (FP8 && warp == 3 && aligned_ok) {
-            // =================================== widening warp (8-bit cache) =================
-            // Lane l handles rows l, l + 32, l + 64, l + 96 of a tile.  The bytes of row r were written
-            // by TMA with the 128-byte swizzle (16-byte chunk c at position c ^ (r & 7)); the fp16 row
-            // goes out in the same swizzle, channels 0-63 to row r of the lower half tile and 64-127
-            // to row r of the upper one, i.e. over the bytes just read.
+        }
+    } else if (FP8 && warp >= 12) {
+        // ======================================= widening warpgroup (8-bit cache) ============
+        // Four warps, one per scheduler: the conversion instruction runs at a few lanes per clock and
+        // scheduler, and one warp alone could not keep up with the tensor pipe (measured: 913 TFLOP/s on
+        // the 32K-cache case with one widening warp, 1,100 with the V tiles left unwidened).  Warp w
+        // handles rows 32 w .. 32 w + 31 of every tile, one row per lane.
+        setmaxnreg_dec<Regs<FP8>::kWiden>();
+        const int wq = warp - 12;
+        if (aligned_ok) {
+            // The bytes of row r were written by TMA with the 128-byte swizzle (16-byte chunk c at position
+            // c ^ (r & 7)); the fp16 row goes out in the same swizzle, channels 0-63 to row r of the lower
+            // half tile and 64-127 to row r of the upper one, i.e. over the bytes just read.
             auto widen_tile = [&](uint8_t* tile) {
-#pragma unroll 1
-                for (int pass = 0; pass < 4; ++pass) {
-                    const int rr = pass * 32 + lane;
+                {
+                    const int rr = wq * 32 + lane;
                     uint8_t* src = tile + HALF_BYTES + rr * 128;
                     uint4 raw[8];
 #pragma unroll
@@ -340,7 +353,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                 if (!(ok = warp_wait(q_full, n_seg & 1u, ab, kWaitRingFull))) break;
                 ++n_seg;
 #pragma unroll 1
-                for (int off = lane * 16; off < 2 * C::TILE_BYTES; off += 32 * 16) {
+                for (int off = (wq * 32 + lane) * 16; off < 2 * C::TILE_BYTES; off += 128 * 16) {
                     uint4 v = *reinterpret_cast<const uint4*>(smem + C::OFF_Q + off);
                     v.x = bf16x2_to_f16x2(v.x); v.y = bf16x2_to_f16x2(v.y);
                     v.z = bf16x2_to_f16x2(v.z); v.w = bf16x2_to_f16x2(v.w);
@@ -362,7 +375,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
     } else {
         // ======================================= softmax warpgroups ==========================
-        setmaxnreg_inc<kRegsSoftmax>();
+        setmaxnreg_inc<Regs<FP8>::kSoftmax>();
         const int r = (warp >> 2) - 1;                 // row tile of this warpgroup
         const int quad = warp & 3;                     // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;              // row inside the 128-row tile
@@ -597,7 +610,7 @@ chunk_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 template <int D, bool FP8>
 cudaError_t launch_one(const ChunkParams& p, const CUtensorMap& tmQ, const CUtensorMap& tmK,
                        const CUtensorMap& tmV, int num_groups, cudaStream_t stream, const ChunkFp8Scales& sc) {
-    chunk_pair_kernel<D, FP8><<<num_groups * p.m_tiles, kThreads, PCfg<D>::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, p, sc);
+    chunk_pair_kernel<D, FP8><<<num_groups * p.m_tiles, kThreadsOf<FP8>, PCfg<D>::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, p, sc);
     return cudaGetLastError();
 }
 
@@ -609,7 +622,7 @@ cudaError_t setup_one() {
     // the register split inside the kernel assumes the launch allocation it was written for
     cudaFuncAttributes attr;
     if ((e = cudaFuncGetAttributes(&attr, chunk_pair_kernel<D, FP8>)) != cudaSuccess) return e;
-    return attr.numRegs >= kRegsLaunch ? cudaSuccess : cudaErrorLaunchOutOfResources;
+    return attr.numRegs >= Regs<FP8>::kLaunch ? cudaSuccess : cudaErrorLaunchOutOfResources;
 }
 
 }  // namespace
