@@ -150,6 +150,46 @@ def test_fp8_cache_decode_where_the_plan_cuts_pieces(name):
     assert_lse_close(L.cpu().numpy().reshape(lse_ref.shape), lse_ref, f"fp8 cache, {name}")
 
 
+def test_fp8_chunk_config_sampled_rows_over_the_full_key_range():
+    """The multi-token path over the 8-bit cache at the size bench.py times it (2 x 512 new rows after
+    262,144 cached keys, a really quantised cache).  The oracle has no row-sampling entry for the 8-bit
+    cache, so a sampled row (b, t) is checked as what it is by definition: one query position that sees
+    the first N - T + t + 1 keys of its sequence -- a one-row problem over the sequence's part of the
+    cache, read in place through a head stride."""
+    import torch
+    from paper_2405_05254_b200 import binding as bd
+    from helpers import bf16_dev_to_f64, to_dev_bf16
+    w = si.workload("chunk")
+    K8, V8, ks, vs = w.make_kv_fp8()
+    Q = w.make_q(0)
+    shape = bd.make_shape(w.B, w.Hq, w.Hkv, w.d, w.T, max_kv_len=int(w.kv_len.max()))
+    n = w.B * w.Hq * w.T
+    ws = torch.empty(bd.yoco_xattn_workspace_size_chunk_fp8(shape, w.kv_len), dtype=torch.uint8, device="cuda")
+    O = torch.empty(n * w.d, dtype=torch.bfloat16, device="cuda")
+    L = torch.empty(n, dtype=torch.float32, device="cuda")
+    bd.yoco_xattn_chunk_fp8(shape, to_dev_bf16(Q.reshape(-1)), torch.from_numpy(K8).cuda(), torch.from_numpy(V8).cuda(),
+                            ks, vs, w.cu, w.kv_len, O, L, ws)
+    assert bd.yoco_xattn_status(ws) == 0
+    o = bf16_dev_to_f64(O).reshape(w.B, w.Hq, w.T, w.d)
+    lse = L.cpu().numpy().reshape(w.B, w.Hq, w.T)
+    assert np.isfinite(o).all() and np.isfinite(lse).all()
+    # the first and last row, both sides of two 128-row tile edges, and seeded draws in between
+    rng = np.random.default_rng(506)
+    ts = sorted({0, 127, 128, 383, 384, 511} | set(int(t) for t in rng.choice(np.arange(1, 511), size=6, replace=False)))
+    per_seq = w.Hkv * w.d
+    for b in range(w.B):
+        N = int(w.kv_len[b])
+        lo, hi = int(w.cu[b]) * per_seq, int(w.cu[b + 1]) * per_seq
+        Kb, Vb = K8[lo:hi], V8[lo:hi]                      # [Hkv, N, d] of this sequence
+        for t in ts:
+            vis = N - w.T + t + 1
+            o_ref, lse_ref = oracle.xattn_fp8(Q[b:b + 1, :, t:t + 1, :], Kb, Vb, ks, vs, np.array([0, N], dtype=np.int32),
+                                              np.array([vis], dtype=np.int32), B=1, Hq=w.Hq, Hkv=w.Hkv, d=w.d, T=1,
+                                              kv_head_stride=N * w.d)
+            assert_close(o[b, :, t, :], o_ref[0, :, 0, :], f"fp8 chunk row b={b} t={t}")
+            assert_lse_close(lse[b, :, t], lse_ref[0, :, 0], f"fp8 chunk row b={b} t={t}")
+
+
 @pytest.mark.parametrize("T", [8, 32])
 def test_few_new_rows_over_a_long_cache(T):
     """T = 8 and 32 new positions per sequence (32 and 128 rows per KV head: the one-tile tensor-core
